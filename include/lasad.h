@@ -1,0 +1,124 @@
+/*
+ * lasad.h -- C ABI of the B200 (sm_100a) LASAD operator library.
+ *
+ * LASAD = causal linear attention with Spatial-Aware Decay over a raster-flattened
+ * h x w token grid (the SAD recurrence and the SAD rule of Section 3.4; Algorithm 1's
+ * loop body).  Per (batch, head) a d_k x d_v state s is carried:
+ *
+ *     s_i = g_i * s_{i-1} + k_i v_i^T ,      o_i = scale * q_i^T s_i ,      s_{-1} = state_in
+ *
+ * where g_i is the head's decay constant gamma_h (data-independent decay, Section 3.3),
+ * except at a row-boundary step, where it is exactly 1.  With absolute 0-based index i,
+ * `prefix_len` leading non-grid tokens (a class token) and `grid_w` tokens per row,
+ * step i is a boundary iff
+ *
+ *     grid_w > 0  and  i >= prefix_len  and  (i - prefix_len + 1) mod grid_w == 0 ,
+ *
+ * i.e. the step that absorbs the last token of a grid row; prefix_len = 0 is the paper's
+ * rule "t mod w = 0" for 1-based t.  grid_w = 0 disables the rule (plain 1-D decay).
+ *
+ * Conventions
+ *   - Every data pointer is DEVICE memory owned by the caller and must stay valid until the
+ *     given stream has passed the call.  `lasad_params` and the ctx handle are HOST memory.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and return without synchronising.  No call allocates device memory except
+ *     lasad_create.
+ *   - Return value: LASAD_OK or a negative LASAD_ERR_*.  On an argument error nothing is
+ *     launched and no output is touched.  The library never aborts the process.
+ *   - Base pointers of q, k, v, o must be 16-byte aligned and every stride, in bytes, a
+ *     multiple of 16; the innermost (channel) dimension is contiguous.  state is contiguous
+ *     fp32 [B, H, dk, dv], 16-byte aligned.
+ *   - Supported: dk == dv in {32, 64}; dtype F32 or BF16 (q, k, v, o share it; state, decay
+ *     and all accumulation are fp32); any B, H, T >= 1.  Otherwise LASAD_ERR_UNSUPPORTED.
+ *   - One ctx is bound to one device and may be used from one host thread at a time.
+ */
+#ifndef LASAD_H_
+#define LASAD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    LASAD_OK = 0,
+    LASAD_ERR_INVALID_ARG = -1, /* NULL pointer, non-positive size, bad alignment or stride  */
+    LASAD_ERR_UNSUPPORTED = -2, /* valid but outside the supported set above                 */
+    LASAD_ERR_CUDA = -3,        /* a CUDA runtime/driver call failed (see lasad_last_cuda_error) */
+    LASAD_ERR_TIMEOUT = -4      /* a bounded device-side wait expired (see lasad_last_device_status) */
+};
+
+enum { LASAD_F32 = 0, LASAD_BF16 = 1 };
+
+/* Options for lasad_set_option. */
+enum {
+    LASAD_OPT_PREFILL_IMPL = 0, /* 0 auto, 1 CUDA-core fp32 kernel, 2 tcgen05 tensor-core kernel */
+    LASAD_OPT_PREFILL_CHUNK = 1,/* CUDA-core prefill chunk length: 0 auto, else 16/32/64          */
+    LASAD_OPT_DECODE_TPU = 2,   /* decode: threads per (b,h) state; 0 auto, else 32/64/128/256 */
+    LASAD_OPT_WAIT_LIMIT = 3    /* iteration cap of device-side waits; 0 = library default   */
+};
+
+typedef struct lasad_params {
+    int32_t B, T, H, dk, dv; /* T = tokens in this call (ignored by lasad_decode_step)        */
+    int32_t grid_w;          /* w: tokens per grid row; 0 = boundary rule off                  */
+    int32_t prefix_len;      /* P: leading non-grid tokens; 0 = the paper's literal rule       */
+    int32_t dtype;           /* LASAD_F32 or LASAD_BF16: element type of q, k, v, o            */
+    int64_t t0;              /* absolute 0-based sequence index of the call's first token      */
+    float scale;             /* multiplies o; the paper's operator has none: pass 1.0f         */
+    int32_t reserved;        /* must be 0                                                      */
+    /* element strides of the (batch, token, head) dimensions; channels are contiguous.
+       [B,T,H,d] contiguous is {T*H*d, H*d, d}.  lasad_decode_step reads [0] and [2] only.   */
+    int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];
+} lasad_params;
+
+typedef struct lasad_ctx lasad_ctx;
+
+/* Creates a context on CUDA device `device` (it owns one device status word).  The only
+ * entry point that allocates. */
+int lasad_create(lasad_ctx** out, int device);
+int lasad_destroy(lasad_ctx* ctx);
+int lasad_set_option(lasad_ctx* ctx, int option, int value);
+
+/*
+ * Full-sequence (teacher-forced) prefill: the SAD recurrence (Section 3.4) evaluated for T
+ * tokens per (batch, head) in chunk-parallel form -- intra-chunk decayed scores
+ * (Q K^T o D) V plus the carried state, D built on the fly from the tokens' (row, col)
+ * grid positions.
+ *
+ *   q, k    [B,T,H,dk]  (strided)      decay      [H] fp32, gamma_h in [0,1]
+ *   v       [B,T,H,dv]                 state_in   [B,H,dk,dv] fp32 or NULL (zero state)
+ *   o       [B,T,H,dv]  written        state_out  [B,H,dk,dv] fp32 or NULL; may alias state_in
+ */
+int lasad_forward(lasad_ctx* ctx, const lasad_params* p,
+                  const void* q, const void* k, const void* v,
+                  const float* decay, const float* state_in,
+                  void* o, float* state_out, void* cuda_stream);
+
+/*
+ * One generation step (Algorithm 1's loop body for the token at absolute index p->t0):
+ * state <- g * state + k v^T in place, o = scale * q^T state, fused in one pass over the state.
+ *
+ *   q, k [B,H,dk], v [B,H,dv], o [B,H,dv] (strides [0] and [2] of the params)
+ *   state [B,H,dk,dv] fp32, updated in place      decay [H] fp32
+ */
+int lasad_decode_step(lasad_ctx* ctx, const lasad_params* p,
+                      const void* q, const void* k, const void* v,
+                      const float* decay, float* state, void* o, void* cuda_stream);
+
+/* After the caller has synchronised the stream: 0, or LASAD_ERR_TIMEOUT if a kernel gave up a
+ * bounded wait since the last query (the flag is cleared by the query).  Synchronous copy. */
+int lasad_last_device_status(lasad_ctx* ctx, int* status);
+
+/* cudaError_t value of the last failed CUDA call on this ctx (0 if none). */
+int lasad_last_cuda_error(const lasad_ctx* ctx);
+
+/* Number of kernels this ctx has launched since creation (host-side counter). */
+uint64_t lasad_launch_count(const lasad_ctx* ctx);
+
+const char* lasad_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LASAD_H_ */

@@ -1,0 +1,223 @@
+// Host side of the LASAD C ABI: argument validation, kernel selection, launches.
+#include "../../include/lasad.h"
+#include "lasad_common.cuh"
+
+#include <cmath>
+#include <new>
+
+struct lasad_ctx {
+    int device;
+    int* d_status;        // device status word
+    int last_cuda_error;
+    uint64_t launches;
+    int opt_prefill_impl; // 0 auto, 1 simt, 2 tensor
+    int opt_prefill_chunk;
+    int opt_decode_tpu;
+    unsigned wait_limit;
+    int sm_count;
+};
+
+namespace {
+
+constexpr unsigned kDefaultWaitLimit = 20u * 1000u * 1000u;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int fail_cuda(lasad_ctx* ctx, cudaError_t e)
+{
+    ctx->last_cuda_error = (int)e;
+    return LASAD_ERR_CUDA;
+}
+
+// Shape / dtype / stride checks shared by both entry points.
+int check_common(const lasad_ctx* ctx, const lasad_params* p, bool decode)
+{
+    if (!ctx || !p) return LASAD_ERR_INVALID_ARG;
+    if (p->B <= 0 || p->H <= 0 || p->dk <= 0 || p->dv <= 0) return LASAD_ERR_INVALID_ARG;
+    if (!decode && p->T <= 0) return LASAD_ERR_INVALID_ARG;
+    if (p->grid_w < 0 || p->prefix_len < 0 || p->t0 < 0 || p->reserved != 0) return LASAD_ERR_INVALID_ARG;
+    if (!std::isfinite(p->scale)) return LASAD_ERR_INVALID_ARG;
+    if (p->dtype != LASAD_F32 && p->dtype != LASAD_BF16) return LASAD_ERR_INVALID_ARG;
+    const int64_t esz = p->dtype == LASAD_F32 ? 4 : 2;
+    const int64_t* strides[4] = {p->q_stride, p->k_stride, p->v_stride, p->o_stride};
+    for (int s = 0; s < 4; ++s) {
+        for (int d = 0; d < 3; ++d) {
+            if (decode && d == 1) continue;
+            const int64_t st = strides[s][d];
+            if (st < 0 || (st * esz) % 16 != 0) return LASAD_ERR_INVALID_ARG;
+        }
+        const int width = (s < 2) ? p->dk : p->dv;
+        if (strides[s][2] < width && p->H > 1) return LASAD_ERR_INVALID_ARG;
+    }
+    if (p->dk != p->dv || (p->dk != 32 && p->dk != 64)) return LASAD_ERR_UNSUPPORTED;
+    if ((int64_t)p->B * p->H > 0x7fffffffLL) return LASAD_ERR_UNSUPPORTED;
+    return LASAD_OK;
+}
+
+void fill_args(lasad::KernelArgs& a, const lasad_ctx* ctx, const lasad_params* p)
+{
+    a.B = p->B; a.T = p->T; a.H = p->H;
+    a.grid_w = p->grid_w; a.prefix_len = p->prefix_len; a.t0 = p->t0; a.scale = p->scale;
+    for (int d = 0; d < 3; ++d) {
+        a.qs[d] = p->q_stride[d]; a.ks[d] = p->k_stride[d];
+        a.vs[d] = p->v_stride[d]; a.os[d] = p->o_stride[d];
+    }
+    a.status = ctx->d_status;
+    a.wait_limit = ctx->wait_limit;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lasad_create(lasad_ctx** out, int device)
+{
+    if (!out) return LASAD_ERR_INVALID_ARG;
+    *out = nullptr;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) return LASAD_ERR_CUDA;
+    lasad_ctx* ctx = new (std::nothrow) lasad_ctx();
+    if (!ctx) return LASAD_ERR_CUDA;
+    ctx->device = device;
+    ctx->wait_limit = kDefaultWaitLimit;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, 256);
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    cudaSetDevice(prev);
+    if (e != cudaSuccess) {
+        delete ctx;
+        return LASAD_ERR_CUDA;
+    }
+    *out = ctx;
+    return LASAD_OK;
+}
+
+int lasad_destroy(lasad_ctx* ctx)
+{
+    if (!ctx) return LASAD_ERR_INVALID_ARG;
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    delete ctx;
+    return LASAD_OK;
+}
+
+int lasad_set_option(lasad_ctx* ctx, int option, int value)
+{
+    if (!ctx) return LASAD_ERR_INVALID_ARG;
+    switch (option) {
+        case LASAD_OPT_PREFILL_IMPL:
+            if (value < 0 || value > 2) return LASAD_ERR_INVALID_ARG;
+            ctx->opt_prefill_impl = value;
+            return LASAD_OK;
+        case LASAD_OPT_PREFILL_CHUNK:
+            if (value != 0 && value != 16 && value != 32 && value != 64) return LASAD_ERR_INVALID_ARG;
+            ctx->opt_prefill_chunk = value;
+            return LASAD_OK;
+        case LASAD_OPT_DECODE_TPU:
+            if (value != 0 && value != 32 && value != 64 && value != 128 && value != 256)
+                return LASAD_ERR_INVALID_ARG;
+            ctx->opt_decode_tpu = value;
+            return LASAD_OK;
+        case LASAD_OPT_WAIT_LIMIT:
+            if (value < 0) return LASAD_ERR_INVALID_ARG;
+            ctx->wait_limit = value == 0 ? kDefaultWaitLimit : (unsigned)value;
+            return LASAD_OK;
+        default:
+            return LASAD_ERR_INVALID_ARG;
+    }
+}
+
+int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
+                  const float* decay, const float* state_in, void* o, float* state_out,
+                  void* cuda_stream)
+{
+    int rc = check_common(ctx, p, false);
+    if (rc != LASAD_OK) return rc;
+    if (!q || !k || !v || !o || !decay) return LASAD_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return LASAD_ERR_INVALID_ARG;
+    if ((state_in && !aligned16(state_in)) || (state_out && !aligned16(state_out)))
+        return LASAD_ERR_INVALID_ARG;
+
+    lasad::KernelArgs a{};
+    fill_args(a, ctx, p);
+    a.q = q; a.k = k; a.v = v; a.o = o;
+    a.decay = decay; a.state_in = state_in; a.state_out = state_out;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const bool bf16 = p->dtype == LASAD_BF16;
+
+    int impl = ctx->opt_prefill_impl;
+    if (impl == 0) impl = 1;
+    if (impl == 2) return LASAD_ERR_UNSUPPORTED;
+    int chunk = ctx->opt_prefill_chunk;
+    if (chunk == 0) chunk = p->dk == 64 ? 32 : 64;
+    if (p->T <= 16) chunk = 16;
+    const cudaError_t e = lasad::launch_prefill_simt(a, p->dk, p->dv, bf16, chunk, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    ctx->launches += 1;
+    return LASAD_OK;
+}
+
+int lasad_decode_step(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k,
+                      const void* v, const float* decay, float* state, void* o, void* cuda_stream)
+{
+    int rc = check_common(ctx, p, true);
+    if (rc != LASAD_OK) return rc;
+    if (!q || !k || !v || !o || !decay || !state) return LASAD_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(state))
+        return LASAD_ERR_INVALID_ARG;
+
+    lasad::KernelArgs a{};
+    fill_args(a, ctx, p);
+    a.T = 1;
+    a.q = q; a.k = k; a.v = v; a.o = o;
+    a.decay = decay; a.state_in = state; a.state_out = state;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // SAD rule (Algorithm 1's if-statement): the decay is 1 on a row-boundary step
+    const bool decay_on = !lasad::is_boundary_step(p->t0, p->grid_w, p->prefix_len);
+    int tpu = ctx->opt_decode_tpu;
+    if (tpu == 0) {
+        // few states: spread each over a whole CTA so that all of its loads are in flight at
+        // once; many states: fewer threads per state, more states per CTA
+        const long long units = (long long)p->B * p->H;
+        tpu = units >= 16LL * ctx->sm_count ? 128 : 256;
+    }
+    const cudaError_t e = lasad::launch_decode(a, p->dk, p->dv, p->dtype == LASAD_BF16, decay_on, tpu, st);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    ctx->launches += 1;
+    return LASAD_OK;
+}
+
+int lasad_last_device_status(lasad_ctx* ctx, int* status)
+{
+    if (!ctx || !status) return LASAD_ERR_INVALID_ARG;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(ctx->device);
+    int hv = 0;
+    cudaError_t e = cudaMemcpy(&hv, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && hv != 0) e = cudaMemset(ctx->d_status, 0, sizeof(int));
+    cudaSetDevice(prev);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    *status = hv != 0 ? LASAD_ERR_TIMEOUT : LASAD_OK;
+    return LASAD_OK;
+}
+
+int lasad_last_cuda_error(const lasad_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+uint64_t lasad_launch_count(const lasad_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* lasad_strerror(int code)
+{
+    switch (code) {
+        case LASAD_OK: return "ok";
+        case LASAD_ERR_INVALID_ARG: return "invalid argument (null pointer, size, alignment or stride)";
+        case LASAD_ERR_UNSUPPORTED: return "unsupported configuration (need dk == dv in {32, 64}, f32 or bf16)";
+        case LASAD_ERR_CUDA: return "CUDA call failed";
+        case LASAD_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown error code";
+    }
+}
+
+}  // extern "C"

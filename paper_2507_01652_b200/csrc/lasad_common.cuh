@@ -1,0 +1,64 @@
+// Shared device/host helpers of the LASAD CUDA library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lasad {
+
+// What every kernel needs to know about one call (host fills it from lasad_params).
+struct KernelArgs {
+    int B, T, H;
+    int grid_w;      // w; 0 = boundary rule off
+    int prefix_len;  // P
+    long long t0;    // absolute index of the call's first token
+    float scale;
+    long long qs[3], ks[3], vs[3], os[3];  // element strides for (b, t, h)
+    const void* q;
+    const void* k;
+    const void* v;
+    void* o;
+    const float* decay;     // [H]
+    const float* state_in;  // [B,H,dk,dv] or nullptr
+    float* state_out;       // [B,H,dk,dv] or nullptr
+    int* status;            // device status word (bounded waits report here)
+    unsigned wait_limit;
+};
+
+// Number of decaying (non-boundary) steps among absolute indices 0..i, from the token's 2-D
+// grid position alone (SAD rule, Section 3.4): a step decays unless it absorbs the last token
+// of a grid row.  Prefix tokens always decay.  The decay between tokens s < t of one head is
+// gamma^(steps(t) - steps(s)); with (row, col) of each this difference equals
+// (row_t-row_s)(w-1) + (col_t-col_s) - [col_t = w-1] + [col_s = w-1].
+__host__ __device__ inline long long decay_steps_upto(long long i, int grid_w, int prefix_len)
+{
+    if (i < 0) return 0;
+    if (grid_w <= 0 || i < prefix_len) return i + 1;
+    const long long j = i - prefix_len;
+    const long long row = j / grid_w;
+    const int col = (int)(j - row * grid_w);
+    return prefix_len + row * (grid_w - 1) + col + (col == grid_w - 1 ? 0 : 1);
+}
+
+__host__ __device__ inline bool is_boundary_step(long long i, int grid_w, int prefix_len)
+{
+    return grid_w > 0 && i >= prefix_len && ((i - prefix_len + 1) % grid_w) == 0;
+}
+
+template <typename T> struct io;
+template <> struct io<float> {
+    __device__ static float load(const float* p) { return *p; }
+    __device__ static void store(float* p, float x) { *p = x; }
+};
+template <> struct io<__nv_bfloat16> {
+    __device__ static float load(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    __device__ static void store(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+};
+
+// Launchers implemented in the kernel files; each returns the cudaError_t of its launch.
+cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool decay_on, int tpu,
+                          cudaStream_t st);
+cudaError_t launch_prefill_simt(const KernelArgs& a, int dk, int dv, bool bf16, int chunk,
+                                cudaStream_t st);
+
+}  // namespace lasad

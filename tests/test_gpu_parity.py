@@ -1,0 +1,250 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle.
+
+Tolerances (max|err| / max|ref| over the whole tensor): 1e-4 for fp32 I/O, 2e-2 for bf16 I/O
+with fp32 accumulation; the same bounds for the fp32 state.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2507_01652_b200 import binding, workloads
+from tests._util import TOL, oracle, rel_err, to64
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = [1]  # 1 = CUDA-core fp32 kernel, 2 = tcgen05 tensor-core kernel (added when built)
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Lasad(0)
+    yield c
+    c.close()
+
+
+def _dev(*ts):
+    return [None if t is None else t.cuda() for t in ts]
+
+
+def _supported(impl, dtype, d):
+    return impl == 1 or (dtype == torch.bfloat16 and d == 64)
+
+
+def _forward(ctx, impl, *args, chunk=0, **kw):
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, impl)
+    ctx.set_option(binding.LASAD_OPT_PREFILL_CHUNK, chunk)
+    try:
+        out = ctx.lasad_forward(*args, **kw)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        return out
+    finally:
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
+        ctx.set_option(binding.LASAD_OPT_PREFILL_CHUNK, 0)
+
+
+def _small(name, B, H):
+    return workloads.WORKLOADS[name].scaled(B=B, H=H)
+
+
+# ------------------------------------------------------------------------------------------
+# config 1 in full: fp32 prefill, 256 decode steps, state agreement
+# ------------------------------------------------------------------------------------------
+def test_config1_prefill_and_decode_full(ctx):
+    wl = workloads.WORKLOADS["config1"]
+    q, k, v = workloads.make_qkv(wl)
+    g = workloads.make_decay(wl)
+    o_ref, s_ref = oracle(q, k, v, g, wl.grid_w, form="recurrent")
+    o_quad, s_quad = oracle(q, k, v, g, wl.grid_w, form="quadratic")
+    np.testing.assert_allclose(o_ref, o_quad, rtol=1e-10, atol=1e-12)
+    dq, dk_, dv_, dg = _dev(q, k, v, g)
+    o, s = _forward(ctx, 1, dq, dk_, dv_, dg, wl.grid_w)
+    assert rel_err(o, o_ref) <= TOL[torch.float32]
+    assert rel_err(s, s_ref) <= TOL[torch.float32]
+    # decode from the zero state, token by token
+    state = torch.zeros(wl.B, wl.H, wl.d, wl.d, device="cuda")
+    outs = []
+    for t in range(wl.T):
+        outs.append(ctx.lasad_decode_step(dq[:, t], dk_[:, t], dv_[:, t], dg, state, wl.grid_w, 0, t))
+    torch.cuda.synchronize()
+    od = torch.stack(outs, 1)
+    assert rel_err(od, o_ref) <= TOL[torch.float32]
+    assert rel_err(state, s_ref) <= TOL[torch.float32]
+    # decode state after N steps equals prefill's final state
+    assert rel_err(state, to64(s)) <= TOL[torch.float32]
+
+
+# ------------------------------------------------------------------------------------------
+# the bf16 configurations at oracle-sized batch, every prefill kernel
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("name,B,H", [("config2", 2, 12), ("config3", 2, 4), ("config4", 3, 5),
+                                      ("config5a", 1, 2)])
+def test_bf16_configs_prefill(ctx, impl, name, B, H):
+    wl = _small(name, B, H)
+    q, k, v = workloads.make_qkv(wl)
+    g = workloads.make_decay(wl)
+    o_ref, s_ref = oracle(q, k, v, g, wl.grid_w, wl.prefix_len)
+    o, s = _forward(ctx, impl, *_dev(q, k, v, g), wl.grid_w, prefix_len=wl.prefix_len)
+    assert rel_err(o, o_ref) <= TOL[torch.bfloat16]
+    assert rel_err(s, s_ref) <= TOL[torch.bfloat16]
+
+
+@pytest.mark.parametrize("name,B,H", [("config2", 2, 12), ("config4", 2, 20)])
+def test_bf16_decode_sweep_matches_oracle_and_prefill(ctx, name, B, H):
+    wl = _small(name, B, H)
+    q, k, v = workloads.make_qkv(wl)
+    g = workloads.make_decay(wl)
+    o_ref, s_ref = oracle(q, k, v, g, wl.grid_w, wl.prefix_len)
+    dq, dk_, dv_, dg = _dev(q, k, v, g)
+    P = wl.prefix_len
+    # class-token prefix through prefill (T = P), then one decode step per grid token
+    if P:
+        o0, state = _forward(ctx, 1, dq[:, :P], dk_[:, :P], dv_[:, :P], dg, wl.grid_w, prefix_len=P)
+        assert rel_err(o0, o_ref[:, :P]) <= TOL[torch.bfloat16]
+    else:
+        state = torch.zeros(wl.B, wl.H, wl.d, wl.d, device="cuda")
+    outs = []
+    for t in range(P, wl.T):
+        outs.append(ctx.lasad_decode_step(dq[:, t], dk_[:, t], dv_[:, t], dg, state, wl.grid_w, P, t))
+    torch.cuda.synchronize()
+    od = torch.stack(outs, 1)
+    assert rel_err(od, o_ref[:, P:]) <= TOL[torch.bfloat16]
+    assert rel_err(state, s_ref) <= TOL[torch.bfloat16]
+    for impl in IMPLS:
+        _, s_pre = _forward(ctx, impl, dq, dk_, dv_, dg, wl.grid_w, prefix_len=P)
+        assert rel_err(state, to64(s_pre)) <= TOL[torch.bfloat16]
+
+
+# ------------------------------------------------------------------------------------------
+# ragged lengths, several tiles, both head sizes, both dtypes, every chunk size
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d", [32, 64])
+@pytest.mark.parametrize("T,w,P", [(1, 4, 0), (2, 2, 0), (3, 1, 0), (17, 5, 0), (64, 8, 0),
+                                   (100, 7, 1), (129, 16, 0), (257, 16, 1), (300, 0, 0), (391, 23, 3)])
+def test_ragged_shapes(ctx, impl, dtype, d, T, w, P):
+    if not _supported(impl, dtype, d):
+        pytest.skip("tensor-core prefill covers bf16, d = 64")
+    gen = torch.Generator().manual_seed(1000 + T + d)
+    B, H = 2, 3
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / d ** 0.5).to(dtype) for _ in range(3)]
+    g = torch.tensor([0.8, 0.95, 0.999])
+    s_in = torch.randn(B, H, d, d, generator=gen)
+    o_ref, s_ref = oracle(q, k, v, g, w, P, 5, 0.5, s_in)
+    for chunk in ([0, 16, 32, 64] if impl == 1 else [0]):
+        o, s = _forward(ctx, impl, *_dev(q, k, v, g), w, prefix_len=P, t0=5, scale=0.5,
+                        state_in=s_in.cuda(), chunk=chunk)
+        assert rel_err(o, o_ref) <= TOL[dtype], f"chunk {chunk}"
+        assert rel_err(s, s_ref) <= TOL[dtype], f"chunk {chunk}"
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_decay_edge_cases(ctx, impl):
+    """gamma = 0 (state wiped except across boundary steps), gamma = 1 (plain causal linear
+    attention), and a mix, on a grid whose rows straddle chunk borders."""
+    B, T, H, d, w = 1, 150, 4, 64, 9
+    gen = torch.Generator().manual_seed(7)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+    g = torch.tensor([0.0, 1.0, 0.5, 0.9999])
+    o_ref, s_ref = oracle(q, k, v, g, w)
+    o, s = _forward(ctx, impl, *_dev(q, k, v, g), w)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(s).all()
+    for h in range(H):
+        assert rel_err(o[:, :, h], o_ref[:, :, h]) <= TOL[torch.bfloat16], f"head {h}"
+        assert rel_err(s[:, h], s_ref[:, h]) <= TOL[torch.bfloat16], f"head {h}"
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_state_handoff_mid_row(ctx, impl):
+    """forward(0..T) == forward(0..m) then forward(m..T) from the carried state (t0 = m)."""
+    wl = _small("config3", 1, 3)
+    q, k, v = workloads.make_qkv(wl)
+    g = workloads.make_decay(wl)
+    dq, dk_, dv_, dg = _dev(q, k, v, g)
+    o_ref, s_ref = oracle(q, k, v, g, wl.grid_w)
+    for m in (1, 37, 128, 300, 575):
+        o1, s1 = _forward(ctx, impl, dq[:, :m], dk_[:, :m], dv_[:, :m], dg, wl.grid_w)
+        o2, s2 = _forward(ctx, impl, dq[:, m:], dk_[:, m:], dv_[:, m:], dg, wl.grid_w, t0=m, state_in=s1,
+                          state_out=s1)  # in-place state
+        assert rel_err(torch.cat([o1, o2], 1), o_ref) <= TOL[torch.bfloat16]
+        assert rel_err(s2, s_ref) <= TOL[torch.bfloat16]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_head_major_layout_through_strides(ctx, impl):
+    """[B,H,T,d] storage viewed as [B,T,H,d]: only the strides change."""
+    B, T, H, d, w = 2, 96, 3, 64, 12
+    gen = torch.Generator().manual_seed(11)
+    q, k, v = [(torch.randn(B, H, T, d, generator=gen) / 8).to(torch.bfloat16).cuda().transpose(1, 2)
+               for _ in range(3)]
+    g = torch.tensor([0.9, 0.99, 0.7])
+    o_ref, _ = oracle(q, k, v, g, w)
+    o_store = torch.empty(B, H, T, d, dtype=torch.bfloat16, device="cuda").transpose(1, 2)
+    o, _ = _forward(ctx, impl, q, k, v, g.cuda(), w, o=o_store)
+    assert not q.is_contiguous()
+    assert rel_err(o, o_ref) <= TOL[torch.bfloat16]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_outputs_stay_inside_their_buffers_and_are_deterministic(ctx, impl):
+    B, T, H, d, w = 2, 77, 3, 64, 8
+    gen = torch.Generator().manual_seed(12)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16).cuda() for _ in range(3)]
+    g = torch.tensor([0.9, 0.99, 0.7]).cuda()
+    pad = 4096
+    obuf = torch.full((B * T * H * d + 2 * pad,), 7.0, dtype=torch.bfloat16, device="cuda")
+    sbuf = torch.full((B * H * d * d + 2 * pad,), 7.0, dtype=torch.float32, device="cuda")
+    o = obuf[pad:-pad].view(B, T, H, d)
+    s = sbuf[pad:-pad].view(B, H, d, d)
+    _forward(ctx, impl, q, k, v, g, w, o=o, state_out=s)
+    assert (obuf[:pad] == 7).all() and (obuf[-pad:] == 7).all()
+    assert (sbuf[:pad] == 7).all() and (sbuf[-pad:] == 7).all()
+    o2, s2 = _forward(ctx, impl, q, k, v, g, w)
+    assert torch.equal(o, o2) and torch.equal(s, s2)
+
+
+def test_decode_every_thread_mapping(ctx):
+    B, H, w = 3, 5, 4
+    gen = torch.Generator().manual_seed(13)
+    for dtype in (torch.float32, torch.bfloat16):
+        for d in (32, 64):
+            q, k, v = [(torch.randn(B, 1, H, d, generator=gen) / d ** 0.5).to(dtype) for _ in range(3)]
+            g = torch.rand(H, generator=gen)
+            s_in = torch.randn(B, H, d, d, generator=gen)
+            for t in (2, 3):  # t = 3 is a boundary step for w = 4
+                o_ref, s_ref = oracle(q, k, v, g, w, 0, t, 0.25, s_in)
+                for tpu in (0, 32, 64, 128, 256):
+                    ctx.set_option(binding.LASAD_OPT_DECODE_TPU, tpu)
+                    state = s_in.clone().cuda()
+                    dq, dk_, dv_, dg = _dev(q[:, 0], k[:, 0], v[:, 0], g)
+                    o = ctx.lasad_decode_step(dq, dk_, dv_, dg, state, w, 0, t, scale=0.25)
+                    torch.cuda.synchronize()
+                    assert rel_err(o, o_ref[:, 0]) <= TOL[dtype]
+                    assert rel_err(state, s_ref) <= 1e-6
+    ctx.set_option(binding.LASAD_OPT_DECODE_TPU, 0)
+
+
+def test_argument_errors_launch_nothing(ctx):
+    B, T, H, d = 1, 8, 2, 64
+    q = torch.zeros(B, T, H, d, dtype=torch.bfloat16, device="cuda")
+    g = torch.ones(H, device="cuda")
+    n0 = ctx.launch_count
+    with pytest.raises(binding.LasadError) as e:
+        ctx.lasad_forward(q, q, q, g, -1)
+    assert e.value.code == binding.LASAD_ERR_INVALID_ARG
+    q48 = torch.zeros(B, T, H, 48, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.LasadError) as e:
+        ctx.lasad_forward(q48, q48, q48, g, 4)
+    assert e.value.code == binding.LASAD_ERR_UNSUPPORTED
+    with pytest.raises(binding.LasadError) as e:  # misaligned base pointer
+        flat = torch.zeros(B * T * H * d + 8, dtype=torch.bfloat16, device="cuda")
+        qm = flat[1:1 + B * T * H * d].view(B, T, H, d)
+        ctx.lasad_forward(qm, q, q, g, 4)
+    assert e.value.code == binding.LASAD_ERR_INVALID_ARG
+    with pytest.raises(ValueError):
+        ctx.lasad_forward(q.cpu(), q, q, g, 4)
+    assert ctx.launch_count == n0

@@ -1,0 +1,432 @@
+#!/usr/bin/env python
+"""LASAD operator benchmark on B200: prefill tokens/s and decode us/step against the rooflines.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A *step* is one full-sequence prefill (`lasad_forward`) over the prefill workload; the headline
+`value` is prefill tokens/s with inputs resident in HBM.  The same run then times the decode
+workload (`lasad_decode_step`, one sweep = one step per grid position against the persistent
+fp32 state) in its own region and reports it under "decode".  One JSON line goes to stdout.
+
+Multi-GPU (torchrun, one rank per GPU): the operator has no cross-(batch, head) term, so every
+rank runs the same per-GPU workload on its own seed with no data-path collective ("weak"
+scaling); the time is the max over ranks and `value` sums all ranks' tokens.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) from the ncu captures
+# summarised under profiles/; None until a capture of that kernel exists.
+NCU_TRAFFIC_BYTES = {"prefill": None, "decode": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "source": "measured"}
+    return {**FALLBACK_PEAKS, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------------------------
+# clocks under load (read-only NVML polling in a thread)
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+               0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, device_index: int, period_s: float = 0.004):
+        self.period = period_s
+        self.samples, self.reason_bits = [], 0
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            self._nv = pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # NVML unavailable: report that instead of inventing numbers
+            self.error = repr(e)
+            self._h = None
+
+    def _poll(self):
+        nv = self._nv
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.reason_bits |= int(get_reasons(self._h))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._stop.clear()
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+            self._thread = None
+
+    def summary(self):
+        if self._h is None or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [],
+                    "note": "NVML clocks unavailable: " + getattr(self, "error", "no samples")}
+        reasons = sorted(name for bit, name in self.REASONS.items() if self.reason_bits & bit)
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------------------------
+# algorithmic traffic
+# --------------------------------------------------------------------------------------------
+def prefill_bytes(wl) -> int:
+    """q, k, v read once and o written once, plus the final fp32 state."""
+    return wl.B * wl.T * wl.H * 4 * wl.d * wl.elem_bytes + wl.B * wl.H * wl.d * wl.d * 4
+
+
+def prefill_flops(wl, chunk: int) -> int:
+    """Executed flops of the chunked method with dense C x C tiles: 4 dk dv + 2 C (dk + dv)."""
+    return wl.B * wl.T * wl.H * (4 * wl.d * wl.d + 2 * chunk * 2 * wl.d)
+
+
+def decode_bytes(wl) -> int:
+    """fp32 state read + written, q, k, v read and o written, per step."""
+    return wl.B * wl.H * (8 * wl.d * wl.d + 4 * wl.d * wl.elem_bytes)
+
+
+# --------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2507_01652_b200 import binding, workloads
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the LASAD operator has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    peaks = load_peaks()
+    ctx = binding.Lasad(local)
+    K, W = args.steps, max(args.warmup, 3)
+    wl = workloads.WORKLOADS[args.prefill_workload]
+    wl = dataclasses.replace(wl, seed=wl.seed + 1000 * rank)
+    stream = torch.cuda.current_stream()
+
+    # ---- prefill: inputs resident in HBM -------------------------------------------------
+    hq, hk, hv = [t.pin_memory() for t in workloads.make_qkv(wl)]
+    g = workloads.make_decay(wl).to(dev)
+    q, k, v = hq.to(dev), hk.to(dev), hv.to(dev)
+    o = torch.empty_like(v)
+    s_out = torch.empty(wl.B, wl.H, wl.d, wl.d, dtype=torch.float32, device=dev)
+    fwd = lambda: ctx.lasad_forward(q, k, v, g, wl.grid_w, prefix_len=wl.prefix_len, o=o,
+                                    state_out=s_out)
+    for _ in range(W):
+        fwd()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    t_beg, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    n0 = ctx.launch_count
+    barrier()
+    with sampler:
+        t_beg.record(stream)
+        for a, b in ev:
+            a.record(stream)
+            fwd()
+            b.record(stream)
+        t_end.record(stream)
+        torch.cuda.synchronize()
+    barrier()
+    launches = ctx.launch_count - n0
+    assert ctx.device_status() == 0, "a device-side wait timed out during the timed region"
+    total_ms = max_over_ranks(t_beg.elapsed_time(t_end))
+    kern_ms = statistics.mean(a.elapsed_time(b) for a, b in ev)
+    ms_per_step = total_ms / K
+    tokens_per_step = wl.B * wl.T
+    value = world * tokens_per_step / (ms_per_step * 1e-3)
+    pf_bytes = prefill_bytes(wl)
+    achieved = pf_bytes / (kern_ms * 1e-3) / 1e9
+    chunk = args.chunk_for_flops
+    tc_tflops = prefill_flops(wl, chunk) / (kern_ms * 1e-3) / 1e12
+
+    # ---- prefill end to end: host buffers, copies inside the timed region ----------------
+    ho = torch.empty(o.shape, dtype=o.dtype).pin_memory()
+    Ke = max(3, min(K, 20))
+
+    def e2e_step():
+        q.copy_(hq, non_blocking=True)
+        k.copy_(hk, non_blocking=True)
+        v.copy_(hv, non_blocking=True)
+        fwd()
+        ho.copy_(o, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e_beg, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e_beg.record(stream)
+    for _ in range(Ke):
+        e2e_step()
+    e_end.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    e2e_ms = max_over_ranks(e_beg.elapsed_time(e_end)) / Ke
+    h2d = 3 * hq.numel() * hq.element_size()
+    d2h = ho.numel() * ho.element_size()
+    del hq, hk, hv, ho, q, k, v, o
+
+    # ---- decode sweep (config 4 shape): persistent fp32 state, one step per position ------
+    dw = workloads.WORKLOADS[args.decode_workload]
+    dw = dataclasses.replace(dw, seed=dw.seed + 1000 * rank)
+    P = dw.prefix_len
+    dq, dk_, dv_ = [t.to(dev) for t in workloads.make_qkv(dw)]
+    dg = workloads.make_decay(dw).to(dev)
+    n_sets = 3  # rotating state sets: together > 2x L2, so no step finds its state in L2
+    states = [torch.zeros(dw.B, dw.H, dw.d, dw.d, dtype=torch.float32, device=dev) for _ in range(n_sets)]
+    do = torch.empty(dw.B, dw.H, dw.d, dtype=dq.dtype, device=dev)
+    positions = list(range(P, dw.T))
+    sweeps = max(2, min(10, K // 10))
+
+    def reset_states():
+        for s_ in states:
+            if P:
+                ctx.lasad_forward(dq[:, :P], dk_[:, :P], dv_[:, :P], dg, dw.grid_w, prefix_len=P,
+                                  state_out=s_, want_state=True)
+            else:
+                s_.zero_()
+
+    def sweep(cold: bool):
+        for n, t in enumerate(positions):
+            ctx.lasad_decode_step(dq[:, t], dk_[:, t], dv_[:, t], dg, states[n % n_sets if cold else 0],
+                                  dw.grid_w, P, t, o=do)
+
+    dec = {}
+    for mode, cold in (("cold", True), ("hot", False)):
+        reset_states()
+        sweep(cold)  # warm-up sweep
+        barrier()
+        d_beg, d_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with sampler:
+            d_beg.record(stream)
+            for _ in range(sweeps):
+                sweep(cold)
+            d_end.record(stream)
+            torch.cuda.synchronize()
+        barrier()
+        us = max_over_ranks(d_beg.elapsed_time(d_end)) * 1e3 / (sweeps * len(positions))
+        dec[mode] = us
+    # the same cold sweep replayed as a CUDA graph: kernel time without per-launch host cost
+    graph_us = None
+    try:
+        reset_states()
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            sweep(True)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(gr, stream=side):
+                sweep(True)
+        torch.cuda.synchronize()
+        gr.replay()
+        barrier()
+        g_beg, g_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with sampler:
+            g_beg.record(stream)
+            for _ in range(sweeps):
+                gr.replay()
+            g_end.record(stream)
+            torch.cuda.synchronize()
+        barrier()
+        graph_us = max_over_ranks(g_beg.elapsed_time(g_end)) * 1e3 / (sweeps * len(positions))
+    except Exception as e:  # pragma: no cover - reported, never hidden
+        dec["graph_error"] = repr(e)
+    assert ctx.device_status() == 0
+    dbytes = decode_bytes(dw)
+    best_us = graph_us if graph_us is not None else dec["cold"]
+    decode = {
+        "workload": f"{dw.name}: B={dw.B} H={dw.H} d={dw.d} grid={dw.grid_h}x{dw.grid_w} prefix={P}, "
+                    f"{len(positions)} positions, bf16 q/k/v/o, fp32 state",
+        "us_per_step_cold_stream": round(dec["cold"], 3),
+        "us_per_step_hot_stream": round(dec["hot"], 3),
+        "us_per_step_cold_graph": None if graph_us is None else round(graph_us, 3),
+        "bytes_per_step": dbytes,
+        "states_rotated": n_sets,
+        "roofline": {"bound": "hbm", "achieved": round(dbytes / (best_us * 1e-6) / 1e9, 1),
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": round(dbytes / (best_us * 1e-6) / 1e9 / peaks["hbm_gbs"], 4),
+                     "traffic": NCU_TRAFFIC_BYTES["decode"], "peak_source": peaks["source"],
+                     "timed": "cold sweep, CUDA graph" if graph_us is not None else "cold sweep, stream"},
+    }
+    if "graph_error" in dec:
+        decode["graph_error"] = dec["graph_error"]
+
+    # ---- CPU baseline: the oracle as it stands on this machine's host cores (rank 0, N = 1) ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(wl)
+
+    if rank == 0:
+        line = {
+            "metric": "lasad_prefill_tokens_per_s", "value": round(value, 1), "unit": "tokens/s",
+            "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": round(ms_per_step, 5),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": f"{wl.name}: B={wl.B} H={wl.H} T={wl.T} ({wl.grid_h}x{wl.grid_w} grid) "
+                                   f"d_k=d_v={wl.d}, {wl.dtype} I/O, fp32 accumulate and state",
+                       "per_gpu_tokens": tokens_per_step, "parallelism": f"replicated x{world}, no collective",
+                       "l2_policy": "inputs larger than L2 (q,k,v,o = %.0f MB)" % (pf_bytes / 1e6)},
+            "e2e": {"value": round(world * tokens_per_step / (e2e_ms * 1e-3), 1), "unit": "tokens/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4),
+                    "steps": Ke},
+            "gpu_launches": int(launches),
+            "clocks": sampler.summary(),
+            "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4),
+                         "traffic": NCU_TRAFFIC_BYTES["prefill"], "peak_source": peaks["source"],
+                         "kernel_ms": round(kern_ms, 5), "bytes_per_launch": pf_bytes},
+            "tensor": {"executed_tflops": round(tc_tflops, 1), "chunk": chunk,
+                       "frac_of_bf16_peak": round(tc_tflops / peaks["bf16_tflops"], 4)},
+            "decode": decode,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------------
+# CPU baseline / reference arm: the oracle, as it stands, on the host cores
+# --------------------------------------------------------------------------------------------
+def _oracle_sample(wl, units_b: int, reps: int):
+    import numpy as np
+    import torch
+
+    from oracle import lasad_oracle as orc
+    from paper_2507_01652_b200 import workloads
+
+    sub = dataclasses.replace(wl, B=units_b)
+    q, k, v = [t.to(torch.float64).numpy() for t in workloads.make_qkv(sub)]
+    g = workloads.make_decay(sub).to(torch.float64).numpy()
+    times = []
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        orc.recurrent(q, k, v, g, sub.grid_w, sub.prefix_len)
+        times.append(time.perf_counter() - t0)
+    return sub, times, orc.threads()
+
+
+def cpu_baseline(wl, units_b: int = 2, reps: int = 3):
+    sub, times, threads = _oracle_sample(wl, units_b, reps)
+    best = min(times)
+    return {"value": round(sub.B * sub.T / best, 1), "unit": "tokens/s", "cores": threads,
+            "kind": "oracle",
+            "sample": f"oracle recurrent form (fp64, OpenMP over batch x head) on batch 0..{sub.B - 1} of "
+                      f"{wl.name} (all {wl.H} heads, T={wl.T}); best of {reps} runs, {best:.2f} s each"}
+
+
+def run_reference(args):
+    """The reference arm of this tier is the CPU oracle, timed on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return
+    from paper_2507_01652_b200 import workloads
+
+    wl = workloads.WORKLOADS[args.prefill_workload]
+    K, W = max(1, min(args.steps, 5)), max(1, min(args.warmup, 2))
+    sub, times, threads = _oracle_sample(wl, 1, K + W)
+    timed = times[W:]
+    ms = 1e3 * sum(timed) / len(timed)
+    value = sub.B * sub.T / (ms * 1e-3)
+    sample = (f"oracle recurrent form (fp64) on batch 0 of {wl.name} (all {wl.H} heads, T={wl.T}) per step; "
+              f"{len(timed)} timed steps after {W} warm-up")
+    line = {
+        "impl": "reference", "metric": "lasad_prefill_tokens_per_s", "value": round(value, 1),
+        "unit": "tokens/s", "n_gpus": world, "steps": len(timed), "warmup": W,
+        "ms_per_step": round(ms, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{wl.name}: B={wl.B} H={wl.H} T={wl.T} ({wl.grid_h}x{wl.grid_w} grid) "
+                               f"d_k=d_v={wl.d}; bounded sample: batch 0 only"},
+        "cpu_baseline": {"value": round(value, 1), "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": round(value, 1), "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--prefill-workload", default="config5b")
+    ap.add_argument("--decode-workload", default="config4")
+    ap.add_argument("--chunk-for-flops", type=int, default=64,
+                    help="chunk length used to count executed tensor flops")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -19,7 +19,7 @@ struct lasad_ctx {
 
 namespace {
 
-constexpr unsigned kDefaultWaitLimit = 20u * 1000u * 1000u;
+constexpr unsigned kDefaultWaitLimit = 1u << 22;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -148,8 +148,15 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
     const bool bf16 = p->dtype == LASAD_BF16;
 
     int impl = ctx->opt_prefill_impl;
-    if (impl == 0) impl = 1;
-    if (impl == 2) return LASAD_ERR_UNSUPPORTED;
+    const bool tc_ok = lasad::prefill_tc_supported(p->dk, p->dv, bf16);
+    if (impl == 0) impl = tc_ok ? 2 : 1;
+    if (impl == 2) {
+        if (!tc_ok) return LASAD_ERR_UNSUPPORTED;
+        const cudaError_t e = lasad::launch_prefill_tc(a, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        ctx->launches += 1;
+        return LASAD_OK;
+    }
     int chunk = ctx->opt_prefill_chunk;
     if (chunk == 0) chunk = p->dk == 64 ? 32 : 64;
     if (p->T <= 16) chunk = 16;

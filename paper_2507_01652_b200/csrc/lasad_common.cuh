@@ -58,6 +58,8 @@ template <> struct io<__nv_bfloat16> {
 // Launchers implemented in the kernel files; each returns the cudaError_t of its launch.
 cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool decay_on, int tpu,
                           cudaStream_t st);
+bool prefill_tc_supported(int dk, int dv, bool bf16);
+cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st);
 cudaError_t launch_prefill_simt(const KernelArgs& a, int dk, int dv, bool bf16, int chunk,
                                 cudaStream_t st);
 

@@ -2,26 +2,37 @@
 // TMEM accumulators, bf16 I/O, fp32 accumulation and an fp32 master state.
 //
 // One CTA owns one (batch, head) and walks its sequence in chunks of C = 128 tokens; two CTAs
-// fit on an SM (256 TMEM columns and ~105 KB of shared memory each) so that one CTA's
-// tensor-core and TMA latencies are covered by the other's CUDA-core work.  Per chunk, with
-// n_i = number of decaying steps from the chunk start up to token i (SAD rule, Section 3.4,
-// from the token's grid position) and gamma the head's decay:
+// fit on an SM (256 TMEM columns and ~106 KB of shared memory each).  With n_i = number of
+// decaying steps from the chunk start up to and including token i (SAD rule, Section 3.4, from
+// the token's grid position), N = n of the chunk's last token and gamma the head's decay, the
+// SAD recurrence (Section 3.4) unrolled over one chunk is
 //
-//   M1  S  = Q K^T                                  tcgen05.mma  128x128x64   (smem x smem)
-//   E1  P  = S o gamma^(n_i - n_j) o [j <= i]  -> bf16 back into TMEM over S's columns;
-//       Q~ = diag(gamma^(n_i)) Q,  K~ = diag(gamma^(n_last - n_j)) K   in place in smem
-//   M2  O  = P V + Q~ S_prev                        tcgen05.mma  128x64x128 (tmem x smem) + 128x64x64
-//       dS = K~^T V                                 tcgen05.mma  64x64x128
-//   E2  o  = scale * O -> bf16 -> smem -> TMA store
-//   E3  S_new = gamma^(n_last) S_prev + dS          fp32 registers; bf16 copy to smem for M2
+//     o_i   = scale * ( sum_{j<=i} (q_i.k_j) gamma^(n_i-n_j) v_j  +  gamma^(n_i) q_i^T S_prev )
+//     S_new = gamma^N S_prev + sum_j gamma^(N-n_j) k_j v_j^T
 //
-// which is the SAD recurrence (Section 3.4) unrolled over the chunk.  Every power of gamma has
-// an integer exponent in [0, 128] and comes from a per-CTA table, so gamma = 0 is exact.
+// Normal path (gamma >= 0.6, so that gamma^-128 stays far inside fp32 range).  Every decay
+// factor is moved onto V and onto one per-row factor of the output, so that Q and K feed the
+// tensor cores untouched and the scores only need the causal mask:
 //
-// Warp roles: warps 0-3 do E1/E2/E3 (thread i owns chunk row i = TMEM lane i), warp 4 issues
-// the TMA loads, warp 5 allocates TMEM and issues every MMA.  All waits are bounded: a wait that
-// runs out raises a status word the host can read and the CTA leaves through the normal exit
-// (copies in flight are waited for, TMEM is freed).
+//     V~ = diag(gamma^(N-n_j)) V                       in place in smem, before the scores exist
+//     S  = Q K^T                         (M1)          tcgen05.mma 128x128x64, smem x smem
+//     A  = tril(S) -> bf16               (E1)          back into TMEM over S's own columns
+//     dS = K^T V~                        (M2a)         tcgen05.mma 64x64x128
+//     O' = A V~ + Q (gamma^N S_prev)     (M2b)         tcgen05.mma 128x64x128 (tmem x smem) + 128x64x64
+//     o_i = scale * gamma^-(N-n_i) * O'_i   (E2)       -> bf16 -> smem -> TMA store
+//     S_new = gamma^N S_prev + dS        (E3)          fp32 registers; bf16 copy to smem for M2b
+//
+// Exact path (gamma < 0.6, including 0, where gamma^-(N-n_i) would overflow): only factors
+// with non-negative exponents are formed, all from a table of gamma^m, m = 0..128:
+// P = S o gamma^(n_i-n_j) o [j<=i], Q~ = diag(gamma^(n_i)) Q and K~ = diag(gamma^(N-n_j)) K
+// in place, O = P V + Q~ S_prev, dS = K~^T V.  Same MMAs, same barriers, slower element-wise
+// stages; it exists for correctness over the whole decay range [0, 1].
+//
+// Warp roles: warps 0-7 do the element-wise stages; warp w works on TMEM lane quadrant w & 3
+// (chunk rows 32(w&3)..+31) and the two warps of a quadrant split its columns.  Warp 8
+// allocates TMEM and issues every MMA, warp 9 issues the TMA loads and stores.  All waits are
+// bounded: a wait that runs out raises a status word the host can read and the CTA leaves
+// through the normal exit (copies in flight are waited for, TMEM is freed).
 #include "lasad_common.cuh"
 
 #include <cuda.h>
@@ -29,23 +40,27 @@
 namespace lasad {
 namespace {
 
-constexpr int kC = 128;            // chunk length (tokens) = MMA M
-constexpr int kD = 64;             // d_k = d_v
-constexpr int kThreads = 192;
-constexpr int kTileBytes = kC * kD * 2;          // 16 KB: one [128 x 64] bf16 tile, 128 B rows
+constexpr int kC = 128;                    // chunk length (tokens) = MMA M
+constexpr int kD = 64;                     // d_k = d_v
+constexpr int kEThreads = 256;             // element-wise warps 0-7
+constexpr int kThreads = kEThreads + 64;   // + the MMA warp and the TMA warp
+constexpr int kTileBytes = kC * kD * 2;    // 16 KB: one [128 x 64] bf16 tile, 128 B rows
 constexpr int kStages = 2;
 constexpr int kTmemCols = 256;
-constexpr uint32_t kColS = 0;      // S (fp32, 128 columns); P (bf16 pairs) aliases columns 0..63
+constexpr uint32_t kColS = 0;      // S (fp32, 128 columns); A/P (bf16 pairs) aliases columns 0..31 and 64..95
 constexpr uint32_t kColO = 128;    // O accumulator, 64 columns
 constexpr uint32_t kColDS = 192;   // dS accumulator (M = 64 layout), 64 columns
 constexpr unsigned kTeardownLimit = 1u << 26;
+constexpr float kFastPathMinDecay = 0.6f;
 
 struct __align__(8) Barriers {
-    unsigned long long full[kStages];
-    unsigned long long empty[kStages];
+    unsigned long long full[kStages];   // TMA loads of a stage have landed
     unsigned long long s_done;     // M1 complete
-    unsigned long long p_ready;    // E1 complete (P in TMEM, Q~/K~/S_bf16 in smem)
-    unsigned long long o_done;     // M2 complete
+    unsigned long long x_ready;    // V~ (normal path) or K~ (exact path) written: dS may start (256 arrivals)
+    unsigned long long ds_done;    // dS MMAs complete
+    unsigned long long p_ready;    // A/P in TMEM, state copy (and Q~) in smem (256 arrivals)
+    unsigned long long o_done;     // O MMAs complete (and every MMA issued before them)
+    unsigned long long st_ready;   // output tile staged in smem (256 arrivals)
     unsigned long long drain;      // teardown: all MMAs retired
 };
 
@@ -55,9 +70,8 @@ struct Smem {
     unsigned char k[kStages][kTileBytes];
     unsigned char v[kStages][kTileBytes];
     unsigned char sb[kD * kD * 2];  // bf16 copy of the state, [dk][dv], 128 B rows, swizzled
-    float pw[kC + 4];               // gamma^m, m = 0..128
-    int nj[kC];                     // n_j of the current chunk
-    int warp_cnt[4];
+    float pw[kC + 4];               // gamma^m,  m = 0..128
+    float ipw[kC + 4];              // gamma^-m, m = 0..128 (normal path only)
     Barriers bar;
     uint32_t tmem_base;
     int abort_flag;
@@ -101,6 +115,9 @@ __device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity, unsigned l
 {
     for (unsigned it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
+#ifdef LASAD_WAIT_SLEEP
+        __nanosleep(LASAD_WAIT_SLEEP);
+#endif
         if ((it & 63u) == 63u && *abort_flag) return false;
     }
     *abort_flag = 1;
@@ -191,21 +208,6 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&r)[16]
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// AND-reduction of a predicate over the 128 threads of warps 0-3 (named barrier 1).
-__device__ __forceinline__ bool wg_all(bool ok)
-{
-    unsigned r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.and.pred p, 1, 128, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r)
-        : "r"((unsigned)ok)
-        : "memory");
-    return r != 0;
-}
-__device__ __forceinline__ void wg_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);  // .x (low 16 bits) = lo
@@ -214,22 +216,35 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
-// Multiply the 64 bf16 values of one 128-byte tile row by a scalar, in place (fp32 product,
-// one rounding).  The swizzle permutes 16-byte pieces within the row, so a row-uniform factor
-// needs no address arithmetic.
-__device__ __forceinline__ void scale_row_inplace(unsigned char* row, float f)
+// Multiply `pieces` 16-byte pieces (8 bf16 each) of one 128-byte tile row by a scalar, in
+// place (fp32 product, one rounding).  The swizzle only permutes 16-byte pieces within the row,
+// so a row-uniform factor needs no un-swizzling; `rot` staggers the order in which neighbouring
+// rows walk their pieces so that the 8 threads of a quarter-warp touch 8 different bank groups.
+template <int kPieces>
+__device__ __forceinline__ void scale_row_inplace(unsigned char* row, float f, int first, int rot)
 {
     uint4* p = reinterpret_cast<uint4*>(row);
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        uint4 x = p[c];
+    for (int c = 0; c < kPieces; ++c) {
+        const int idx = (first + c) ^ rot;
+        uint4 x = p[idx];
         x.x = pack_bf16(bf16_lo(x.x) * f, bf16_hi(x.x) * f);
         x.y = pack_bf16(bf16_lo(x.y) * f, bf16_hi(x.y) * f);
         x.z = pack_bf16(bf16_lo(x.z) * f, bf16_hi(x.z) * f);
         x.w = pack_bf16(bf16_lo(x.w) * f, bf16_hi(x.w) * f);
-        p[c] = x;
+        p[idx] = x;
     }
 }
+
+#ifdef LASAD_TC_TRACE
+// Debug builds only: per-phase clock64() stamps of CTA 0 (E-thread 0: slots 0..; MMA thread: slots 2048..).
+__device__ long long g_trace[4096];
+#define TRACE_E(slot) do { if (blockIdx.x == 0 && tid == 0) g_trace[(slot)] = clock64(); } while (0)
+#define TRACE_M(slot) do { if (blockIdx.x == 0 && lane == 0) g_trace[2048 + (slot)] = clock64(); } while (0)
+#else
+#define TRACE_E(slot) do { } while (0)
+#define TRACE_M(slot) do { } while (0)
+#endif
 
 struct TcParams {
     int B, T, H;
@@ -243,7 +258,54 @@ struct TcParams {
     unsigned wait_limit;
 };
 
-__global__ void __launch_bounds__(kThreads, 2)
+// Decay bookkeeping of one chunk, computed by every warp on its own with four ballots (one per
+// 32-token block): which steps decay, and from their popcounts n_i for the thread's own row.
+struct ChunkDecay {
+    unsigned mask[4];   // bit l of mask[x]: token 32 x + l of the chunk is a decaying step
+    int cum[4];         // decaying steps up to the end of block x
+    int ni;             // n of the thread's own row
+    int n_last;         // n of the chunk's last token
+    // n of chunk column j (warp-uniform j)
+    __device__ __forceinline__ int n_of(int j) const
+    {
+        const int x = j >> 5;
+        return (x ? cum[x - 1] : 0) + __popc(mask[x] & (0xffffffffu >> (31 - (j & 31))));
+    }
+};
+
+struct GridPos {
+    int grid_w;
+    int pre;        // tokens of this call that precede the grid (class-token prefix)
+    unsigned col0;  // grid column of the call's first grid token
+};
+
+__device__ __forceinline__ ChunkDecay chunk_decay(const GridPos& g, int cs, int L, int qd, int lane)
+{
+    ChunkDecay d;
+    int run = 0;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const int tok = 32 * x + lane;
+        // the token sits at grid index gi (negative inside the prefix); its step is a boundary
+        // step (decay 1) when it is the last token of its grid row, i.e. its column is w - 1
+        const int gi = cs + tok - g.pre;
+        const bool boundary =
+            g.grid_w > 0 && gi >= 0 && ((g.col0 + (unsigned)gi + 1u) % (unsigned)g.grid_w) == 0u;
+        d.mask[x] = __ballot_sync(0xffffffffu, tok < L && !boundary);
+        run += __popc(d.mask[x]);
+        d.cum[x] = run;
+    }
+    d.n_last = run;
+    const unsigned own = qd == 0 ? d.mask[0] : qd == 1 ? d.mask[1] : qd == 2 ? d.mask[2] : d.mask[3];
+    const int before = qd == 0 ? 0 : qd == 1 ? d.cum[0] : qd == 2 ? d.cum[1] : d.cum[2];
+    d.ni = before + __popc(own & (0xffffffffu >> (31 - lane)));
+    return d;
+}
+
+#ifndef LASAD_MINBLOCKS
+#define LASAD_MINBLOCKS 2
+#endif
+__global__ void __launch_bounds__(kThreads, LASAD_MINBLOCKS)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, TcParams p)
 {
@@ -256,257 +318,360 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int n_chunks = (p.T + kC - 1) / kC;
     volatile int* abort_flag = &sm.abort_flag;
     const unsigned limit = p.wait_limit;
+    const float gamma = p.decay[h];
+    const bool fast = gamma >= kFastPathMinDecay;
 
     // ---- set-up ---------------------------------------------------------------------------
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(&sm.bar.full[s], 1);
-            mbar_init(&sm.bar.empty[s], 1);
-        }
+        for (int s = 0; s < kStages; ++s) mbar_init(&sm.bar.full[s], 1);
         mbar_init(&sm.bar.s_done, 1);
-        mbar_init(&sm.bar.p_ready, 128);
+        mbar_init(&sm.bar.x_ready, kEThreads);
+        mbar_init(&sm.bar.ds_done, 1);
+        mbar_init(&sm.bar.p_ready, kEThreads);
         mbar_init(&sm.bar.o_done, 1);
+        mbar_init(&sm.bar.st_ready, kEThreads);
         mbar_init(&sm.bar.drain, 1);
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 5) {
+    if (warp == 8) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
                      "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (tid < 128) {
-        // gamma^m for m = 0..128 in double precision (0^0 = 1)
-        const double g = (double)p.decay[h];
-        sm.pw[tid] = (float)pow(g, (double)tid);
-        if (tid == 0) sm.pw[kC] = (float)pow(g, (double)kC);
+    if (tid <= kC) {
+        // gamma^m for m = 0..128 by binary exponentiation in double precision (0^0 = 1)
+        double base = (double)gamma, acc = 1.0;
+        for (int e = tid; e > 0; e >>= 1) {
+            if (e & 1) acc *= base;
+            base *= base;
+        }
+        sm.pw[tid] = (float)acc;
+        sm.ipw[tid] = fast ? (float)(1.0 / acc) : 0.0f;
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
 
-    if (warp == 4) {
-        // ===================== TMA producer ===============================================
+    if (warp == 9) {
+        // ===================== TMA warp: loads two chunks ahead, stores each output tile =======
         if (lane == 0) {
-            int issued = 0;
-            for (int n = 0; n < n_chunks; ++n) {
+            auto issue_loads = [&](int n) {
                 const int s = n % kStages;
-                if (n >= kStages) {
-                    if (!mbar_wait(&sm.bar.empty[s], ((n / kStages) - 1) & 1, limit, abort_flag, p.status)) break;
-                }
                 mbar_arrive_expect_tx(&sm.bar.full[s], 3 * kTileBytes);
                 tma_load_4d(sm.q[s], &tm_q, &sm.bar.full[s], 0, h, n * kC, b);
                 tma_load_4d(sm.k[s], &tm_k, &sm.bar.full[s], 0, h, n * kC, b);
                 tma_load_4d(sm.v[s], &tm_v, &sm.bar.full[s], 0, h, n * kC, b);
-                issued = n + 1;
+            };
+            int loads_issued = min(n_chunks, kStages);
+            for (int n = 0; n < loads_issued; ++n) issue_loads(n);
+            for (int n = 0; n < n_chunks; ++n) {
+                const int s = n % kStages;
+                // the output tile of chunk n sits in the Q buffer of its stage; by now every MMA
+                // that read this stage has retired (the element-wise warps waited for o_done)
+                if (!mbar_wait(&sm.bar.st_ready, n & 1, limit, abort_flag, p.status)) break;
+                tma_store_4d(&tm_o, sm.q[s], 0, h, n * kC, b);
+                tma_store_commit();
+                if (n + kStages < n_chunks) {
+                    tma_store_wait_read();        // the store has finished reading the buffer
+                    issue_loads(n + kStages);
+                    loads_issued = n + kStages + 1;
+                }
             }
+            tma_store_wait_all();
             // leave only when every issued load has landed (they write this CTA's shared memory)
-            for (int n = max(0, issued - kStages); n < issued; ++n) {
-                const int s = n % kStages;
+            for (int n = max(0, loads_issued - kStages); n < loads_issued; ++n)
                 for (unsigned it = 0; it < kTeardownLimit; ++it)
-                    if (mbar_try_wait(&sm.bar.full[s], (n / kStages) & 1)) break;
-            }
+                    if (mbar_try_wait(&sm.bar.full[n % kStages], (n / kStages) & 1)) break;
         }
-    } else if (warp == 5) {
-        // ===================== MMA issuer =================================================
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);   // Q (K-major) x K (K-major)
-            constexpr uint32_t idesc_pv = make_idesc(128, 64, 0, 1);   // P (tmem) x V (MN-major)
-            constexpr uint32_t idesc_qs = make_idesc(128, 64, 0, 1);   // Q~ (K-major) x S (MN-major)
-            constexpr uint32_t idesc_kv = make_idesc(64, 64, 1, 1);    // K~^T (MN-major) x V (MN-major)
-            const uint64_t d_sb = make_desc(smem_u32(sm.sb));
-            bool ok = true;
-            auto issue_m1 = [&](int n) {
-                const int s = n % kStages;
-                if (!mbar_wait(&sm.bar.full[s], (n / kStages) & 1, limit, abort_flag, p.status)) return false;
-                tc_fence_after();
-                const uint64_t dq = make_desc(smem_u32(sm.q[s])), dk = make_desc(smem_u32(sm.k[s]));
+        __syncwarp();
+    } else if (warp == 8) {
+        // ===================== MMA issuer: the whole warp runs the loop, one lane issues =======
+        constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);   // Q (K-major) x K (K-major)
+        constexpr uint32_t idesc_pv = make_idesc(128, 64, 0, 1);   // A/P (tmem) x V (MN-major)
+        constexpr uint32_t idesc_qs = make_idesc(128, 64, 0, 1);   // Q (K-major) x state (MN-major)
+        constexpr uint32_t idesc_kv = make_idesc(64, 64, 1, 1);    // K^T (MN-major) x V (MN-major)
+        const uint64_t d_sb = make_desc(smem_u32(sm.sb));
+        uint64_t dq[kStages], dk[kStages], dv[kStages];
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) {
+            dq[s] = make_desc(smem_u32(sm.q[s]));
+            dk[s] = make_desc(smem_u32(sm.k[s]));
+            dv[s] = make_desc(smem_u32(sm.v[s]));
+        }
+        auto issue_m1 = [&](int n) {
+            const int s = n % kStages;
+            if (!mbar_wait(&sm.bar.full[s], (n / kStages) & 1, limit, abort_flag, p.status)) return false;
+            tc_fence_after();
+            if (lane == 0) {
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk)  // 32 bytes along K per step
-                    mma_ss(tmem + kColS, dq + 2 * kk, dk + 2 * kk, idesc_s, kk > 0);
+                    mma_ss(tmem + kColS, dq[s] + 2 * kk, dk[s] + 2 * kk, idesc_s, kk > 0);
                 mma_commit(&sm.bar.s_done);
-                return true;
-            };
-            ok = n_chunks > 0 && issue_m1(0);
-            for (int n = 0; ok && n < n_chunks; ++n) {
-                const int s = n % kStages;
-                if (!mbar_wait(&sm.bar.p_ready, n & 1, limit, abort_flag, p.status)) { ok = false; break; }
-                tc_fence_after();
-                const uint64_t dq = make_desc(smem_u32(sm.q[s])), dk = make_desc(smem_u32(sm.k[s]));
-                const uint64_t dv = make_desc(smem_u32(sm.v[s]));
+            }
+            __syncwarp();
+            return true;
+        };
+        bool ok = n_chunks > 0 && issue_m1(0);
+        for (int n = 0; ok && n < n_chunks; ++n) {
+            const int s = n % kStages;
+            TRACE_M(8 * n + 0);
+            if (!mbar_wait(&sm.bar.x_ready, n & 1, limit, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            if (lane == 0) {
 #pragma unroll
-                for (int kk = 0; kk < kC / 16; ++kk)  // P: 8 columns per step; V: 16 rows = 2048 B per step
-                    mma_ts(tmem + kColO, tmem + kColS + 8 * kk, dv + 128 * kk, idesc_pv, kk > 0);
+                for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K and of V per step
+                    mma_ss(tmem + kColDS, dk[s] + 128 * kk, dv[s] + 128 * kk, idesc_kv, kk > 0);
+                mma_commit(&sm.bar.ds_done);
+            }
+            __syncwarp();
+            TRACE_M(8 * n + 1);
+            if (!mbar_wait(&sm.bar.p_ready, n & 1, limit, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            TRACE_M(8 * n + 2);
+            if (lane == 0) {
+#pragma unroll
+                for (int kk = 0; kk < kC / 16; ++kk)  // A/P: 8 TMEM columns per step (tokens 0..63 at columns
+                                                      // 0..31, tokens 64..127 at 64..95); V: 2048 B per step
+                    mma_ts(tmem + kColO, tmem + kColS + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), dv[s] + 128 * kk,
+                           idesc_pv, kk > 0);
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk)
-                    mma_ss(tmem + kColO, dq + 2 * kk, d_sb + 128 * kk, idesc_qs, 1);
-#pragma unroll
-                for (int kk = 0; kk < kC / 16; ++kk)
-                    mma_ss(tmem + kColDS, dk + 128 * kk, dv + 128 * kk, idesc_kv, kk > 0);
+                    mma_ss(tmem + kColO, dq[s] + 2 * kk, d_sb + 128 * kk, idesc_qs, 1);
                 mma_commit(&sm.bar.o_done);
-                if (n + 1 < n_chunks) ok = issue_m1(n + 1);
             }
-            // make sure nothing is still running on the tensor pipe before TMEM is freed
+            __syncwarp();
+            TRACE_M(8 * n + 3);
+            if (n + 1 < n_chunks) ok = issue_m1(n + 1);
+            TRACE_M(8 * n + 4);
+        }
+        // make sure nothing is still running on the tensor pipe before TMEM is freed
+        if (lane == 0) {
             mma_commit(&sm.bar.drain);
             for (unsigned it = 0; it < kTeardownLimit; ++it)
                 if (mbar_try_wait(&sm.bar.drain, 0)) break;
         }
+        __syncwarp();
     } else {
-        // ===================== E1 / E2 / E3: thread i owns chunk row i ====================
-        const int i = tid;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        const int srow = warp * 16 + lane;       // state row held by lanes 0..15 (M = 64 TMEM layout)
+        // ===================== element-wise warps ==============================================
+        const int qd = warp & 3;                 // TMEM lane quadrant
+        const int grp = warp >> 2;               // which half of the quadrant's columns
+        const int i = qd * 32 + lane;            // chunk row owned by this thread
+        const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+        const int srow = qd * 16 + lane;         // state row (M = 64 TMEM layout: lanes 0..15 of a quadrant)
         const bool has_state = lane < 16;
         const size_t unit = (size_t)blockIdx.x * kD * kD;
-        float st[kD];
+
+        // position of the call's first token relative to the grid (SAD rule, Section 3.4)
+        GridPos gp;
+        {
+            const long long g0 = p.t0 - p.prefix_len;
+            gp.grid_w = p.grid_w;
+            gp.pre = g0 < 0 ? (int)min(-g0, (long long)0x7fffffff) : 0;
+            gp.col0 = (p.grid_w > 0 && g0 > 0) ? (unsigned)(g0 % p.grid_w) : 0u;
+        }
+
+        float st[32];                            // state[srow][32 grp .. 32 grp + 31], fp32 master
 #pragma unroll
-        for (int e = 0; e < kD; ++e) st[e] = 0.0f;
+        for (int e = 0; e < 32; ++e) st[e] = 0.0f;
         if (has_state && p.state_in) {
-            const float4* src = reinterpret_cast<const float4*>(p.state_in + unit + (size_t)srow * kD);
+            const float4* src = reinterpret_cast<const float4*>(p.state_in + unit + (size_t)srow * kD + 32 * grp);
 #pragma unroll
-            for (int e4 = 0; e4 < kD / 4; ++e4) {
+            for (int e4 = 0; e4 < 8; ++e4) {
                 const float4 t = src[e4];
                 st[4 * e4] = t.x; st[4 * e4 + 1] = t.y; st[4 * e4 + 2] = t.z; st[4 * e4 + 3] = t.w;
             }
         }
-        auto write_state_bf16 = [&]() {
+        // bf16 copy of mult * state for the Q x state MMA of the next chunk
+        auto write_state_bf16 = [&](float mult) {
             if (has_state) {
                 uint4* row = reinterpret_cast<uint4*>(sm.sb + srow * 128);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
+                for (int c = 0; c < 4; ++c) {
                     uint4 x;
-                    x.x = pack_bf16(st[8 * c], st[8 * c + 1]);
-                    x.y = pack_bf16(st[8 * c + 2], st[8 * c + 3]);
-                    x.z = pack_bf16(st[8 * c + 4], st[8 * c + 5]);
-                    x.w = pack_bf16(st[8 * c + 6], st[8 * c + 7]);
-                    row[c ^ (srow & 7)] = x;
+                    x.x = pack_bf16(mult * st[8 * c], mult * st[8 * c + 1]);
+                    x.y = pack_bf16(mult * st[8 * c + 2], mult * st[8 * c + 3]);
+                    x.z = pack_bf16(mult * st[8 * c + 4], mult * st[8 * c + 5]);
+                    x.w = pack_bf16(mult * st[8 * c + 6], mult * st[8 * c + 7]);
+                    row[(4 * grp + c) ^ (srow & 7)] = x;
                 }
             }
         };
-        write_state_bf16();
+        // E3: S_new = g * S_prev + dS (this thread's 32 columns of its state row)
+        auto update_state = [&](float g) {
+            uint32_t dsv[32];
+            tmem_ld32(tmem + lane_base + kColDS + 32 * grp, dsv);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) st[e] = fmaf(g, st[e], __uint_as_float(dsv[e]));
+        };
+        // E2: this thread's 32 columns of output row i -> bf16 -> the stage's Q buffer
+        auto stage_output = [&](int s, float f) {
+            unsigned char* orow = sm.q[s] + i * 128;
+            uint32_t ov[32];
+            tmem_ld32(tmem + lane_base + kColO + 32 * grp, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint4 x;
+                x.x = pack_bf16(f * __uint_as_float(ov[8 * c]), f * __uint_as_float(ov[8 * c + 1]));
+                x.y = pack_bf16(f * __uint_as_float(ov[8 * c + 2]), f * __uint_as_float(ov[8 * c + 3]));
+                x.z = pack_bf16(f * __uint_as_float(ov[8 * c + 4]), f * __uint_as_float(ov[8 * c + 5]));
+                x.w = pack_bf16(f * __uint_as_float(ov[8 * c + 6]), f * __uint_as_float(ov[8 * c + 7]));
+                reinterpret_cast<uint4*>(orow)[(4 * grp + c) ^ (i & 7)] = x;
+            }
+        };
 
         bool ok = true;
-        for (int n = 0; n < n_chunks; ++n) {
-            const int s = n % kStages;
-            const int cs = n * kC;
-            const int L = min(kC, p.T - cs);
-
-            // ---- decay bookkeeping: n_i by ballot + popcount over the chunk --------------------
-            const long long abs_i = p.t0 + cs + i;
-            const bool decays = i < L && !is_boundary_step(abs_i, p.grid_w, p.prefix_len);
-            const unsigned m = __ballot_sync(0xffffffffu, decays);
-            if (lane == 0) sm.warp_cnt[warp] = __popc(m);
-            wg_sync();
-            int ni = __popc(m & (0xffffffffu >> (31 - lane)));
-            int n_last = 0;
-#pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                const int c = sm.warp_cnt[w];
-                if (w < warp) ni += c;
-                n_last += c;
+        if (fast) {
+            // ------------------------------- normal path ---------------------------------------
+            ChunkDecay cd = chunk_decay(gp, 0, min(kC, p.T), qd, lane);
+            write_state_bf16(sm.pw[cd.n_last]);
+            ok = mbar_wait(&sm.bar.full[0], 0, limit, abort_flag, p.status);
+            if (ok) {
+                scale_row_inplace<4>(sm.v[0] + i * 128, sm.pw[cd.n_last - cd.ni], 4 * grp, i & 7);
+                fence_proxy_async();
+                mbar_arrive(&sm.bar.x_ready);
             }
-            sm.nj[i] = ni;
+            for (int n = 0; ok && n < n_chunks; ++n) {
+                const int s = n % kStages;
+                TRACE_E(8 * n + 0);
+                if (!(ok = mbar_wait(&sm.bar.s_done, n & 1, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+                TRACE_E(8 * n + 1);
+                // ---- E1: A = tril(S) -> bf16 over S's own columns.  This warp converts the
+                //      32-column blocks 2 grp and 2 grp + 1 of its rows and keeps the result inside
+                //      its own half of S's columns (block pc -> columns 64 grp + 16 (pc & 1), always
+                //      behind this warp's own reads); the A V~ MMAs walk the columns in that order.
+#pragma unroll
+                for (int pi = 0; pi < 2; ++pi) {
+                    const int pc = 2 * grp + pi;
+                    uint32_t pk[16];
+                    if (pc <= qd) {
+                        uint32_t sv[32];
+                        tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
+                        tmem_wait_ld();
+                        if (pc < qd) {
+#pragma unroll
+                            for (int c = 0; c < 16; ++c)
+                                pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 16; ++c)
+                                pk[c] = pack_bf16(2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
+                                                  2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                    }
+                    tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
+                }
+                tmem_wait_st();
+                fence_proxy_async();   // state copy written at the end of the previous iteration
+                tc_fence_before();
+                mbar_arrive(&sm.bar.p_ready);
+                TRACE_E(8 * n + 2);
 
-            ok = wg_all(mbar_wait(&sm.bar.s_done, n & 1, limit, abort_flag, p.status));  // also publishes nj
-            if (!ok) break;
-            tc_fence_after();
+                // ---- while the O MMAs run: state arithmetic, next chunk's bookkeeping and V~ -----
+                const float out_f = p.scale * sm.ipw[cd.n_last - cd.ni];   // scale * gamma^-(N - n_i)
+                if (!(ok = mbar_wait(&sm.bar.ds_done, n & 1, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+                update_state(sm.pw[cd.n_last]);
+                TRACE_E(8 * n + 3);
+                float next_mult = 1.0f;
+                if (n + 1 < n_chunks) {
+                    const int cs1 = (n + 1) * kC;
+                    cd = chunk_decay(gp, cs1, min(kC, p.T - cs1), qd, lane);
+                    next_mult = sm.pw[cd.n_last];
+                    const int s1 = (n + 1) % kStages;
+                    if (!(ok = mbar_wait(&sm.bar.full[s1], ((n + 1) / kStages) & 1, limit, abort_flag, p.status))) break;
+                    scale_row_inplace<4>(sm.v[s1] + i * 128, sm.pw[cd.n_last - cd.ni], 4 * grp, i & 7);
+                    fence_proxy_async();
+                    tc_fence_before();     // dS of this chunk has been read (update_state above)
+                    mbar_arrive(&sm.bar.x_ready);
+                }
+                TRACE_E(8 * n + 4);
 
-            // ---- E1: P = S o decay o causal, written over S as bf16 pairs -----------------------
+                // ---- E2: o_i = scale * gamma^-(N - n_i) * O'_i ------------------------------------
+                if (!(ok = mbar_wait(&sm.bar.o_done, n & 1, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+                TRACE_E(8 * n + 5);
+                stage_output(s, out_f);
+                if (n + 1 < n_chunks) write_state_bf16(next_mult);   // gamma^N(next) * S_new
+                fence_proxy_async();
+                tc_fence_before();
+                mbar_arrive(&sm.bar.st_ready);
+                TRACE_E(8 * n + 6);
+            }
+        } else {
+            // ------------------------------- exact path ----------------------------------------
+            write_state_bf16(1.0f);
+            for (int n = 0; ok && n < n_chunks; ++n) {
+                const int s = n % kStages;
+                const int cs = n * kC;
+                const ChunkDecay cd = chunk_decay(gp, cs, min(kC, p.T - cs), qd, lane);
+                if (!(ok = mbar_wait(&sm.bar.s_done, n & 1, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+                // K~ first (M1 has finished reading K): it unblocks the dS MMAs
+                if (grp == 1) scale_row_inplace<8>(sm.k[s] + i * 128, sm.pw[cd.n_last - cd.ni], 0, i & 7);
+                fence_proxy_async();
+                mbar_arrive(&sm.bar.x_ready);
+                // P = S o gamma^(n_i - n_j) o [j <= i], weights straight from the table
 #pragma unroll 1
-            for (int pc = 0; pc < 4; ++pc) {
-                uint32_t pk[16];
-                if (pc <= warp) {
-                    uint32_t sv[32];
-                    tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
-                    tmem_wait_ld();
-                    float val[32];
+                for (int pi = 0; pi < 2; ++pi) {
+                    const int pc = 2 * grp + pi;
+                    uint32_t pk[16];
+                    if (pc <= qd) {
+                        uint32_t sv[32];
+                        tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        const int j = 32 * pc + jj;
-                        const int dn = ni - sm.nj[j];
-                        const float w = sm.pw[dn > 0 ? dn : 0];
-                        val[jj] = (j <= i) ? __uint_as_float(sv[jj]) * w : 0.0f;
+                        for (int c = 0; c < 16; ++c) {
+                            const int j0 = 32 * pc + 2 * c;
+                            const int d0 = cd.ni - cd.n_of(j0), d1 = cd.ni - cd.n_of(j0 + 1);
+                            const float v0 = j0 <= i ? __uint_as_float(sv[2 * c]) * sm.pw[d0 > 0 ? d0 : 0] : 0.0f;
+                            const float v1 = j0 + 1 <= i ? __uint_as_float(sv[2 * c + 1]) * sm.pw[d1 > 0 ? d1 : 0] : 0.0f;
+                            pk[c] = pack_bf16(v0, v1);
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) pk[c] = 0u;
                     }
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) pk[c] = pack_bf16(val[2 * c], val[2 * c + 1]);
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                    tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
                 }
-                tmem_st16(tmem + lane_base + kColS + 16 * pc, pk);
-            }
-            // Q~ and K~ in place (M1 has finished reading both tiles)
-            scale_row_inplace(sm.q[s] + i * 128, sm.pw[ni]);
-            scale_row_inplace(sm.k[s] + i * 128, sm.pw[n_last - ni]);
-            tmem_wait_st();
-            fence_proxy_async();
-            tc_fence_before();
-            mbar_arrive(&sm.bar.p_ready);
+                if (grp == 0) scale_row_inplace<8>(sm.q[s] + i * 128, sm.pw[cd.ni], 0, i & 7);
+                tmem_wait_st();
+                fence_proxy_async();
+                tc_fence_before();
+                mbar_arrive(&sm.bar.p_ready);
 
-            // ---- E2: o = scale * O -> bf16 -> smem (the Q tile's buffer) -> TMA store -----------
-            ok = wg_all(mbar_wait(&sm.bar.o_done, n & 1, limit, abort_flag, p.status));
-            if (!ok) break;
-            tc_fence_after();
-            {
-                unsigned char* orow = sm.q[s] + i * 128;
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t ov[32];
-                    tmem_ld32(tmem + lane_base + kColO + 32 * half, ov);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint4 x;
-                        x.x = pack_bf16(p.scale * __uint_as_float(ov[8 * c]), p.scale * __uint_as_float(ov[8 * c + 1]));
-                        x.y = pack_bf16(p.scale * __uint_as_float(ov[8 * c + 2]), p.scale * __uint_as_float(ov[8 * c + 3]));
-                        x.z = pack_bf16(p.scale * __uint_as_float(ov[8 * c + 4]), p.scale * __uint_as_float(ov[8 * c + 5]));
-                        x.w = pack_bf16(p.scale * __uint_as_float(ov[8 * c + 6]), p.scale * __uint_as_float(ov[8 * c + 7]));
-                        reinterpret_cast<uint4*>(orow)[(4 * half + c) ^ (i & 7)] = x;
-                    }
-                }
-            }
-            fence_proxy_async();
-            wg_sync();
-            if (tid == 0) {
-                tma_store_4d(&tm_o, sm.q[s], 0, h, cs, b);
-                tma_store_commit();
-            }
-
-            // ---- E3: S_new = gamma^(n_last) S_prev + dS (fp32 master in registers) --------------
-            {
-                const float gl = sm.pw[n_last];
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t dv_[32];
-                    tmem_ld32(tmem + lane_base + kColDS + 32 * half, dv_);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        st[32 * half + e] = fmaf(gl, st[32 * half + e], __uint_as_float(dv_[e]));
-                }
-                write_state_bf16();
-            }
-            tc_fence_before();
-            if (tid == 0) {
-                tma_store_wait_read();            // the store has finished reading the Q buffer
-                mbar_arrive(&sm.bar.empty[s]);    // stage s may be refilled
+                if (!(ok = mbar_wait(&sm.bar.ds_done, n & 1, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+                update_state(sm.pw[cd.n_last]);
+                if (!(ok = mbar_wait(&sm.bar.o_done, n & 1, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+                stage_output(s, p.scale);
+                write_state_bf16(1.0f);
+                fence_proxy_async();
+                tc_fence_before();
+                mbar_arrive(&sm.bar.st_ready);
             }
         }
         if (ok && has_state && p.state_out) {
-            float4* dst = reinterpret_cast<float4*>(p.state_out + unit + (size_t)srow * kD);
+            float4* dst = reinterpret_cast<float4*>(p.state_out + unit + (size_t)srow * kD + 32 * grp);
 #pragma unroll
-            for (int e4 = 0; e4 < kD / 4; ++e4)
+            for (int e4 = 0; e4 < 8; ++e4)
                 dst[e4] = make_float4(st[4 * e4], st[4 * e4 + 1], st[4 * e4 + 2], st[4 * e4 + 3]);
         }
-        if (tid == 0) tma_store_wait_all();
     }
 
     // ---- teardown ---------------------------------------------------------------------------
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == 8) {
         __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -547,6 +712,13 @@ bool encode_map(CUtensorMap* map, const void* base, int B, int T, int H, const l
 }
 
 }  // namespace
+
+#ifdef LASAD_TC_TRACE
+extern "C" int lasad_debug_read_trace(long long* host, int n)
+{
+    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * n);
+}
+#endif
 
 bool prefill_tc_supported(int dk, int dv, bool bf16) { return bf16 && dk == kD && dv == kD; }
 

@@ -418,7 +418,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--prefill-workload", default="config5b")
     ap.add_argument("--decode-workload", default="config4")
-    ap.add_argument("--chunk-for-flops", type=int, default=64,
+    ap.add_argument("--chunk-for-flops", type=int, default=128,
                     help="chunk length used to count executed tensor flops")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

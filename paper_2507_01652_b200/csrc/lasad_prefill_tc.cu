@@ -273,28 +273,56 @@ struct ChunkDecay {
     }
 };
 
+// Where the chunks of this call sit on the token grid, in a form that needs no division inside
+// the chunk loop: token `tok` of the chunk that starts at call offset cs absorbs the last token
+// of a grid row (a boundary step, SAD rule of Section 3.4) iff it lies on the grid
+// (cs + tok >= pre) and (phase + r[tok / 32]) is 0 or w, where r = (tok mod w) is fixed per
+// thread and phase = (grid column of the chunk's first token + 1) mod w advances by
+// (128 mod w) per chunk.
 struct GridPos {
     int grid_w;
-    int pre;        // tokens of this call that precede the grid (class-token prefix)
-    unsigned col0;  // grid column of the call's first grid token
+    int pre;         // tokens of this call that precede the grid (class-token prefix)
+    int r[4];        // (32 x + lane) mod w
+    int step;        // 128 mod w
+    int phase;       // ((grid index of the current chunk's first token) + 1) mod w
 };
 
-__device__ __forceinline__ ChunkDecay chunk_decay(const GridPos& g, int cs, int L, int qd, int lane)
+__device__ __forceinline__ GridPos grid_pos_init(int grid_w, int prefix_len, long long t0, int lane)
+{
+    GridPos g;
+    g.grid_w = grid_w;
+    const long long g0 = t0 - prefix_len;   // grid index of the call's first token (may be < 0)
+    g.pre = g0 < 0 ? (int)min(-g0, (long long)0x7fffffff) : 0;
+    g.step = 0; g.phase = 0;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) g.r[x] = 0;
+    if (grid_w > 0) {
+        long long ph = (g0 + 1) % grid_w;    // C remainder: may be negative inside the prefix
+        if (ph < 0) ph += grid_w;
+        g.phase = (int)ph;
+        g.step = kC % grid_w;
+#pragma unroll
+        for (int x = 0; x < 4; ++x) g.r[x] = (32 * x + lane) % grid_w;
+    }
+    return g;
+}
+
+// Decay bookkeeping of the chunk at call offset cs (L live tokens); advances g to the next chunk.
+__device__ __forceinline__ ChunkDecay chunk_decay(GridPos& g, int cs, int L, int qd, int lane)
 {
     ChunkDecay d;
     int run = 0;
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
         const int tok = 32 * x + lane;
-        // the token sits at grid index gi (negative inside the prefix); its step is a boundary
-        // step (decay 1) when it is the last token of its grid row, i.e. its column is w - 1
-        const int gi = cs + tok - g.pre;
-        const bool boundary =
-            g.grid_w > 0 && gi >= 0 && ((g.col0 + (unsigned)gi + 1u) % (unsigned)g.grid_w) == 0u;
+        const int m = g.phase + g.r[x];
+        const bool boundary = g.grid_w > 0 && cs + tok >= g.pre && (m == 0 || m == g.grid_w);
         d.mask[x] = __ballot_sync(0xffffffffu, tok < L && !boundary);
         run += __popc(d.mask[x]);
         d.cum[x] = run;
     }
+    g.phase += g.step;
+    if (g.phase >= g.grid_w) g.phase -= g.grid_w;
     d.n_last = run;
     const unsigned own = qd == 0 ? d.mask[0] : qd == 1 ? d.mask[1] : qd == 2 ? d.mask[2] : d.mask[3];
     const int before = qd == 0 ? 0 : qd == 1 ? d.cum[0] : qd == 2 ? d.cum[1] : d.cum[2];
@@ -465,13 +493,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const size_t unit = (size_t)blockIdx.x * kD * kD;
 
         // position of the call's first token relative to the grid (SAD rule, Section 3.4)
-        GridPos gp;
-        {
-            const long long g0 = p.t0 - p.prefix_len;
-            gp.grid_w = p.grid_w;
-            gp.pre = g0 < 0 ? (int)min(-g0, (long long)0x7fffffff) : 0;
-            gp.col0 = (p.grid_w > 0 && g0 > 0) ? (unsigned)(g0 % p.grid_w) : 0u;
-        }
+        GridPos gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0, lane);
 
         float st[32];                            // state[srow][32 grp .. 32 grp + 31], fp32 master
 #pragma unroll
@@ -575,23 +597,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 mbar_arrive(&sm.bar.p_ready);
                 TRACE_E(8 * n + 2);
 
-                // ---- while the O MMAs run: state arithmetic, next chunk's bookkeeping and V~ -----
+                // ---- while the O MMAs run: the state recurrence in fp32 registers ----------------
                 const float out_f = p.scale * sm.ipw[cd.n_last - cd.ni];   // scale * gamma^-(N - n_i)
                 if (!(ok = mbar_wait(&sm.bar.ds_done, n & 1, limit, abort_flag, p.status))) break;
                 tc_fence_after();
                 update_state(sm.pw[cd.n_last]);
                 TRACE_E(8 * n + 3);
-                float next_mult = 1.0f;
-                if (n + 1 < n_chunks) {
+                const bool more = n + 1 < n_chunks;
+                if (more) {
                     const int cs1 = (n + 1) * kC;
                     cd = chunk_decay(gp, cs1, min(kC, p.T - cs1), qd, lane);
-                    next_mult = sm.pw[cd.n_last];
-                    const int s1 = (n + 1) % kStages;
-                    if (!(ok = mbar_wait(&sm.bar.full[s1], ((n + 1) / kStages) & 1, limit, abort_flag, p.status))) break;
-                    scale_row_inplace<4>(sm.v[s1] + i * 128, sm.pw[cd.n_last - cd.ni], 4 * grp, i & 7);
-                    fence_proxy_async();
-                    tc_fence_before();     // dS of this chunk has been read (update_state above)
-                    mbar_arrive(&sm.bar.x_ready);
                 }
                 TRACE_E(8 * n + 4);
 
@@ -600,11 +615,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tc_fence_after();
                 TRACE_E(8 * n + 5);
                 stage_output(s, out_f);
-                if (n + 1 < n_chunks) write_state_bf16(next_mult);   // gamma^N(next) * S_new
+                if (more) write_state_bf16(sm.pw[cd.n_last]);   // gamma^N(next) * S_new
                 fence_proxy_async();
                 tc_fence_before();
                 mbar_arrive(&sm.bar.st_ready);
                 TRACE_E(8 * n + 6);
+
+                // ---- V~ of the next chunk, once its loads have landed.  This stage is released
+                //      (st_ready above) before the wait, so the wait never holds a buffer back.
+                if (more) {
+                    const int s1 = (n + 1) % kStages;
+                    if (!(ok = mbar_wait(&sm.bar.full[s1], ((n + 1) / kStages) & 1, limit, abort_flag, p.status))) break;
+                    scale_row_inplace<4>(sm.v[s1] + i * 128, sm.pw[cd.n_last - cd.ni], 4 * grp, i & 7);
+                    fence_proxy_async();
+                    mbar_arrive(&sm.bar.x_ready);
+                }
             }
         } else {
             // ------------------------------- exact path ----------------------------------------

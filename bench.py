@@ -163,8 +163,16 @@ def run_ours(args):
     ctx = binding.Lasad(local)
     K, W = args.steps, max(args.warmup, 3)
     wl = workloads.WORKLOADS[args.prefill_workload]
+    if args.prefill_batch:
+        wl = wl.scaled(B=args.prefill_batch)
     wl = dataclasses.replace(wl, seed=wl.seed + 1000 * rank)
     stream = torch.cuda.current_stream()
+    if args.only == "decode":
+        dec = run_decode(args, ctx, peaks, dev, rank, barrier, max_over_ranks, K)
+        if rank == 0:
+            print(json.dumps({"decode": dec}), flush=True)
+        ctx.close()
+        return
 
     # ---- prefill: inputs resident in HBM -------------------------------------------------
     hq, hk, hv = [t.pin_memory() for t in workloads.make_qkv(wl)]
@@ -228,8 +236,99 @@ def run_ours(args):
     d2h = ho.numel() * ho.element_size()
     del hq, hk, hv, ho, q, k, v, o
 
-    # ---- decode sweep (config 4 shape): persistent fp32 state, one step per position ------
+    # ---- the other prefill configurations (context for the headline; rank 0 reports) ----------
+    sweep = None
+    if args.only == "all" and not args.no_sweep:
+        sweep = prefill_sweep(ctx, peaks, dev, ("config1", "config2", "config3", "config5a"))
+
+    decode = None
+    if args.only != "prefill":
+        decode = run_decode(args, ctx, peaks, dev, rank, barrier, max_over_ranks, K)
+
+    # ---- CPU baseline: the oracle as it stands on this box's host cores (rank 0, N = 1) ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(wl)
+
+    if rank == 0:
+        line = {
+            "metric": "lasad_prefill_tokens_per_s", "value": round(value, 1), "unit": "tokens/s",
+            "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": round(ms_per_step, 5),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": f"{wl.name}: B={wl.B} H={wl.H} T={wl.T} ({wl.grid_h}x{wl.grid_w} grid) "
+                                   f"d_k=d_v={wl.d}, {wl.dtype} I/O, fp32 accumulate and state",
+                       "per_gpu_tokens": tokens_per_step, "parallelism": f"replicated x{world}, no collective",
+                       "l2_policy": "inputs larger than L2 (q,k,v,o = %.0f MB)" % (pf_bytes / 1e6)},
+            "e2e": {"value": round(world * tokens_per_step / (e2e_ms * 1e-3), 1), "unit": "tokens/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4),
+                    "steps": Ke},
+            "gpu_launches": int(launches),
+            "clocks": sampler.summary(),
+            "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4),
+                         "traffic": NCU_TRAFFIC_BYTES["prefill"], "peak_source": peaks["source"],
+                         "kernel_ms": round(kern_ms, 5), "bytes_per_launch": pf_bytes},
+            "tensor": {"executed_tflops": round(tc_tflops, 1), "chunk": chunk,
+                       "frac_of_bf16_peak": round(tc_tflops / peaks["bf16_tflops"], 4)},
+            "decode": decode,
+            "prefill_sweep": sweep,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def prefill_sweep(ctx, peaks, dev, names, reps: int = 10):
+    """Kernel time of one prefill per named workload (CUDA events around each launch, median of
+    `reps`); a buffer larger than L2 is written between launches so that no launch finds its
+    inputs in L2."""
+    import torch
+
+    from paper_2507_01652_b200 import workloads
+
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    out = []
+    for name in names:
+        wl = workloads.WORKLOADS[name]
+        q, k, v = [t.to(dev) for t in workloads.make_qkv(wl)]
+        g = workloads.make_decay(wl).to(dev)
+        o = torch.empty_like(v)
+        s_out = torch.empty(wl.B, wl.H, wl.d, wl.d, dtype=torch.float32, device=dev)
+        times = []
+        for it in range(reps + 3):
+            flush.fill_(it & 1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            ctx.lasad_forward(q, k, v, g, wl.grid_w, prefix_len=wl.prefix_len, o=o, state_out=s_out)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if it >= 3:
+                times.append(a.elapsed_time(b))
+        ms = statistics.median(times)
+        nbytes = prefill_bytes(wl)
+        out.append({"workload": f"{wl.name}: B={wl.B} H={wl.H} T={wl.T} d={wl.d} {wl.dtype}",
+                    "kernel_us": round(ms * 1e3, 2), "tokens_per_s": round(wl.B * wl.T / (ms * 1e-3), 1),
+                    "algorithmic_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                    "frac_of_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)})
+        del q, k, v, o, s_out
+    return out
+
+
+def run_decode(args, ctx, peaks, dev, rank, barrier, max_over_ranks, K):
+    """Decode sweep (config 4 shape): persistent fp32 state, one `lasad_decode_step` per grid position."""
+    import torch
+
+    from paper_2507_01652_b200 import workloads
+
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(dev.index)
     dw = workloads.WORKLOADS[args.decode_workload]
+    if args.decode_batch:
+        dw = dw.scaled(B=args.decode_batch)
     dw = dataclasses.replace(dw, seed=dw.seed + 1000 * rank)
     P = dw.prefix_len
     dq, dk_, dv_ = [t.to(dev) for t in workloads.make_qkv(dw)]
@@ -314,39 +413,8 @@ def run_ours(args):
     if "graph_error" in dec:
         decode["graph_error"] = dec["graph_error"]
 
-    # ---- CPU baseline: the oracle as it stands on this box's host cores (rank 0, N = 1) ----
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = cpu_baseline(wl)
-
-    if rank == 0:
-        line = {
-            "metric": "lasad_prefill_tokens_per_s", "value": round(value, 1), "unit": "tokens/s",
-            "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": round(ms_per_step, 5),
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": f"{wl.name}: B={wl.B} H={wl.H} T={wl.T} ({wl.grid_h}x{wl.grid_w} grid) "
-                                   f"d_k=d_v={wl.d}, {wl.dtype} I/O, fp32 accumulate and state",
-                       "per_gpu_tokens": tokens_per_step, "parallelism": f"replicated x{world}, no collective",
-                       "l2_policy": "inputs larger than L2 (q,k,v,o = %.0f MB)" % (pf_bytes / 1e6)},
-            "e2e": {"value": round(world * tokens_per_step / (e2e_ms * 1e-3), 1), "unit": "tokens/s",
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4),
-                    "steps": Ke},
-            "gpu_launches": int(launches),
-            "clocks": sampler.summary(),
-            "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
-                         "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4),
-                         "traffic": NCU_TRAFFIC_BYTES["prefill"], "peak_source": peaks["source"],
-                         "kernel_ms": round(kern_ms, 5), "bytes_per_launch": pf_bytes},
-            "tensor": {"executed_tflops": round(tc_tflops, 1), "chunk": chunk,
-                       "frac_of_bf16_peak": round(tc_tflops / peaks["bf16_tflops"], 4)},
-            "decode": decode,
-            "cpu_baseline": cpu,
-        }
-        print(json.dumps(line), flush=True)
-    ctx.close()
-    if world > 1:
-        dist.destroy_process_group()
+    decode["clocks"] = sampler.summary()
+    return decode
 
 
 # --------------------------------------------------------------------------------------------
@@ -370,13 +438,19 @@ def _oracle_sample(wl, units_b: int, reps: int):
     return sub, times, orc.threads()
 
 
-def cpu_baseline(wl, units_b: int = 2, reps: int = 3):
-    sub, times, threads = _oracle_sample(wl, units_b, reps)
+def cpu_baseline(wl, budget_s: float = 12.0):
+    """The oracle's recurrent form over whole batches of the workload, repeated for about
+    `budget_s` seconds of CPU work; the best repetition is reported."""
+    units_b = min(wl.B, 4)
+    sub, times, threads = _oracle_sample(wl, units_b, 2)
+    reps = max(1, min(60, int(budget_s / max(min(times), 1e-3)) - 2))
+    times += _oracle_sample(wl, units_b, reps)[1]
     best = min(times)
     return {"value": round(sub.B * sub.T / best, 1), "unit": "tokens/s", "cores": threads,
             "kind": "oracle",
             "sample": f"oracle recurrent form (fp64, OpenMP over batch x head) on batch 0..{sub.B - 1} of "
-                      f"{wl.name} (all {wl.H} heads, T={wl.T}); best of {reps} runs, {best:.2f} s each"}
+                      f"{wl.name} (all {wl.H} heads, T={wl.T}); best of {len(times)} runs, {best:.2f} s each, "
+                      f"{sum(times):.1f} s of CPU work in total"}
 
 
 def run_reference(args):
@@ -421,6 +495,11 @@ def main():
     ap.add_argument("--chunk-for-flops", type=int, default=128,
                     help="chunk length used to count executed tensor flops")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the per-configuration prefill sweep")
+    ap.add_argument("--only", choices=["all", "prefill", "decode"], default="all",
+                    help="time only one of the two kernels (small profiling runs)")
+    ap.add_argument("--prefill-batch", type=int, default=0, help="override the prefill workload's batch")
+    ap.add_argument("--decode-batch", type=int, default=0, help="override the decode workload's batch")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

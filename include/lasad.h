@@ -21,8 +21,8 @@
  *   - Every data pointer is DEVICE memory owned by the caller and must stay valid until the
  *     given stream has passed the call.  `lasad_params` and the ctx handle are HOST memory.
  *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
- *     stream) and return without synchronising.  No call allocates device memory except
- *     lasad_create.
+ *     stream) and return without synchronising.  lasad_create and lasad_reserve allocate device
+ *     memory; lasad_forward allocates only in the case described at lasad_reserve.
  *   - Return value: LASAD_OK or a negative LASAD_ERR_*.  On an argument error nothing is
  *     launched and no output is touched.  The library never aborts the process.
  *   - Base pointers of q, k, v, o must be 16-byte aligned and every stride, in bytes, a
@@ -30,7 +30,9 @@
  *     fp32 [B, H, dk, dv], 16-byte aligned.
  *   - Supported: dk == dv in {32, 64}; dtype F32 or BF16 (q, k, v, o share it; state, decay
  *     and all accumulation are fp32); any B, H, T >= 1.  Otherwise LASAD_ERR_UNSUPPORTED.
- *   - One ctx is bound to one device and may be used from one host thread at a time.
+ *   - One ctx is bound to one device and may be used from one host thread at a time; its
+ *     prefill calls share per-chain relay storage, so two lasad_forward calls on one ctx must
+ *     not overlap on the device (issue them on one stream, or order the streams).
  */
 #ifndef LASAD_H_
 #define LASAD_H_
@@ -53,7 +55,8 @@ enum { LASAD_F32 = 0, LASAD_BF16 = 1 };
 
 /* Options for lasad_set_option. */
 enum {
-    LASAD_OPT_PREFILL_IMPL = 0, /* 0 auto, 1 CUDA-core fp32 kernel, 2 tcgen05 tensor-core kernel */
+    LASAD_OPT_PREFILL_IMPL = 0, /* 0 auto, 1 CUDA-core fp32 kernel, 2 tcgen05 kernel with one CTA per
+                                   (batch, head), 3 tcgen05 kernel streaming (batch, head, chunk) tasks  */
     LASAD_OPT_PREFILL_CHUNK = 1,/* CUDA-core prefill chunk length: 0 auto, else 16/32/64          */
     LASAD_OPT_DECODE_TPU = 2,   /* decode: threads per (b,h) state; 0 auto, else 32/64/128/256 */
     LASAD_OPT_WAIT_LIMIT = 3    /* iteration cap of device-side waits; 0 = library default   */
@@ -79,6 +82,18 @@ typedef struct lasad_ctx lasad_ctx;
 int lasad_create(lasad_ctx** out, int device);
 int lasad_destroy(lasad_ctx* ctx);
 int lasad_set_option(lasad_ctx* ctx, int option, int value);
+
+/*
+ * Makes the context's relay storage large enough for prefill calls with B * H <= units.  The
+ * task-streaming tensor-core prefill passes each chain's carried state (the s of the SAD
+ * recurrence, Section 3.4) from the CTA that absorbed one chunk of the sequence to the CTA that
+ * absorbs the next through one 32 KiB slot per (batch, head) in context-owned device memory.
+ * lasad_create allocates 1024 slots.  A lasad_forward call with more (batch, head) pairs than
+ * the context holds grows the storage first (cudaMalloc, which synchronises the device and must
+ * not happen inside a stream capture); calling lasad_reserve up front keeps lasad_forward
+ * allocation-free.
+ */
+int lasad_reserve(lasad_ctx* ctx, int64_t units);
 
 /*
  * Full-sequence (teacher-forced) prefill: the SAD recurrence (Section 3.4) evaluated for T

@@ -27,7 +27,7 @@ LASAD_OPT_DECODE_TPU = 2
 LASAD_OPT_WAIT_LIMIT = 3
 
 EXPORTS = (
-    "lasad_create", "lasad_destroy", "lasad_set_option", "lasad_forward", "lasad_decode_step",
+    "lasad_create", "lasad_destroy", "lasad_set_option", "lasad_reserve", "lasad_forward", "lasad_decode_step",
     "lasad_last_device_status", "lasad_last_cuda_error", "lasad_launch_count", "lasad_strerror",
 )
 
@@ -71,6 +71,8 @@ def load_library() -> ctypes.CDLL:
         lib.lasad_destroy.argtypes = [vp]
         lib.lasad_set_option.restype = i32
         lib.lasad_set_option.argtypes = [vp, i32, i32]
+        lib.lasad_reserve.restype = i32
+        lib.lasad_reserve.argtypes = [vp, ctypes.c_int64]
         lib.lasad_forward.restype = i32
         lib.lasad_forward.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_decode_step.restype = i32
@@ -147,6 +149,12 @@ class Lasad:
         rc = self._lib.lasad_set_option(self._h, option, value)
         if rc != LASAD_OK:
             raise LasadError(rc, "lasad_set_option")
+
+    def reserve(self, units: int) -> None:
+        """Pre-allocate the context's relay storage for prefill calls with B * H <= units."""
+        rc = self._lib.lasad_reserve(self._h, int(units))
+        if rc != LASAD_OK:
+            self._raise(rc, "lasad_reserve")
 
     @property
     def launch_count(self) -> int:

@@ -15,11 +15,46 @@ struct lasad_ctx {
     int opt_decode_tpu;
     unsigned wait_limit;
     int sm_count;
+    // state relay of the task-streaming prefill (see lasad_prefill_tc_stream.cu)
+    void* d_relay;                // [relay_cap] slots of kTcRelaySlotBytes
+    int64_t relay_cap;
+    uint64_t epoch;               // launches of the task-streaming prefill so far
+    int stream_max_ctas;
 };
 
 namespace {
 
 constexpr unsigned kDefaultWaitLimit = 1u << 22;
+
+constexpr int64_t kDefaultRelayUnits = 1024;   // chains covered by the relay storage lasad_create allocates
+
+// Grows the context-owned relay storage to `units` chains.  Allocates (and therefore
+// synchronises the device) only when the current storage is too small.
+int reserve_units(lasad_ctx* ctx, int64_t units)
+{
+    if (units <= ctx->relay_cap) return LASAD_OK;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();   // an earlier launch may still use the old slots
+    void* nr = nullptr;
+    if (e == cudaSuccess) e = cudaMalloc(&nr, (size_t)units * lasad::kTcRelaySlotBytes);
+    // stale bytes must never look like a tag of a later launch: start from zero (tags are never 0)
+    if (e == cudaSuccess) e = cudaMemset(nr, 0, (size_t)units * lasad::kTcRelaySlotBytes);
+    if (e == cudaSuccess) {
+        if (ctx->d_relay) cudaFree(ctx->d_relay);
+        ctx->d_relay = nr;
+        ctx->relay_cap = units;
+    } else if (nr) {
+        cudaFree(nr);
+    }
+    cudaSetDevice(prev);
+    if (e != cudaSuccess) {
+        ctx->last_cuda_error = (int)e;
+        return LASAD_ERR_CUDA;
+    }
+    return LASAD_OK;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -86,8 +121,12 @@ int lasad_create(lasad_ctx** out, int device)
     if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, 256);
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) ctx->stream_max_ctas = lasad::prefill_stream_max_ctas(device);
     cudaSetDevice(prev);
+    if (e == cudaSuccess && reserve_units(ctx, kDefaultRelayUnits) != LASAD_OK) e = cudaErrorMemoryAllocation;
     if (e != cudaSuccess) {
+        if (ctx->d_status) cudaFree(ctx->d_status);
+        if (ctx->d_relay) cudaFree(ctx->d_relay);
         delete ctx;
         return LASAD_ERR_CUDA;
     }
@@ -99,8 +138,15 @@ int lasad_destroy(lasad_ctx* ctx)
 {
     if (!ctx) return LASAD_ERR_INVALID_ARG;
     if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->d_relay) cudaFree(ctx->d_relay);
     delete ctx;
     return LASAD_OK;
+}
+
+int lasad_reserve(lasad_ctx* ctx, int64_t units)
+{
+    if (!ctx || units <= 0) return LASAD_ERR_INVALID_ARG;
+    return reserve_units(ctx, units);
 }
 
 int lasad_set_option(lasad_ctx* ctx, int option, int value)
@@ -108,7 +154,7 @@ int lasad_set_option(lasad_ctx* ctx, int option, int value)
     if (!ctx) return LASAD_ERR_INVALID_ARG;
     switch (option) {
         case LASAD_OPT_PREFILL_IMPL:
-            if (value < 0 || value > 2) return LASAD_ERR_INVALID_ARG;
+            if (value < 0 || value > 3) return LASAD_ERR_INVALID_ARG;
             ctx->opt_prefill_impl = value;
             return LASAD_OK;
         case LASAD_OPT_PREFILL_CHUNK:
@@ -149,7 +195,34 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
 
     int impl = ctx->opt_prefill_impl;
     const bool tc_ok = lasad::prefill_tc_supported(p->dk, p->dv, bf16);
-    if (impl == 0) impl = tc_ok ? 2 : 1;
+    if (impl == 0) impl = tc_ok ? 3 : 1;
+    if (impl == 3) {
+        if (!tc_ok) return LASAD_ERR_UNSUPPORTED;
+        const int64_t units = (int64_t)p->B * p->H;
+        const int64_t chunks = lasad::prefill_stream_chunks(p->T);
+        if (units * chunks > 0x7fffffffLL || ctx->stream_max_ctas <= 0) return LASAD_ERR_UNSUPPORTED;
+        // the carried state travels from chunk to chunk through context-owned relay slots
+        if (chunks > 1) {
+            rc = reserve_units(ctx, units);
+            if (rc != LASAD_OK) return rc;
+        }
+        lasad::TcRelay r{};
+        r.relay = ctx->d_relay;
+        // The packets' tag holds the launch number modulo 65535; before a value comes round
+        // again the slots are cleared, so that no packet of an old launch can pass for a new one.
+        ctx->epoch += 1;
+        r.epoch16 = (unsigned)(ctx->epoch % 65535u) + 1u;
+        if (ctx->epoch % 65535u == 0 && ctx->d_relay) {
+            const cudaError_t em =
+                cudaMemsetAsync(ctx->d_relay, 0, (size_t)ctx->relay_cap * lasad::kTcRelaySlotBytes, st);
+            if (em != cudaSuccess) return fail_cuda(ctx, em);
+        }
+        r.max_ctas = ctx->stream_max_ctas;
+        const cudaError_t e = lasad::launch_prefill_stream(a, r, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        ctx->launches += 1;
+        return LASAD_OK;
+    }
     if (impl == 2) {
         if (!tc_ok) return LASAD_ERR_UNSUPPORTED;
         const cudaError_t e = lasad::launch_prefill_tc(a, st);

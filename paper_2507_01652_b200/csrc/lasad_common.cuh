@@ -60,6 +60,18 @@ cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool d
                           cudaStream_t st);
 bool prefill_tc_supported(int dk, int dv, bool bf16);
 cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st);
+
+// What the task-streaming tensor-core prefill needs beyond the caller's buffers: the per-chain
+// relay slots through which the carried state passes from one chunk's CTA to the next chunk's.
+struct TcRelay {
+    void* relay;                // [B*H] slots of kTcRelaySlotBytes
+    unsigned epoch16;           // this launch's number folded into 1..65535: part of the packets' tag
+    int max_ctas;               // largest fully resident grid (prefill_stream_max_ctas)
+};
+constexpr long long kTcRelaySlotBytes = 64 * 64 * 8;   // dk * dv values, each with a 4-byte tag
+int prefill_stream_chunks(int T);
+int prefill_stream_max_ctas(int device);
+cudaError_t launch_prefill_stream(const KernelArgs& a, const TcRelay& r, cudaStream_t st);
 cudaError_t launch_prefill_simt(const KernelArgs& a, int dk, int dv, bool bf16, int chunk,
                                 cudaStream_t st);
 

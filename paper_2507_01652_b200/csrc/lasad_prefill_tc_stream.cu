@@ -1,0 +1,758 @@
+// LASAD chunked prefill on the 5th-generation tensor cores (sm_100a), task-streaming form:
+// TMA-fed tcgen05.mma with TMEM accumulators, bf16 I/O, fp32 accumulation, fp32 carried state.
+//
+// Work decomposition.  The sequence of one (batch, head) -- a chain -- is cut into chunks of
+// C = 128 tokens.  One task = one chunk of one chain.  Tasks are numbered chunk-major
+// (id = n * X + x for chunk n of chain x, X = B * H chains) and dealt round-robin to a grid of
+// persistent CTAs, two per SM (256 TMEM columns and ~106 KB of shared memory each): CTA c runs
+// tasks c, c + G, c + 2 G, ...  Everything in a task except the carried state is independent of
+// every other task; the d_k x d_v fp32 state is relayed from the CTA that ran chunk n-1 of the
+// chain to the CTA that runs chunk n through a per-chain slot in global memory (it stays in L2).
+// Consecutive tasks of one CTA belong to different chains, so every SM holds the same amount of
+// work however B * H relates to the SM count, and consecutive chunks of one chain are loaded and
+// multiplied concurrently on different SMs; only the state relay (read 32 KB of packets, fp32
+// update, write 32 KB of packets) is serial along a chain.  Tasks are taken in increasing id and a
+// task only waits for a smaller id, so the grid cannot deadlock as long as all its CTAs are
+// resident (the host sizes the grid from the occupancy query); every wait is bounded anyway.
+//
+// Relay packets.  A state value travels as an 8-byte (value, tag) pair, two pairs per 16-byte
+// access.  An aligned 8-byte access is single-copy atomic, so a pair whose tag matches carries its
+// value: the relay needs no fence and no separate flag (release/acquire at GPU scope stalled for
+// microseconds while bulk copies were in flight).  The tag is the launch number (folded into
+// 1..65535 by the host, which clears the slots before a value comes round again) and the chunk
+// index.  Waiting CTAs poll one packet per warp, never the whole slot.
+//
+// With n_i = number of decaying steps from the chunk start up to and including token i (SAD rule,
+// Section 3.4, from the token's grid position), N = n of the chunk's last token and gamma the
+// head's decay, the SAD recurrence (Section 3.4) unrolled over one chunk is
+//
+//     o_i   = scale * ( sum_{j<=i} (q_i.k_j) gamma^(n_i-n_j) v_j  +  gamma^(n_i) q_i^T S_prev )
+//     S_new = gamma^N S_prev + sum_j gamma^(N-n_j) k_j v_j^T
+//
+// Normal path (gamma >= 0.6, so that gamma^-128 stays far inside fp32 range).  Every decay
+// factor is moved onto V and onto one per-row factor of the output, so that Q and K feed the
+// tensor cores untouched and the scores only need the causal mask:
+//
+//     V~ = diag(gamma^(N-n_j)) V                       in place in smem
+//     dS = K^T V~                        (M2a)         tcgen05.mma 64x64x128
+//     S_new = gamma^N S_prev + dS        (E3)          as soon as S_prev has arrived; relayed on at once
+//     S  = Q K^T                         (M1)          tcgen05.mma 128x128x64, smem x smem
+//     A  = tril(S) -> bf16               (E1)          back into TMEM over S's own columns
+//     O' = A V~ + Q (gamma^N S_prev)     (M2b)         tcgen05.mma 128x64x128 (tmem x smem) + 128x64x64
+//     o_i = scale * gamma^-(N-n_i) * O'_i   (E2)       -> bf16 -> smem -> TMA store
+//
+// Exact path (gamma < 0.6, including 0, where gamma^-(N-n_i) would overflow): only factors
+// with non-negative exponents are formed, all from a table of gamma^m, m = 0..128:
+// P = S o gamma^(n_i-n_j) o [j<=i], Q~ = diag(gamma^(n_i)) Q and K~ = diag(gamma^(N-n_j)) K
+// in place, O = P V + Q~ S_prev, dS = K~^T V.  Same MMAs, same barriers, slower element-wise
+// stages; it exists for correctness over the whole decay range [0, 1].
+//
+// Warp roles: warps 0-7 do the element-wise stages; warp w works on TMEM lane quadrant w & 3
+// (chunk rows 32(w&3)..+31) and the two warps of a quadrant split its columns.  Warp 8
+// allocates TMEM and issues every MMA, warp 9 issues the TMA loads and stores.  All waits are
+// bounded: a wait that runs out raises a status word the host can read and the CTA leaves
+// through the normal exit (copies in flight are waited for, TMEM is freed).
+#include "lasad_common.cuh"
+#include "lasad_tc_ptx.cuh"
+
+namespace lasad {
+namespace {
+
+using namespace tcx;
+
+constexpr int kC = 128;                    // chunk length (tokens) = MMA M
+constexpr int kD = 64;                     // d_k = d_v
+constexpr int kEThreads = 256;             // element-wise warps 0-7
+constexpr int kThreads = kEThreads + 64;   // + the MMA warp and the TMA warp
+constexpr int kTileBytes = kC * kD * 2;    // 16 KB: one [128 x 64] bf16 tile, 128 B rows
+constexpr int kStages = 2;
+constexpr int kTmemCols = 256;
+constexpr uint32_t kColS = 0;      // S (fp32, 128 columns); A/P (bf16 pairs) aliases columns 0..31 and 64..95
+constexpr uint32_t kColO = 128;    // O accumulator, 64 columns
+constexpr uint32_t kColDS = 192;   // dS accumulator (M = 64 layout), 64 columns
+constexpr unsigned kTeardownLimit = 1u << 26;
+constexpr float kFastPathMinDecay = 0.6f;
+
+struct __align__(8) Barriers {
+    unsigned long long full[kStages];   // TMA loads of a stage have landed
+    unsigned long long s_done;     // M1 complete
+    unsigned long long x_ready;    // V~ (normal path) or K~ (exact path) written: dS may start (256 arrivals)
+    unsigned long long ds_done;    // dS MMAs complete
+    unsigned long long p_ready;    // A/P in TMEM (and Q~ in smem) (256 arrivals)
+    unsigned long long sb_ready;   // bf16 copy of the incoming state in smem (256 arrivals)
+    unsigned long long o_done;     // O MMAs complete (and every MMA issued before them)
+    unsigned long long st_ready;   // output tile staged in smem (256 arrivals)
+    unsigned long long tbl_free;   // exact path: every thread is done with the current table (256)
+    unsigned long long tbl_ready;  // exact path: the table of this task's head is written (256)
+    unsigned long long drain;      // teardown: all MMAs retired
+};
+
+struct Smem {
+    // tiles first: each must sit on a 1024-byte boundary (128-byte swizzle atom = 8 rows)
+    unsigned char q[kStages][kTileBytes];
+    unsigned char k[kStages][kTileBytes];
+    unsigned char v[kStages][kTileBytes];
+    unsigned char sb[kD * kD * 2];  // bf16 copy of the incoming state, [dk][dv], 128 B rows, swizzled
+    float pw[kC + 4];               // gamma^m, m = 0..128 (exact path only, rebuilt per task)
+    Barriers bar;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+#ifdef LASAD_TC_TRACE
+// Debug builds only: clock64() stamps of CTA 0's first element-wise thread, 8 slots per task.
+__device__ long long g_stream_trace[4096];
+#define TRACE_E(slot) do { if (blockIdx.x == 0 && tid == 0 && g < 500) g_stream_trace[8 * g + (slot)] = clock64(); } while (0)
+#else
+#define TRACE_E(slot) do { } while (0)
+#endif
+
+struct StreamParams {
+    int B, T, H;
+    int X;                     // chains = B * H
+    int n_chunks;              // chunks per chain
+    int n_tasks;               // X * n_chunks
+    int grid_w, prefix_len;
+    long long t0;
+    float scale;
+    const float* decay;
+    const float* state_in;
+    float* state_out;
+    uint4* relay;              // [X][dk * dv / 2]: two (value, tag) packets per element
+    unsigned epoch16;          // launch number folded into 1..65535: high half of the packets' tag
+    int* status;
+    unsigned wait_limit;
+};
+
+// One task = chunk n of chain x = (b, h).
+struct Task {
+    int n, x, b, h;
+};
+__device__ __forceinline__ Task decode_task(int id, int X, int H)
+{
+    Task t;
+    t.n = id / X;
+    t.x = id - t.n * X;
+    t.b = t.x / H;
+    t.h = t.x - t.b * H;
+    return t;
+}
+
+// Decay bookkeeping of one chunk, computed by every warp on its own with four ballots (one per
+// 32-token block): which steps decay, and from their popcounts n_i for the thread's own row.
+struct ChunkDecay {
+    unsigned mask[4];   // bit l of mask[x]: token 32 x + l of the chunk is a decaying step
+    int cum[4];         // decaying steps up to the end of block x
+    int ni;             // n of the thread's own row
+    int n_last;         // n of the chunk's last token
+    // n of chunk column j (warp-uniform j)
+    __device__ __forceinline__ int n_of(int j) const
+    {
+        const int x = j >> 5;
+        return (x ? cum[x - 1] : 0) + __popc(mask[x] & (0xffffffffu >> (31 - (j & 31))));
+    }
+};
+
+// Where the call sits on the token grid, in a form that needs no division per token: token `tok`
+// of the chunk that starts at call offset cs absorbs the last token of a grid row (a boundary
+// step, SAD rule of Section 3.4) iff it lies on the grid (cs + tok >= pre) and phase + r[tok / 32]
+// is 0 or w, where r = (tok mod w) is fixed per thread and
+// phase = (grid index of the chunk's first token + 1) mod w.
+struct GridPos {
+    int grid_w;
+    int pre;         // tokens of this call that precede the grid (class-token prefix)
+    int r[4];        // (32 x + lane) mod w
+    int step;        // 128 mod w
+    int phase0;      // (grid index of the call's first token + 1) mod w
+};
+
+__device__ __forceinline__ GridPos grid_pos_init(int grid_w, int prefix_len, long long t0, int lane)
+{
+    GridPos g;
+    g.grid_w = grid_w;
+    const long long g0 = t0 - prefix_len;   // grid index of the call's first token (may be < 0)
+    g.pre = g0 < 0 ? (int)min(-g0, (long long)0x7fffffff) : 0;
+    g.step = 0; g.phase0 = 0;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) g.r[x] = 0;
+    if (grid_w > 0) {
+        long long ph = (g0 + 1) % grid_w;    // C remainder: may be negative inside the prefix
+        if (ph < 0) ph += grid_w;
+        g.phase0 = (int)ph;
+        g.step = kC % grid_w;
+#pragma unroll
+        for (int x = 0; x < 4; ++x) g.r[x] = (32 * x + lane) % grid_w;
+    }
+    return g;
+}
+
+// Decay bookkeeping of chunk n of the call (L live tokens).
+__device__ __forceinline__ ChunkDecay chunk_decay(const GridPos& g, int n, int L, int qd, int lane)
+{
+    ChunkDecay d;
+    int phase = 0;
+    if (g.grid_w > 0) {
+        // (phase0 + n * 128) mod w, with a 64-bit division only for very wide grids
+        const unsigned w = (unsigned)g.grid_w;
+        const unsigned long long prod = (unsigned long long)((unsigned)n % w) * (unsigned)g.step + (unsigned)g.phase0;
+        phase = prod < 0x100000000ull ? (int)((unsigned)prod % w) : (int)(prod % w);
+    }
+    const int cs = n * kC;
+    int run = 0;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const int tok = 32 * x + lane;
+        const int m = phase + g.r[x];
+        const bool boundary = g.grid_w > 0 && cs + tok >= g.pre && (m == 0 || m == g.grid_w);
+        d.mask[x] = __ballot_sync(0xffffffffu, tok < L && !boundary);
+        run += __popc(d.mask[x]);
+        d.cum[x] = run;
+    }
+    d.n_last = run;
+    const unsigned own = qd == 0 ? d.mask[0] : qd == 1 ? d.mask[1] : qd == 2 ? d.mask[2] : d.mask[3];
+    const int before = qd == 0 ? 0 : qd == 1 ? d.cum[0] : qd == 2 ? d.cum[1] : d.cum[2];
+    d.ni = before + __popc(own & (0xffffffffu >> (31 - lane)));
+    return d;
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                      StreamParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int G = (int)gridDim.x;
+    const int first = (int)blockIdx.x;
+    // tasks of this CTA: first, first + G, ...
+    const int n_local = first < p.n_tasks ? (p.n_tasks - first + G - 1) / G : 0;
+    volatile int* abort_flag = &sm.abort_flag;
+    const unsigned limit = p.wait_limit;
+
+    // ---- set-up ---------------------------------------------------------------------------
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(&sm.bar.full[s], 1);
+        mbar_init(&sm.bar.s_done, 1);
+        mbar_init(&sm.bar.x_ready, kEThreads);
+        mbar_init(&sm.bar.ds_done, 1);
+        mbar_init(&sm.bar.p_ready, kEThreads);
+        mbar_init(&sm.bar.sb_ready, kEThreads);
+        mbar_init(&sm.bar.o_done, 1);
+        mbar_init(&sm.bar.st_ready, kEThreads);
+        mbar_init(&sm.bar.tbl_free, kEThreads);
+        mbar_init(&sm.bar.tbl_ready, kEThreads);
+        mbar_init(&sm.bar.drain, 1);
+        sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 8) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    if (warp == 9) {
+        // ===================== TMA warp: loads two tasks ahead, stores each output tile ========
+        if (lane == 0) {
+            auto issue_loads = [&](int g) {
+                const Task t = decode_task(first + g * G, p.X, p.H);
+                const int s = g % kStages;
+                mbar_arrive_expect_tx(&sm.bar.full[s], 3 * kTileBytes);
+                tma_load_4d(sm.q[s], &tm_q, &sm.bar.full[s], 0, t.h, t.n * kC, t.b);
+                tma_load_4d(sm.k[s], &tm_k, &sm.bar.full[s], 0, t.h, t.n * kC, t.b);
+                tma_load_4d(sm.v[s], &tm_v, &sm.bar.full[s], 0, t.h, t.n * kC, t.b);
+            };
+            int loads_issued = min(n_local, kStages);
+            for (int g = 0; g < loads_issued; ++g) issue_loads(g);
+            for (int g = 0; g < n_local; ++g) {
+                const int s = g % kStages;
+                // the output tile of task g sits in the Q buffer of its stage; by now every MMA
+                // that read this stage has retired (the element-wise warps waited for o_done)
+                if (!mbar_wait(&sm.bar.st_ready, g & 1, limit, abort_flag, p.status)) break;
+                const Task t = decode_task(first + g * G, p.X, p.H);
+                tma_store_4d(&tm_o, sm.q[s], 0, t.h, t.n * kC, t.b);
+                tma_store_commit();
+                if (g + kStages < n_local) {
+                    tma_store_wait_read();        // the store has finished reading the buffer
+                    issue_loads(g + kStages);
+                    loads_issued = g + kStages + 1;
+                }
+            }
+            tma_store_wait_all();
+            // leave only when every issued load has landed (they write this CTA's shared memory)
+            for (int g = max(0, loads_issued - kStages); g < loads_issued; ++g)
+                for (unsigned it = 0; it < kTeardownLimit; ++it)
+                    if (mbar_try_wait(&sm.bar.full[g % kStages], (g / kStages) & 1)) break;
+        }
+        __syncwarp();
+    } else if (warp == 8) {
+        // ===================== MMA issuer: the whole warp runs the loop, one lane issues =======
+        constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);   // Q (K-major) x K (K-major)
+        constexpr uint32_t idesc_pv = make_idesc(128, 64, 0, 1);   // A/P (tmem) x V (MN-major)
+        constexpr uint32_t idesc_qs = make_idesc(128, 64, 0, 1);   // Q (K-major) x state (MN-major)
+        constexpr uint32_t idesc_kv = make_idesc(64, 64, 1, 1);    // K^T (MN-major) x V (MN-major)
+        const uint64_t d_sb = make_desc(smem_u32(sm.sb));
+        const uint64_t dq0 = make_desc(smem_u32(sm.q[0])), dq1 = make_desc(smem_u32(sm.q[1]));
+        const uint64_t dk0 = make_desc(smem_u32(sm.k[0])), dk1 = make_desc(smem_u32(sm.k[1]));
+        const uint64_t dv0 = make_desc(smem_u32(sm.v[0])), dv1 = make_desc(smem_u32(sm.v[1]));
+        auto issue_m1 = [&](int g) {
+            const uint64_t dq = (g & 1) ? dq1 : dq0, dk = (g & 1) ? dk1 : dk0;
+            tc_fence_after();
+            if (lane == 0) {
+#pragma unroll
+                for (int kk = 0; kk < kD / 16; ++kk)  // 32 bytes along K per step
+                    mma_ss(tmem + kColS, dq + 2 * kk, dk + 2 * kk, idesc_s, kk > 0);
+                mma_commit(&sm.bar.s_done);
+            }
+            __syncwarp();
+        };
+        bool ok = n_local > 0 && mbar_wait(&sm.bar.full[0], 0, limit, abort_flag, p.status);
+        if (ok) issue_m1(0);
+        for (int g = 0; ok && g < n_local; ++g) {
+            const uint64_t dq = (g & 1) ? dq1 : dq0, dk = (g & 1) ? dk1 : dk0, dv = (g & 1) ? dv1 : dv0;
+            if (!mbar_wait(&sm.bar.x_ready, g & 1, limit, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            if (lane == 0) {
+#pragma unroll
+                for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K and of V per step
+                    mma_ss(tmem + kColDS, dk + 128 * kk, dv + 128 * kk, idesc_kv, kk > 0);
+                mma_commit(&sm.bar.ds_done);
+            }
+            __syncwarp();
+            if (!mbar_wait(&sm.bar.p_ready, g & 1, limit, abort_flag, p.status)) { ok = false; break; }
+            if (!mbar_wait(&sm.bar.sb_ready, g & 1, limit, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            if (lane == 0) {
+#pragma unroll
+                for (int kk = 0; kk < kC / 16; ++kk)  // A/P: 8 TMEM columns per step (tokens 0..63 at columns
+                                                      // 0..31, tokens 64..127 at 64..95); V: 2048 B per step
+                    mma_ts(tmem + kColO, tmem + kColS + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), dv + 128 * kk,
+                           idesc_pv, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < kD / 16; ++kk)
+                    mma_ss(tmem + kColO, dq + 2 * kk, d_sb + 128 * kk, idesc_qs, 1);
+                mma_commit(&sm.bar.o_done);
+            }
+            __syncwarp();
+            // the scores of the next task (they overwrite A's columns: the tensor pipe runs in
+            // issue order, so the A V MMAs above read A first)
+            if (g + 1 < n_local) {
+                if (!mbar_wait(&sm.bar.full[(g + 1) % kStages], ((g + 1) / kStages) & 1, limit, abort_flag, p.status)) {
+                    ok = false;
+                    break;
+                }
+                issue_m1(g + 1);
+            }
+        }
+        // make sure nothing is still running on the tensor pipe before TMEM is freed
+        if (lane == 0) {
+            mma_commit(&sm.bar.drain);
+            for (unsigned it = 0; it < kTeardownLimit; ++it)
+                if (mbar_try_wait(&sm.bar.drain, 0)) break;
+        }
+        __syncwarp();
+    } else {
+        // ===================== element-wise warps ==============================================
+        const int qd = warp & 3;                 // TMEM lane quadrant
+        const int grp = warp >> 2;               // which half of the quadrant's columns
+        const int i = qd * 32 + lane;            // chunk row owned by this thread
+        const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+        const int srow = qd * 16 + lane;         // state row (M = 64 TMEM layout: lanes 0..15 of a quadrant)
+        const bool has_state = lane < 16;
+        const size_t st_off = (size_t)srow * kD + 32 * grp;   // this thread's 32 state elements in a slot
+
+        // position of the call's first token relative to the grid (SAD rule, Section 3.4)
+        const GridPos gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0, lane);
+
+        float st[32];                            // state[srow][32 grp .. 32 grp + 31]
+        auto load_state = [&](const float* src_state) {
+            if (has_state) {
+                const float4* src = reinterpret_cast<const float4*>(src_state + st_off);
+#pragma unroll
+                for (int e4 = 0; e4 < 8; ++e4) {
+                    const float4 t = __ldcg(src + e4);
+                    st[4 * e4] = t.x; st[4 * e4 + 1] = t.y; st[4 * e4 + 2] = t.z; st[4 * e4 + 3] = t.w;
+                }
+            }
+        };
+        auto store_state = [&](float* dst_state) {
+            if (has_state) {
+                float4* dst = reinterpret_cast<float4*>(dst_state + st_off);
+#pragma unroll
+                for (int e4 = 0; e4 < 8; ++e4)
+                    dst[e4] = make_float4(st[4 * e4], st[4 * e4 + 1], st[4 * e4 + 2], st[4 * e4 + 3]);
+            }
+        };
+        // relay: this thread's 32 state values travel as 32 tagged packets in 16 stores
+        auto relay_out = [&](uint4* slot, uint32_t tag) {
+            if (has_state) {
+                uint4* dst = slot + st_off / 2;
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    st_cg_v4(dst + j, make_uint4(__float_as_uint(st[2 * j]), tag, __float_as_uint(st[2 * j + 1]), tag));
+            }
+        };
+        // Cheap look at the relay slot: one lane per warp reads the last packets of its row (the
+        // writer stores a thread's packets in ascending order, so these usually land last).
+        // Polling loops use this, never the full read, so that waiting CTAs do not load L2 with
+        // 32 KB per poll.
+        auto relay_peek = [&](const uint4* slot, uint32_t tag) {
+            bool hit = true;
+            if (lane == 15) {
+                const uint4 v = ld_cg_v4(slot + st_off / 2 + 15);
+                hit = v.y == tag && v.w == tag;
+            }
+            return __all_sync(0xffffffffu, hit);
+        };
+        // one pass over the thread's packets, eight 16-byte loads in flight at a time; true when
+        // every tag matched (warp-uniform result)
+        auto relay_in_once = [&](const uint4* slot, uint32_t tag) {
+            bool all = true;
+            if (has_state) {
+                const uint4* src = slot + st_off / 2;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    uint4 v[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[j] = ld_cg_v4(src + 8 * half + j);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        st[16 * half + 2 * j] = __uint_as_float(v[j].x);
+                        st[16 * half + 2 * j + 1] = __uint_as_float(v[j].z);
+                        all = all && v[j].y == tag && v[j].w == tag;
+                    }
+                }
+            }
+            return __all_sync(0xffffffffu, all);
+        };
+        // bf16 copy of mult * state for the Q x state MMAs
+        auto write_state_bf16 = [&](float mult) {
+            if (has_state) {
+                uint4* row = reinterpret_cast<uint4*>(sm.sb + srow * 128);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint4 x;
+                    x.x = pack_bf16(mult * st[8 * c], mult * st[8 * c + 1]);
+                    x.y = pack_bf16(mult * st[8 * c + 2], mult * st[8 * c + 3]);
+                    x.z = pack_bf16(mult * st[8 * c + 4], mult * st[8 * c + 5]);
+                    x.w = pack_bf16(mult * st[8 * c + 6], mult * st[8 * c + 7]);
+                    row[(4 * grp + c) ^ (srow & 7)] = x;
+                }
+            }
+        };
+        // E3: S_new = g * S_prev + dS (this thread's 32 columns of its state row)
+        auto update_state = [&](float g) {
+            uint32_t dsv[32];
+            tmem_ld32(tmem + lane_base + kColDS + 32 * grp, dsv);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) st[e] = fmaf(g, st[e], __uint_as_float(dsv[e]));
+        };
+        // E2: this thread's 32 columns of output row i -> bf16 -> the stage's Q buffer
+        auto stage_output = [&](int s, float f) {
+            unsigned char* orow = sm.q[s] + i * 128;
+            uint32_t ov[32];
+            tmem_ld32(tmem + lane_base + kColO + 32 * grp, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint4 x;
+                x.x = pack_bf16(f * __uint_as_float(ov[8 * c]), f * __uint_as_float(ov[8 * c + 1]));
+                x.y = pack_bf16(f * __uint_as_float(ov[8 * c + 2]), f * __uint_as_float(ov[8 * c + 3]));
+                x.z = pack_bf16(f * __uint_as_float(ov[8 * c + 4]), f * __uint_as_float(ov[8 * c + 5]));
+                x.w = pack_bf16(f * __uint_as_float(ov[8 * c + 6]), f * __uint_as_float(ov[8 * c + 7]));
+                reinterpret_cast<uint4*>(orow)[(4 * grp + c) ^ (i & 7)] = x;
+            }
+        };
+
+        bool ok = true;
+        unsigned exact_tasks = 0;    // exact-path tasks this CTA has run (phase of the table barriers)
+        for (int g = 0; ok && g < n_local; ++g) {
+            const Task t = decode_task(first + g * G, p.X, p.H);
+            const int s = g % kStages;
+            const unsigned par = g & 1;
+            TRACE_E(0);
+            const float gamma = p.decay[t.h];
+            const bool fast = gamma >= kFastPathMinDecay;
+            const bool last_chunk = t.n + 1 == p.n_chunks;
+            const ChunkDecay cd = chunk_decay(gp, t.n, min(kC, p.T - t.n * kC), qd, lane);
+            uint4* const slot = p.relay ? p.relay + (size_t)t.x * (kD * kD / 2) : nullptr;
+            // tag of the state after chunk n - 1 of this launch (what this task consumes): launch
+            // number and chunk index; the state this task produces carries the next tag
+            const uint32_t tag_in = (p.epoch16 << 16) | ((uint32_t)t.n & 0xffffu);
+            const uint32_t tag_out = (p.epoch16 << 16) | ((uint32_t)(t.n + 1) & 0xffffu);
+
+            // gamma^m: normal path straight from exp2 (|m log2 gamma| <= 95, relative error ~1e-5);
+            // exact path from a table in double precision (0^0 = 1), rebuilt for this task's head
+            const float lg = fast ? log2f(gamma) : 0.0f;
+            auto gpow = [&](int m) { return exp2f((float)m * lg); };
+            if (!fast) {
+                // every thread is done with the previous exact task's table before it is rewritten
+                if (exact_tasks > 0 &&
+                    !(ok = mbar_wait(&sm.bar.tbl_free, (exact_tasks - 1) & 1, limit, abort_flag, p.status))) break;
+                if (tid <= kC) {
+                    double base = (double)gamma, acc = 1.0;
+                    for (int e = tid; e > 0; e >>= 1) {
+                        if (e & 1) acc *= base;
+                        base *= base;
+                    }
+                    sm.pw[tid] = (float)acc;
+                }
+                mbar_arrive(&sm.bar.tbl_ready);
+                if (!(ok = mbar_wait(&sm.bar.tbl_ready, exact_tasks & 1, limit, abort_flag, p.status))) break;
+            }
+            const float g_chunk = fast ? gpow(cd.n_last) : sm.pw[cd.n_last];   // gamma^N
+
+            // ---- operand scaling that the dS MMAs wait for ---------------------------------------
+            bool s_seen = false;
+            if (fast) {
+                // V~ = diag(gamma^(N - n_j)) V, in place
+                if (!(ok = mbar_wait(&sm.bar.full[s], (g / kStages) & 1, limit, abort_flag, p.status))) break;
+                scale_row_inplace<4>(sm.v[s] + i * 128, gpow(cd.n_last - cd.ni), 4 * grp, i & 7);
+            } else {
+                // K~ = diag(gamma^(N - n_j)) K, in place, once M1 has read K
+                if (!(ok = mbar_wait(&sm.bar.s_done, par, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+                s_seen = true;
+                if (grp == 1) scale_row_inplace<8>(sm.k[s] + i * 128, sm.pw[cd.n_last - cd.ni], 0, i & 7);
+            }
+            fence_proxy_async();
+            mbar_arrive(&sm.bar.x_ready);
+            TRACE_E(1);
+
+            // ---- incoming state: chunk 0 takes state_in; later chunks take the chain's relay slot
+            //      as soon as every packet carries the tag of chunk n - 1.  The state recurrence is
+            //      the only serial link along a chain, so it goes first when the state is already
+            //      here; otherwise E1, which needs no state, fills the wait.
+            bool have_state = true;
+            if (t.n == 0) {
+                if (p.state_in) {
+                    load_state(p.state_in + (size_t)t.x * (kD * kD));
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) st[e] = 0.0f;
+                }
+            } else {
+                have_state = relay_peek(slot, tag_in) && relay_in_once(slot, tag_in);
+            }
+            TRACE_E(2);
+#pragma unroll 1
+            for (int step = 0; ok && step < 2; ++step) {
+                if ((step == 0) == have_state) {
+                    // ---- state section: wait for the state if it is not here yet -----------------
+                    if (!have_state) {
+                        bool got = false;
+                        for (unsigned it = 0; it < limit; ++it) {
+                            if (relay_peek(slot, tag_in) && relay_in_once(slot, tag_in)) { got = true; break; }
+                            if ((it & 15u) == 15u && *abort_flag) break;
+                            __nanosleep(64);
+                        }
+                        if (!got) {
+                            if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, 1); }
+                            ok = false;
+                            break;
+                        }
+                    }
+                    TRACE_E(4);
+                    write_state_bf16(fast ? g_chunk : 1.0f);   // gamma^N S_prev (normal) / S_prev (exact: Q~ carries gamma^n_i)
+                    fence_proxy_async();
+                    mbar_arrive(&sm.bar.sb_ready);
+                    // E3: S_new = gamma^N S_prev + dS, then hand it to the chain's next chunk
+                    if (!(ok = mbar_wait(&sm.bar.ds_done, par, limit, abort_flag, p.status))) break;
+                    tc_fence_after();
+                    update_state(g_chunk);
+                    if (!last_chunk) {
+                        relay_out(slot, tag_out);
+                    } else if (p.state_out) {
+                        store_state(p.state_out + (size_t)t.x * (kD * kD));
+                    }
+                    TRACE_E(5);
+                } else {
+                    // ---- E1: A = tril(S) (normal) or P = S o gamma^(n_i - n_j) o [j <= i] (exact)
+                    //      -> bf16 over S's own columns.  This warp converts the 32-column blocks
+                    //      2 grp and 2 grp + 1 of its rows and keeps the result inside its own half
+                    //      of S's columns (block pc -> columns 64 grp + 16 (pc & 1), always behind
+                    //      this warp's own reads); the A V MMAs walk the columns in that order.
+                    if (!s_seen) {
+                        if (!(ok = mbar_wait(&sm.bar.s_done, par, limit, abort_flag, p.status))) break;
+                        tc_fence_after();
+                    }
+                    if (fast) {
+#pragma unroll
+                        for (int pi = 0; pi < 2; ++pi) {
+                            const int pc = 2 * grp + pi;
+                            uint32_t pk[16];
+                            if (pc <= qd) {
+                                uint32_t sv[32];
+                                tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
+                                tmem_wait_ld();
+                                if (pc < qd) {
+#pragma unroll
+                                    for (int c = 0; c < 16; ++c)
+                                        pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
+                                } else {
+#pragma unroll
+                                    for (int c = 0; c < 16; ++c)
+                                        pk[c] = pack_bf16(2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
+                                                          2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
+                                }
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                            }
+                            tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
+                        }
+                    } else {
+#pragma unroll 1
+                        for (int pi = 0; pi < 2; ++pi) {
+                            const int pc = 2 * grp + pi;
+                            uint32_t pk[16];
+                            if (pc <= qd) {
+                                uint32_t sv[32];
+                                tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int c = 0; c < 16; ++c) {
+                                    const int j0 = 32 * pc + 2 * c;
+                                    const int d0 = cd.ni - cd.n_of(j0), d1 = cd.ni - cd.n_of(j0 + 1);
+                                    const float v0 = j0 <= i ? __uint_as_float(sv[2 * c]) * sm.pw[d0 > 0 ? d0 : 0] : 0.0f;
+                                    const float v1 = j0 + 1 <= i ? __uint_as_float(sv[2 * c + 1]) * sm.pw[d1 > 0 ? d1 : 0] : 0.0f;
+                                    pk[c] = pack_bf16(v0, v1);
+                                }
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                            }
+                            tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
+                        }
+                        if (grp == 0) scale_row_inplace<8>(sm.q[s] + i * 128, sm.pw[cd.ni], 0, i & 7);   // Q~
+                    }
+                    tmem_wait_st();
+                    fence_proxy_async();
+                    tc_fence_before();
+                    mbar_arrive(&sm.bar.p_ready);
+                    if (!fast) {
+                        mbar_arrive(&sm.bar.tbl_free);    // last use of the table in this task
+                        ++exact_tasks;
+                    }
+                    TRACE_E(3);
+                }
+            }
+            if (!ok) break;
+
+            // ---- E2: o_i = scale * gamma^-(N - n_i) * O'_i (normal) / scale * O_i (exact) -----------
+            const float out_f = fast ? p.scale * gpow(-(cd.n_last - cd.ni)) : p.scale;
+            if (!(ok = mbar_wait(&sm.bar.o_done, par, limit, abort_flag, p.status))) break;
+            tc_fence_after();
+            TRACE_E(6);
+            stage_output(s, out_f);
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(&sm.bar.st_ready);
+            TRACE_E(7);
+        }
+    }
+
+    // ---- teardown ---------------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// cuTensorMapEncodeTiled, fetched through the runtime so that the library does not link libcuda.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// [B,T,H,64] bf16 with element strides (b,t,h) -> 4-D map (d, h, t, b), box = one chunk of one head.
+bool encode_map(CUtensorMap* map, const void* base, int B, int T, int H, const long long* strides)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    auto bytes = [](long long elems) { return (cuuint64_t)(elems > 0 ? elems * 2 : 128); };
+    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
+    const cuuint64_t gstr[3] = {bytes(strides[2]), bytes(strides[1]), bytes(strides[0])};
+    const cuuint32_t box[4] = {(cuuint32_t)kD, 1u, (cuuint32_t)kC, 1u};
+    const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, gstr, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+#ifdef LASAD_TC_TRACE
+extern "C" int lasad_debug_read_stream_trace(long long* host, int n)
+{
+    return (int)cudaMemcpyFromSymbol(host, g_stream_trace, sizeof(long long) * n);
+}
+#endif
+
+int prefill_stream_chunks(int T) { return (T + kC - 1) / kC; }
+
+// Largest grid whose CTAs are all resident at once on `device` (the state relay needs that).
+int prefill_stream_max_ctas(int device)
+{
+    static int cached[64] = {0};
+    if (device >= 0 && device < 64 && cached[device] > 0) return cached[device];
+    const size_t smem = sizeof(Smem) + 1024;
+    int per_sm = 0, sms = 0;
+    if (cudaFuncSetAttribute(prefill_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, prefill_stream_kernel, kThreads, smem) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+        return 0;
+    const int n = per_sm * sms;
+    if (device >= 0 && device < 64) cached[device] = n;
+    return n;
+}
+
+cudaError_t launch_prefill_stream(const KernelArgs& a, const TcRelay& r, cudaStream_t st)
+{
+    CUtensorMap mq, mk, mv, mo;
+    if (!encode_map(&mq, a.q, a.B, a.T, a.H, a.qs) || !encode_map(&mk, a.k, a.B, a.T, a.H, a.ks) ||
+        !encode_map(&mv, a.v, a.B, a.T, a.H, a.vs) || !encode_map(&mo, a.o, a.B, a.T, a.H, a.os))
+        return cudaErrorInvalidValue;
+    StreamParams p;
+    p.B = a.B; p.T = a.T; p.H = a.H;
+    p.X = a.B * a.H;
+    p.n_chunks = prefill_stream_chunks(a.T);
+    p.n_tasks = p.X * p.n_chunks;
+    p.grid_w = a.grid_w; p.prefix_len = a.prefix_len; p.t0 = a.t0; p.scale = a.scale;
+    p.decay = a.decay; p.state_in = a.state_in; p.state_out = a.state_out;
+    p.relay = static_cast<uint4*>(r.relay); p.epoch16 = r.epoch16;
+    p.status = a.status; p.wait_limit = a.wait_limit;
+    if (r.max_ctas <= 0 || (p.n_chunks > 1 && !p.relay)) return cudaErrorInvalidValue;
+    const size_t smem = sizeof(Smem) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(prefill_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const int grid = p.n_tasks < r.max_ctas ? p.n_tasks : r.max_ctas;
+    prefill_stream_kernel<<<(unsigned)grid, kThreads, smem, st>>>(mq, mk, mv, mo, p);
+    return cudaGetLastError();
+}
+
+}  // namespace lasad

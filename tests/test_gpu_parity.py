@@ -14,7 +14,7 @@ from tests._util import TOL, oracle, rel_err, to64
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = [1, 2]  # 1 = CUDA-core fp32 kernel, 2 = tcgen05 tensor-core kernel
+IMPLS = [1, 2, 3]  # 1 = CUDA-core fp32 kernel, 2 = tcgen05 kernel (CTA per chain), 3 = tcgen05 task-streaming kernel
 
 
 @pytest.fixture(scope="module")

@@ -55,6 +55,9 @@
 #include "lasad_common.cuh"
 #include "lasad_tc_ptx.cuh"
 
+#include <cstdio>
+#include <cstdlib>
+
 namespace lasad {
 namespace {
 
@@ -141,15 +144,17 @@ __device__ __forceinline__ Task decode_task(int id, int X, int H)
 // Decay bookkeeping of one chunk, computed by every warp on its own with four ballots (one per
 // 32-token block): which steps decay, and from their popcounts n_i for the thread's own row.
 struct ChunkDecay {
-    unsigned mask[4];   // bit l of mask[x]: token 32 x + l of the chunk is a decaying step
-    int cum[4];         // decaying steps up to the end of block x
-    int ni;             // n of the thread's own row
-    int n_last;         // n of the chunk's last token
+    unsigned m0, m1, m2, m3;   // bit l of m<x>: token 32 x + l of the chunk is a decaying step
+    int c0, c1, c2;            // decaying steps up to the end of block 0, 1, 2
+    int ni;                    // n of the thread's own row
+    int n_last;                // n of the chunk's last token
     // n of chunk column j (warp-uniform j)
     __device__ __forceinline__ int n_of(int j) const
     {
         const int x = j >> 5;
-        return (x ? cum[x - 1] : 0) + __popc(mask[x] & (0xffffffffu >> (31 - (j & 31))));
+        const unsigned m = x == 0 ? m0 : x == 1 ? m1 : x == 2 ? m2 : m3;
+        const int before = x == 0 ? 0 : x == 1 ? c0 : x == 2 ? c1 : c2;
+        return before + __popc(m & (0xffffffffu >> (31 - (j & 31))));
     }
 };
 
@@ -198,19 +203,21 @@ __device__ __forceinline__ ChunkDecay chunk_decay(const GridPos& g, int n, int L
         phase = prod < 0x100000000ull ? (int)((unsigned)prod % w) : (int)(prod % w);
     }
     const int cs = n * kC;
-    int run = 0;
+    unsigned mk[4];
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
         const int tok = 32 * x + lane;
         const int m = phase + g.r[x];
         const bool boundary = g.grid_w > 0 && cs + tok >= g.pre && (m == 0 || m == g.grid_w);
-        d.mask[x] = __ballot_sync(0xffffffffu, tok < L && !boundary);
-        run += __popc(d.mask[x]);
-        d.cum[x] = run;
+        mk[x] = __ballot_sync(0xffffffffu, tok < L && !boundary);
     }
-    d.n_last = run;
-    const unsigned own = qd == 0 ? d.mask[0] : qd == 1 ? d.mask[1] : qd == 2 ? d.mask[2] : d.mask[3];
-    const int before = qd == 0 ? 0 : qd == 1 ? d.cum[0] : qd == 2 ? d.cum[1] : d.cum[2];
+    d.m0 = mk[0]; d.m1 = mk[1]; d.m2 = mk[2]; d.m3 = mk[3];
+    d.c0 = __popc(d.m0);
+    d.c1 = d.c0 + __popc(d.m1);
+    d.c2 = d.c1 + __popc(d.m2);
+    d.n_last = d.c2 + __popc(d.m3);
+    const unsigned own = qd == 0 ? d.m0 : qd == 1 ? d.m1 : qd == 2 ? d.m2 : d.m3;
+    const int before = qd == 0 ? 0 : qd == 1 ? d.c0 : qd == 2 ? d.c1 : d.c2;
     d.ni = before + __popc(own & (0xffffffffu >> (31 - lane)));
     return d;
 }
@@ -372,104 +379,111 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         // position of the call's first token relative to the grid (SAD rule, Section 3.4)
         const GridPos gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0, lane);
 
-        float st[32];                            // state[srow][32 grp .. 32 grp + 31]
-        auto load_state = [&](const float* src_state) {
-            if (has_state) {
-                const float4* src = reinterpret_cast<const float4*>(src_state + st_off);
+        // Inside a relay slot the packets are laid out for coalescing, not by state index: the
+        // 16-byte word j of the rp-th state-holding thread sits at word j * 128 + rp, so that a
+        // warp's access covers 256 contiguous bytes (both sides use the same thread mapping).
+        constexpr int kRelayThreads = kEThreads / 2;
+        const int rp = warp * 16 + lane;
+        // The thread's 32 state values (state[srow][32 grp .. 32 grp + 31]) are handled as two halves
+        // of 16, one after the other, to keep the register footprint of the relay small.
+        float st[16];
+        auto load_state_half = [&](const float* src_state, int hh) {
 #pragma unroll
-                for (int e4 = 0; e4 < 8; ++e4) {
+            for (int e = 0; e < 16; ++e) st[e] = 0.0f;
+            if (has_state) {
+                const float4* src = reinterpret_cast<const float4*>(src_state + st_off + 16 * hh);
+#pragma unroll
+                for (int e4 = 0; e4 < 4; ++e4) {
                     const float4 t = __ldcg(src + e4);
                     st[4 * e4] = t.x; st[4 * e4 + 1] = t.y; st[4 * e4 + 2] = t.z; st[4 * e4 + 3] = t.w;
                 }
             }
         };
-        auto store_state = [&](float* dst_state) {
+        auto store_state_half = [&](float* dst_state, int hh) {
             if (has_state) {
-                float4* dst = reinterpret_cast<float4*>(dst_state + st_off);
+                float4* dst = reinterpret_cast<float4*>(dst_state + st_off + 16 * hh);
 #pragma unroll
-                for (int e4 = 0; e4 < 8; ++e4)
+                for (int e4 = 0; e4 < 4; ++e4)
                     dst[e4] = make_float4(st[4 * e4], st[4 * e4 + 1], st[4 * e4 + 2], st[4 * e4 + 3]);
             }
         };
-        // relay: this thread's 32 state values travel as 32 tagged packets in 16 stores
-        auto relay_out = [&](uint4* slot, uint32_t tag) {
+        // relay: 16 state values travel as 16 tagged packets in 8 stores
+        auto relay_out_half = [&](uint4* slot, uint32_t tag, int hh) {
             if (has_state) {
-                uint4* dst = slot + st_off / 2;
+                uint4* dst = slot + (8 * hh) * kRelayThreads + rp;
 #pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    st_cg_v4(dst + j, make_uint4(__float_as_uint(st[2 * j]), tag, __float_as_uint(st[2 * j + 1]), tag));
+                for (int j = 0; j < 8; ++j)
+                    st_cg_v4(dst + j * kRelayThreads, make_uint4(__float_as_uint(st[2 * j]), tag, __float_as_uint(st[2 * j + 1]), tag));
             }
         };
-        // Cheap look at the relay slot: one lane per warp reads the last packets of its row (the
-        // writer stores a thread's packets in ascending order, so these usually land last).
-        // Polling loops use this, never the full read, so that waiting CTAs do not load L2 with
-        // 32 KB per poll.
-        auto relay_peek = [&](const uint4* slot, uint32_t tag) {
+        // Cheap look at the relay slot: one lane per warp reads the last packets of its half row
+        // (the writer stores them in ascending order, so these usually land last).  Polling loops
+        // use this, never the full read, so that waiting CTAs do not load L2 with 32 KB per poll.
+        auto relay_peek = [&](const uint4* slot, uint32_t tag, int hh) {
             bool hit = true;
             if (lane == 15) {
-                const uint4 v = ld_cg_v4(slot + st_off / 2 + 15);
+                const uint4 v = ld_cg_v4(slot + (8 * hh + 7) * kRelayThreads + rp);
                 hit = v.y == tag && v.w == tag;
             }
             return __all_sync(0xffffffffu, hit);
         };
-        // one pass over the thread's packets, eight 16-byte loads in flight at a time; true when
-        // every tag matched (warp-uniform result)
-        auto relay_in_once = [&](const uint4* slot, uint32_t tag) {
+        // one pass over the half's packets; true when every tag matched (warp-uniform result)
+        auto relay_in_half = [&](const uint4* slot, uint32_t tag, int hh) {
             bool all = true;
+#pragma unroll
+            for (int e = 0; e < 16; ++e) st[e] = 0.0f;
             if (has_state) {
-                const uint4* src = slot + st_off / 2;
+                const uint4* src = slot + (8 * hh) * kRelayThreads + rp;
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint4 v[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) v[j] = ld_cg_v4(src + 8 * half + j);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        st[16 * half + 2 * j] = __uint_as_float(v[j].x);
-                        st[16 * half + 2 * j + 1] = __uint_as_float(v[j].z);
-                        all = all && v[j].y == tag && v[j].w == tag;
-                    }
+                for (int j = 0; j < 8; ++j) {
+                    const uint4 v = ld_cg_v4(src + j * kRelayThreads);
+                    st[2 * j] = __uint_as_float(v.x);
+                    st[2 * j + 1] = __uint_as_float(v.z);
+                    all = all && v.y == tag && v.w == tag;
                 }
             }
             return __all_sync(0xffffffffu, all);
         };
-        // bf16 copy of mult * state for the Q x state MMAs
-        auto write_state_bf16 = [&](float mult) {
+        // bf16 copy of mult * state half for the Q x state MMAs
+        auto write_state_bf16_half = [&](float mult, int hh) {
             if (has_state) {
                 uint4* row = reinterpret_cast<uint4*>(sm.sb + srow * 128);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     uint4 x;
                     x.x = pack_bf16(mult * st[8 * c], mult * st[8 * c + 1]);
                     x.y = pack_bf16(mult * st[8 * c + 2], mult * st[8 * c + 3]);
                     x.z = pack_bf16(mult * st[8 * c + 4], mult * st[8 * c + 5]);
                     x.w = pack_bf16(mult * st[8 * c + 6], mult * st[8 * c + 7]);
-                    row[(4 * grp + c) ^ (srow & 7)] = x;
+                    row[(4 * grp + 2 * hh + c) ^ (srow & 7)] = x;
                 }
             }
         };
-        // E3: S_new = g * S_prev + dS (this thread's 32 columns of its state row)
-        auto update_state = [&](float g) {
-            uint32_t dsv[32];
-            tmem_ld32(tmem + lane_base + kColDS + 32 * grp, dsv);
+        // E3: S_new = g * S_prev + dS for the half
+        auto update_state_half = [&](float g, int hh) {
+            uint32_t dsv[16];
+            tmem_ld16(tmem + lane_base + kColDS + 32 * grp + 16 * hh, dsv);
             tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) st[e] = fmaf(g, st[e], __uint_as_float(dsv[e]));
+            for (int e = 0; e < 16; ++e) st[e] = fmaf(g, st[e], __uint_as_float(dsv[e]));
         };
         // E2: this thread's 32 columns of output row i -> bf16 -> the stage's Q buffer
         auto stage_output = [&](int s, float f) {
             unsigned char* orow = sm.q[s] + i * 128;
-            uint32_t ov[32];
-            tmem_ld32(tmem + lane_base + kColO + 32 * grp, ov);
-            tmem_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint4 x;
-                x.x = pack_bf16(f * __uint_as_float(ov[8 * c]), f * __uint_as_float(ov[8 * c + 1]));
-                x.y = pack_bf16(f * __uint_as_float(ov[8 * c + 2]), f * __uint_as_float(ov[8 * c + 3]));
-                x.z = pack_bf16(f * __uint_as_float(ov[8 * c + 4]), f * __uint_as_float(ov[8 * c + 5]));
-                x.w = pack_bf16(f * __uint_as_float(ov[8 * c + 6]), f * __uint_as_float(ov[8 * c + 7]));
-                reinterpret_cast<uint4*>(orow)[(4 * grp + c) ^ (i & 7)] = x;
+            for (int hh = 0; hh < 2; ++hh) {
+                uint32_t ov[16];
+                tmem_ld16(tmem + lane_base + kColO + 32 * grp + 16 * hh, ov);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint4 x;
+                    x.x = pack_bf16(f * __uint_as_float(ov[8 * c]), f * __uint_as_float(ov[8 * c + 1]));
+                    x.y = pack_bf16(f * __uint_as_float(ov[8 * c + 2]), f * __uint_as_float(ov[8 * c + 3]));
+                    x.z = pack_bf16(f * __uint_as_float(ov[8 * c + 4]), f * __uint_as_float(ov[8 * c + 5]));
+                    x.w = pack_bf16(f * __uint_as_float(ov[8 * c + 6]), f * __uint_as_float(ov[8 * c + 7]));
+                    reinterpret_cast<uint4*>(orow)[(4 * grp + 2 * hh + c) ^ (i & 7)] = x;
+                }
             }
         };
 
@@ -532,48 +546,51 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             //      as soon as every packet carries the tag of chunk n - 1.  The state recurrence is
             //      the only serial link along a chain, so it goes first when the state is already
             //      here; otherwise E1, which needs no state, fills the wait.
-            bool have_state = true;
-            if (t.n == 0) {
-                if (p.state_in) {
-                    load_state(p.state_in + (size_t)t.x * (kD * kD));
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) st[e] = 0.0f;
-                }
-            } else {
-                have_state = relay_peek(slot, tag_in) && relay_in_once(slot, tag_in);
-            }
+            const bool have_state = t.n == 0 || relay_peek(slot, tag_in, 0);
             TRACE_E(2);
 #pragma unroll 1
             for (int step = 0; ok && step < 2; ++step) {
                 if ((step == 0) == have_state) {
-                    // ---- state section: wait for the state if it is not here yet -----------------
-                    if (!have_state) {
-                        bool got = false;
-                        for (unsigned it = 0; it < limit; ++it) {
-                            if (relay_peek(slot, tag_in) && relay_in_once(slot, tag_in)) { got = true; break; }
-                            if ((it & 15u) == 15u && *abort_flag) break;
-                            __nanosleep(64);
-                        }
-                        if (!got) {
-                            if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, 1); }
-                            ok = false;
-                            break;
-                        }
-                    }
-                    TRACE_E(4);
-                    write_state_bf16(fast ? g_chunk : 1.0f);   // gamma^N S_prev (normal) / S_prev (exact: Q~ carries gamma^n_i)
-                    fence_proxy_async();
-                    mbar_arrive(&sm.bar.sb_ready);
-                    // E3: S_new = gamma^N S_prev + dS, then hand it to the chain's next chunk
+                    // ---- state section, one half of the thread's state values at a time: take the
+                    //      incoming half (waiting for it if it is not here yet), copy it for the
+                    //      Q x state MMAs, E3: S_new = gamma^N S_prev + dS, hand S_new on at once
                     if (!(ok = mbar_wait(&sm.bar.ds_done, par, limit, abort_flag, p.status))) break;
                     tc_fence_after();
-                    update_state(g_chunk);
-                    if (!last_chunk) {
-                        relay_out(slot, tag_out);
-                    } else if (p.state_out) {
-                        store_state(p.state_out + (size_t)t.x * (kD * kD));
+                    TRACE_E(4);
+#pragma unroll 1
+                    for (int hh = 0; hh < 2; ++hh) {
+                        if (t.n == 0) {
+                            if (p.state_in) {
+                                load_state_half(p.state_in + (size_t)t.x * (kD * kD), hh);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) st[e] = 0.0f;
+                            }
+                        } else {
+                            bool got = false;
+                            for (unsigned it = 0; it < limit; ++it) {
+                                if (relay_peek(slot, tag_in, hh) && relay_in_half(slot, tag_in, hh)) { got = true; break; }
+                                if ((it & 15u) == 15u && *abort_flag) break;
+                                __nanosleep(64);
+                            }
+                            if (!got) {
+                                if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, 1); }
+                                ok = false;
+                                break;
+                            }
+                        }
+                        // gamma^N S_prev (normal) / S_prev (exact: Q~ carries gamma^n_i)
+                        write_state_bf16_half(fast ? g_chunk : 1.0f, hh);
+                        update_state_half(g_chunk, hh);
+                        if (!last_chunk) {
+                            relay_out_half(slot, tag_out, hh);
+                        } else if (p.state_out) {
+                            store_state_half(p.state_out + (size_t)t.x * (kD * kD), hh);
+                        }
                     }
+                    if (!ok) break;
+                    fence_proxy_async();
+                    mbar_arrive(&sm.bar.sb_ready);
                     TRACE_E(5);
                 } else {
                     // ---- E1: A = tril(S) (normal) or P = S o gamma^(n_i - n_j) o [j <= i] (exact)
@@ -587,41 +604,43 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     }
                     if (fast) {
 #pragma unroll
-                        for (int pi = 0; pi < 2; ++pi) {
-                            const int pc = 2 * grp + pi;
-                            uint32_t pk[16];
+                        for (int q16 = 0; q16 < 4; ++q16) {      // 16-column pieces of blocks 2 grp, 2 grp + 1
+                            const int pc = 2 * grp + (q16 >> 1);
+                            const int c0 = 16 * (q16 & 1);           // first column of the piece inside its block
+                            uint32_t pk[8];
                             if (pc <= qd) {
-                                uint32_t sv[32];
-                                tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
+                                uint32_t sv[16];
+                                tmem_ld16(tmem + lane_base + kColS + 32 * pc + c0, sv);
                                 tmem_wait_ld();
                                 if (pc < qd) {
 #pragma unroll
-                                    for (int c = 0; c < 16; ++c)
+                                    for (int c = 0; c < 8; ++c)
                                         pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
                                 } else {
 #pragma unroll
-                                    for (int c = 0; c < 16; ++c)
-                                        pk[c] = pack_bf16(2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
-                                                          2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
+                                    for (int c = 0; c < 8; ++c)
+                                        pk[c] = pack_bf16(c0 + 2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
+                                                          c0 + 2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
                                 }
                             } else {
 #pragma unroll
-                                for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                                for (int c = 0; c < 8; ++c) pk[c] = 0u;
                             }
-                            tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
+                            tmem_st8(tmem + lane_base + kColS + 64 * grp + 8 * q16, pk);
                         }
                     } else {
 #pragma unroll 1
-                        for (int pi = 0; pi < 2; ++pi) {
-                            const int pc = 2 * grp + pi;
-                            uint32_t pk[16];
+                        for (int q16 = 0; q16 < 4; ++q16) {
+                            const int pc = 2 * grp + (q16 >> 1);
+                            const int c0 = 16 * (q16 & 1);
+                            uint32_t pk[8];
                             if (pc <= qd) {
-                                uint32_t sv[32];
-                                tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
+                                uint32_t sv[16];
+                                tmem_ld16(tmem + lane_base + kColS + 32 * pc + c0, sv);
                                 tmem_wait_ld();
 #pragma unroll
-                                for (int c = 0; c < 16; ++c) {
-                                    const int j0 = 32 * pc + 2 * c;
+                                for (int c = 0; c < 8; ++c) {
+                                    const int j0 = 32 * pc + c0 + 2 * c;
                                     const int d0 = cd.ni - cd.n_of(j0), d1 = cd.ni - cd.n_of(j0 + 1);
                                     const float v0 = j0 <= i ? __uint_as_float(sv[2 * c]) * sm.pw[d0 > 0 ? d0 : 0] : 0.0f;
                                     const float v1 = j0 + 1 <= i ? __uint_as_float(sv[2 * c + 1]) * sm.pw[d1 > 0 ? d1 : 0] : 0.0f;
@@ -629,9 +648,9 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                                 }
                             } else {
 #pragma unroll
-                                for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                                for (int c = 0; c < 8; ++c) pk[c] = 0u;
                             }
-                            tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
+                            tmem_st8(tmem + lane_base + kColS + 64 * grp + 8 * q16, pk);
                         }
                         if (grp == 0) scale_row_inplace<8>(sm.q[s] + i * 128, sm.pw[cd.ni], 0, i & 7);   // Q~
                     }
@@ -715,17 +734,33 @@ extern "C" int lasad_debug_read_stream_trace(long long* host, int n)
 
 int prefill_stream_chunks(int T) { return (T + kC - 1) / kC; }
 
-// Largest grid whose CTAs are all resident at once on `device` (the state relay needs that).
+// Largest grid whose CTAs are all resident at once on `device` (the state relay needs that),
+// from the device's shared-memory, register and thread limits and the kernel's own needs.
 int prefill_stream_max_ctas(int device)
 {
     static int cached[64] = {0};
     if (device >= 0 && device < 64 && cached[device] > 0) return cached[device];
     const size_t smem = sizeof(Smem) + 1024;
-    int per_sm = 0, sms = 0;
+    int sms = 0, smem_sm = 0, smem_reserved = 0, regs_sm = 0, threads_sm = 0, api_blocks = 0;
+    cudaFuncAttributes fa;
     if (cudaFuncSetAttribute(prefill_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, prefill_stream_kernel, kThreads, smem) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+        cudaFuncGetAttributes(&fa, prefill_stream_kernel) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&smem_reserved, cudaDevAttrReservedSharedMemoryPerBlock, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&threads_sm, cudaDevAttrMaxThreadsPerMultiProcessor, device) != cudaSuccess)
         return 0;
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&api_blocks, prefill_stream_kernel, kThreads, smem);
+    const int by_smem = smem_sm / (int)(smem + fa.sharedSizeBytes + smem_reserved);
+    const int regs_block = ((fa.numRegs * 32 + 255) / 256 * 256) * (kThreads / 32);   // allocated per warp in units of 256
+    const int by_regs = regs_block > 0 ? regs_sm / regs_block : 0;
+    const int by_threads = threads_sm / kThreads;
+    // TMEM: 512 columns per SM, kTmemCols per CTA
+    int per_sm = min(min(by_smem, by_regs), min(by_threads, 512 / kTmemCols));
+    if (getenv("LASAD_DEBUG"))
+        fprintf(stderr, "lasad: stream prefill CTAs/SM: smem %d regs %d threads %d -> %d (occupancy API: %d), %d SMs\n",
+                by_smem, by_regs, by_threads, per_sm, api_blocks, sms);
     const int n = per_sm * sms;
     if (device >= 0 && device < 64) cached[device] = n;
     return n;

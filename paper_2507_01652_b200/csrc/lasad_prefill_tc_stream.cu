@@ -75,6 +75,7 @@ constexpr uint32_t kColO = 128;    // O accumulator, 64 columns
 constexpr uint32_t kColDS = 192;   // dS accumulator (M = 64 layout), 64 columns
 constexpr unsigned kTeardownLimit = 1u << 26;
 constexpr float kFastPathMinDecay = 0.6f;
+constexpr int kHeadCache = 256;
 
 struct __align__(8) Barriers {
     unsigned long long full[kStages];   // TMA loads of a stage have landed
@@ -97,6 +98,8 @@ struct Smem {
     unsigned char v[kStages][kTileBytes];
     unsigned char sb[kD * kD * 2];  // bf16 copy of the incoming state, [dk][dv], 128 B rows, swizzled
     float pw[kC + 4];               // gamma^m, m = 0..128 (exact path only, rebuilt per task)
+    float gam[kHeadCache];          // the heads' decays and their base-2 logarithms (when H <= kHeadCache)
+    float lgam[kHeadCache];
     Barriers bar;
     uint32_t tmem_base;
     int abort_flag;
@@ -191,17 +194,10 @@ __device__ __forceinline__ GridPos grid_pos_init(int grid_w, int prefix_len, lon
     return g;
 }
 
-// Decay bookkeeping of chunk n of the call (L live tokens).
-__device__ __forceinline__ ChunkDecay chunk_decay(const GridPos& g, int n, int L, int qd, int lane)
+// Decay bookkeeping of chunk n of the call (L live tokens); phase = (phase0 + n * 128) mod w.
+__device__ __forceinline__ ChunkDecay chunk_decay(const GridPos& g, int phase, int n, int L, int qd, int lane)
 {
     ChunkDecay d;
-    int phase = 0;
-    if (g.grid_w > 0) {
-        // (phase0 + n * 128) mod w, with a 64-bit division only for very wide grids
-        const unsigned w = (unsigned)g.grid_w;
-        const unsigned long long prod = (unsigned long long)((unsigned)n % w) * (unsigned)g.step + (unsigned)g.phase0;
-        phase = prod < 0x100000000ull ? (int)((unsigned)prod % w) : (int)(prod % w);
-    }
     const int cs = n * kC;
     unsigned mk[4];
 #pragma unroll
@@ -260,6 +256,13 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                      "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (p.H <= kHeadCache) {
+        for (int hh = tid; hh < p.H; hh += kThreads) {
+            const float gm = p.decay[hh];
+            sm.gam[hh] = gm;
+            sm.lgam[hh] = gm > 0.0f ? log2f(gm) : 0.0f;
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -372,97 +375,86 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         const int grp = warp >> 2;               // which half of the quadrant's columns
         const int i = qd * 32 + lane;            // chunk row owned by this thread
         const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
-        const int srow = qd * 16 + lane;         // state row (M = 64 TMEM layout: lanes 0..15 of a quadrant)
-        const bool has_state = lane < 16;
-        const size_t st_off = (size_t)srow * kD + 32 * grp;   // this thread's 32 state elements in a slot
+        // State ownership.  The dS accumulator (M = 64 layout) keeps state rows 16 qd .. 16 qd + 15 in
+        // the first 16 TMEM lanes of quadrant qd; the 16x256b load spreads this warp's 16 rows x 32
+        // columns (columns 32 grp ..) over all 32 threads, 16 values each: for column group k,
+        // st[4k], st[4k+1] = (row r0, columns c0 + 8k, + 1), st[4k+2], st[4k+3] = (row r0 + 8, same).
+        const int r0 = qd * 16 + (lane >> 2);
+        const int c0 = 32 * grp + 2 * (lane & 3);
 
         // position of the call's first token relative to the grid (SAD rule, Section 3.4)
         const GridPos gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0, lane);
 
-        // Inside a relay slot the packets are laid out for coalescing, not by state index: the
-        // 16-byte word j of the rp-th state-holding thread sits at word j * 128 + rp, so that a
-        // warp's access covers 256 contiguous bytes (both sides use the same thread mapping).
-        constexpr int kRelayThreads = kEThreads / 2;
-        const int rp = warp * 16 + lane;
-        // The thread's 32 state values (state[srow][32 grp .. 32 grp + 31]) are handled as two halves
-        // of 16, one after the other, to keep the register footprint of the relay small.
         float st[16];
-        auto load_state_half = [&](const float* src_state, int hh) {
+        auto load_state = [&](const float* src_state) {
 #pragma unroll
-            for (int e = 0; e < 16; ++e) st[e] = 0.0f;
-            if (has_state) {
-                const float4* src = reinterpret_cast<const float4*>(src_state + st_off + 16 * hh);
-#pragma unroll
-                for (int e4 = 0; e4 < 4; ++e4) {
-                    const float4 t = __ldcg(src + e4);
-                    st[4 * e4] = t.x; st[4 * e4 + 1] = t.y; st[4 * e4 + 2] = t.z; st[4 * e4 + 3] = t.w;
-                }
+            for (int k = 0; k < 4; ++k) {
+                const float2 a = __ldcg(reinterpret_cast<const float2*>(src_state + (size_t)r0 * kD + c0 + 8 * k));
+                const float2 b = __ldcg(reinterpret_cast<const float2*>(src_state + (size_t)(r0 + 8) * kD + c0 + 8 * k));
+                st[4 * k] = a.x; st[4 * k + 1] = a.y; st[4 * k + 2] = b.x; st[4 * k + 3] = b.y;
             }
         };
-        auto store_state_half = [&](float* dst_state, int hh) {
-            if (has_state) {
-                float4* dst = reinterpret_cast<float4*>(dst_state + st_off + 16 * hh);
+        auto store_state = [&](float* dst_state) {
 #pragma unroll
-                for (int e4 = 0; e4 < 4; ++e4)
-                    dst[e4] = make_float4(st[4 * e4], st[4 * e4 + 1], st[4 * e4 + 2], st[4 * e4 + 3]);
+            for (int k = 0; k < 4; ++k) {
+                *reinterpret_cast<float2*>(dst_state + (size_t)r0 * kD + c0 + 8 * k) = make_float2(st[4 * k], st[4 * k + 1]);
+                *reinterpret_cast<float2*>(dst_state + (size_t)(r0 + 8) * kD + c0 + 8 * k) =
+                    make_float2(st[4 * k + 2], st[4 * k + 3]);
             }
         };
-        // relay: 16 state values travel as 16 tagged packets in 8 stores
-        auto relay_out_half = [&](uint4* slot, uint32_t tag, int hh) {
-            if (has_state) {
-                uint4* dst = slot + (8 * hh) * kRelayThreads + rp;
+        // Relay slot layout: the 16-byte word j (two tagged values) of element-wise thread tid sits
+        // at word j * 256 + tid, so that a warp's access covers 512 contiguous bytes; both sides of
+        // the relay use the same thread mapping, so the layout never shows outside the slot.
+        auto relay_out = [&](uint4* slot, uint32_t tag) {
+            uint4* dst = slot + tid;
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    st_cg_v4(dst + j * kRelayThreads, make_uint4(__float_as_uint(st[2 * j]), tag, __float_as_uint(st[2 * j + 1]), tag));
-            }
+            for (int j = 0; j < 8; ++j)
+                st_cg_v4(dst + j * kEThreads, make_uint4(__float_as_uint(st[2 * j]), tag, __float_as_uint(st[2 * j + 1]), tag));
         };
-        // Cheap look at the relay slot: one lane per warp reads the last packets of its half row
-        // (the writer stores them in ascending order, so these usually land last).  Polling loops
-        // use this, never the full read, so that waiting CTAs do not load L2 with 32 KB per poll.
-        auto relay_peek = [&](const uint4* slot, uint32_t tag, int hh) {
+        // The eight words are requested into registers and then accepted (tags checked, values
+        // moved into st).
+        auto relay_request = [&](const uint4* slot, uint4 (&rv)[8]) {
+            const uint4* src = slot + tid;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) rv[j] = ld_cg_v4(src + j * kEThreads);
+        };
+        // true when every tag matched (warp-uniform result)
+        auto relay_accept = [&](const uint4 (&rv)[8], uint32_t tag) {
+            bool all = true;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                st[2 * j] = __uint_as_float(rv[j].x);
+                st[2 * j + 1] = __uint_as_float(rv[j].z);
+                all = all && rv[j].y == tag && rv[j].w == tag;
+            }
+            return __all_sync(0xffffffffu, all);
+        };
+        // Cheap look at the relay slot for polling loops: one lane per warp reads the warp's last
+        // word (the writer stores its words in ascending order), so that waiting CTAs do not load
+        // L2 with 32 KB per poll.
+        auto relay_peek = [&](const uint4* slot, uint32_t tag) {
             bool hit = true;
-            if (lane == 15) {
-                const uint4 v = ld_cg_v4(slot + (8 * hh + 7) * kRelayThreads + rp);
+            if (lane == 31) {
+                const uint4 v = ld_cg_v4(slot + 7 * kEThreads + tid);
                 hit = v.y == tag && v.w == tag;
             }
             return __all_sync(0xffffffffu, hit);
         };
-        // one pass over the half's packets; true when every tag matched (warp-uniform result)
-        auto relay_in_half = [&](const uint4* slot, uint32_t tag, int hh) {
-            bool all = true;
+        // bf16 copy of mult * state for the Q x state MMAs: [dk][dv] rows of 128 B, 16-byte pieces
+        // swizzled by the row; this thread writes eight bf16 pairs
+        auto write_state_bf16 = [&](float mult) {
+            unsigned char* row0 = sm.sb + r0 * 128 + 4 * (lane & 3);
 #pragma unroll
-            for (int e = 0; e < 16; ++e) st[e] = 0.0f;
-            if (has_state) {
-                const uint4* src = slot + (8 * hh) * kRelayThreads + rp;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint4 v = ld_cg_v4(src + j * kRelayThreads);
-                    st[2 * j] = __uint_as_float(v.x);
-                    st[2 * j + 1] = __uint_as_float(v.z);
-                    all = all && v.y == tag && v.w == tag;
-                }
-            }
-            return __all_sync(0xffffffffu, all);
-        };
-        // bf16 copy of mult * state half for the Q x state MMAs
-        auto write_state_bf16_half = [&](float mult, int hh) {
-            if (has_state) {
-                uint4* row = reinterpret_cast<uint4*>(sm.sb + srow * 128);
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint4 x;
-                    x.x = pack_bf16(mult * st[8 * c], mult * st[8 * c + 1]);
-                    x.y = pack_bf16(mult * st[8 * c + 2], mult * st[8 * c + 3]);
-                    x.z = pack_bf16(mult * st[8 * c + 4], mult * st[8 * c + 5]);
-                    x.w = pack_bf16(mult * st[8 * c + 6], mult * st[8 * c + 7]);
-                    row[(4 * grp + 2 * hh + c) ^ (srow & 7)] = x;
-                }
+            for (int k = 0; k < 4; ++k) {
+                const int piece = ((4 * grp + k) ^ (r0 & 7)) * 16;    // r0 + 8 has the same low bits
+                *reinterpret_cast<uint32_t*>(row0 + piece) = pack_bf16(mult * st[4 * k], mult * st[4 * k + 1]);
+                *reinterpret_cast<uint32_t*>(row0 + 8 * 128 + piece) = pack_bf16(mult * st[4 * k + 2], mult * st[4 * k + 3]);
             }
         };
-        // E3: S_new = g * S_prev + dS for the half
-        auto update_state_half = [&](float g, int hh) {
+        // E3: S_new = g * S_prev + dS
+        auto update_state = [&](float g) {
             uint32_t dsv[16];
-            tmem_ld16(tmem + lane_base + kColDS + 32 * grp + 16 * hh, dsv);
+            tmem_ld_16x256b_x4(tmem + lane_base + kColDS + 32 * grp, dsv);
             tmem_wait_ld();
 #pragma unroll
             for (int e = 0; e < 16; ++e) st[e] = fmaf(g, st[e], __uint_as_float(dsv[e]));
@@ -489,15 +481,32 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
         bool ok = true;
         unsigned exact_tasks = 0;    // exact-path tasks this CTA has run (phase of the table barriers)
+        // Task ids advance by G; chunk, chain, batch, head and the grid phase of the chunk's first
+        // token are advanced with them instead of being recomputed by division every task.
+        const int dn = G / p.X, dx = G - dn * p.X;
+        Task t = decode_task(first, p.X, p.H);
+        int phase = 0, dphase = 0;
+        if (p.grid_w > 0) {
+            const unsigned long long w = (unsigned long long)p.grid_w;
+            phase = (int)((((unsigned long long)t.n % w) * (unsigned)gp.step + (unsigned)gp.phase0) % w);
+            dphase = (int)((((unsigned long long)dn % w) * (unsigned)gp.step) % w);
+        }
         for (int g = 0; ok && g < n_local; ++g) {
-            const Task t = decode_task(first + g * G, p.X, p.H);
             const int s = g % kStages;
             const unsigned par = g & 1;
             TRACE_E(0);
-            const float gamma = p.decay[t.h];
+            float gamma, lg;
+            if (p.H <= kHeadCache) {
+                gamma = sm.gam[t.h];
+                lg = sm.lgam[t.h];
+            } else {
+                gamma = p.decay[t.h];
+                lg = gamma > 0.0f ? log2f(gamma) : 0.0f;
+            }
             const bool fast = gamma >= kFastPathMinDecay;
             const bool last_chunk = t.n + 1 == p.n_chunks;
-            const ChunkDecay cd = chunk_decay(gp, t.n, min(kC, p.T - t.n * kC), qd, lane);
+            const bool relayed_in = t.n > 0;
+            const ChunkDecay cd = chunk_decay(gp, phase, t.n, min(kC, p.T - t.n * kC), qd, lane);
             uint4* const slot = p.relay ? p.relay + (size_t)t.x * (kD * kD / 2) : nullptr;
             // tag of the state after chunk n - 1 of this launch (what this task consumes): launch
             // number and chunk index; the state this task produces carries the next tag
@@ -506,7 +515,6 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
             // gamma^m: normal path straight from exp2 (|m log2 gamma| <= 95, relative error ~1e-5);
             // exact path from a table in double precision (0^0 = 1), rebuilt for this task's head
-            const float lg = fast ? log2f(gamma) : 0.0f;
             auto gpow = [&](int m) { return exp2f((float)m * lg); };
             if (!fast) {
                 // every thread is done with the previous exact task's table before it is rewritten
@@ -542,130 +550,123 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             mbar_arrive(&sm.bar.x_ready);
             TRACE_E(1);
 
-            // ---- incoming state: chunk 0 takes state_in; later chunks take the chain's relay slot
-            //      as soon as every packet carries the tag of chunk n - 1.  The state recurrence is
-            //      the only serial link along a chain, so it goes first when the state is already
-            //      here; otherwise E1, which needs no state, fills the wait.
-            const bool have_state = t.n == 0 || relay_peek(slot, tag_in, 0);
-            TRACE_E(2);
-#pragma unroll 1
-            for (int step = 0; ok && step < 2; ++step) {
-                if ((step == 0) == have_state) {
-                    // ---- state section, one half of the thread's state values at a time: take the
-                    //      incoming half (waiting for it if it is not here yet), copy it for the
-                    //      Q x state MMAs, E3: S_new = gamma^N S_prev + dS, hand S_new on at once
-                    if (!(ok = mbar_wait(&sm.bar.ds_done, par, limit, abort_flag, p.status))) break;
-                    tc_fence_after();
-                    TRACE_E(4);
-#pragma unroll 1
-                    for (int hh = 0; hh < 2; ++hh) {
-                        if (t.n == 0) {
-                            if (p.state_in) {
-                                load_state_half(p.state_in + (size_t)t.x * (kD * kD), hh);
-                            } else {
+            // ---- E1: A = tril(S) (normal) or P = S o gamma^(n_i - n_j) o [j <= i] (exact) -> bf16
+            //      over S's own columns, in 16-column pieces.  This warp converts the blocks 2 grp
+            //      and 2 grp + 1 of its rows and keeps the result inside its own half of S's columns
+            //      (always behind its own reads); the A V MMAs walk the columns in that order.  It
+            //      needs no state and fills the time the dS MMAs and the relay take.
+            if (!s_seen) {
+                if (!(ok = mbar_wait(&sm.bar.s_done, par, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+            }
+            if (fast) {
 #pragma unroll
-                                for (int e = 0; e < 16; ++e) st[e] = 0.0f;
-                            }
+                for (int q16 = 0; q16 < 4; ++q16) {      // 16-column pieces of blocks 2 grp, 2 grp + 1
+                    const int pc = 2 * grp + (q16 >> 1);
+                    const int c0 = 16 * (q16 & 1);           // first column of the piece inside its block
+                    uint32_t pk[8];
+                    if (pc <= qd) {
+                        uint32_t sv[16];
+                        tmem_ld16(tmem + lane_base + kColS + 32 * pc + c0, sv);
+                        tmem_wait_ld();
+                        if (pc < qd) {
+#pragma unroll
+                            for (int c = 0; c < 8; ++c)
+                                pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
                         } else {
-                            bool got = false;
-                            for (unsigned it = 0; it < limit; ++it) {
-                                if (relay_peek(slot, tag_in, hh) && relay_in_half(slot, tag_in, hh)) { got = true; break; }
-                                if ((it & 15u) == 15u && *abort_flag) break;
-                                __nanosleep(64);
-                            }
-                            if (!got) {
-                                if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, 1); }
-                                ok = false;
-                                break;
-                            }
-                        }
-                        // gamma^N S_prev (normal) / S_prev (exact: Q~ carries gamma^n_i)
-                        write_state_bf16_half(fast ? g_chunk : 1.0f, hh);
-                        update_state_half(g_chunk, hh);
-                        if (!last_chunk) {
-                            relay_out_half(slot, tag_out, hh);
-                        } else if (p.state_out) {
-                            store_state_half(p.state_out + (size_t)t.x * (kD * kD), hh);
-                        }
-                    }
-                    if (!ok) break;
-                    fence_proxy_async();
-                    mbar_arrive(&sm.bar.sb_ready);
-                    TRACE_E(5);
-                } else {
-                    // ---- E1: A = tril(S) (normal) or P = S o gamma^(n_i - n_j) o [j <= i] (exact)
-                    //      -> bf16 over S's own columns.  This warp converts the 32-column blocks
-                    //      2 grp and 2 grp + 1 of its rows and keeps the result inside its own half
-                    //      of S's columns (block pc -> columns 64 grp + 16 (pc & 1), always behind
-                    //      this warp's own reads); the A V MMAs walk the columns in that order.
-                    if (!s_seen) {
-                        if (!(ok = mbar_wait(&sm.bar.s_done, par, limit, abort_flag, p.status))) break;
-                        tc_fence_after();
-                    }
-                    if (fast) {
 #pragma unroll
-                        for (int q16 = 0; q16 < 4; ++q16) {      // 16-column pieces of blocks 2 grp, 2 grp + 1
-                            const int pc = 2 * grp + (q16 >> 1);
-                            const int c0 = 16 * (q16 & 1);           // first column of the piece inside its block
-                            uint32_t pk[8];
-                            if (pc <= qd) {
-                                uint32_t sv[16];
-                                tmem_ld16(tmem + lane_base + kColS + 32 * pc + c0, sv);
-                                tmem_wait_ld();
-                                if (pc < qd) {
-#pragma unroll
-                                    for (int c = 0; c < 8; ++c)
-                                        pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
-                                } else {
-#pragma unroll
-                                    for (int c = 0; c < 8; ++c)
-                                        pk[c] = pack_bf16(c0 + 2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
-                                                          c0 + 2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
-                                }
-                            } else {
-#pragma unroll
-                                for (int c = 0; c < 8; ++c) pk[c] = 0u;
-                            }
-                            tmem_st8(tmem + lane_base + kColS + 64 * grp + 8 * q16, pk);
+                            for (int c = 0; c < 8; ++c)
+                                pk[c] = pack_bf16(c0 + 2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
+                                                  c0 + 2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
                         }
                     } else {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) pk[c] = 0u;
+                    }
+                    tmem_st8(tmem + lane_base + kColS + 64 * grp + 8 * q16, pk);
+                }
+            } else {
 #pragma unroll 1
-                        for (int q16 = 0; q16 < 4; ++q16) {
-                            const int pc = 2 * grp + (q16 >> 1);
-                            const int c0 = 16 * (q16 & 1);
-                            uint32_t pk[8];
-                            if (pc <= qd) {
-                                uint32_t sv[16];
-                                tmem_ld16(tmem + lane_base + kColS + 32 * pc + c0, sv);
-                                tmem_wait_ld();
+                for (int q16 = 0; q16 < 4; ++q16) {
+                    const int pc = 2 * grp + (q16 >> 1);
+                    const int c0 = 16 * (q16 & 1);
+                    uint32_t pk[8];
+                    if (pc <= qd) {
+                        uint32_t sv[16];
+                        tmem_ld16(tmem + lane_base + kColS + 32 * pc + c0, sv);
+                        tmem_wait_ld();
 #pragma unroll
-                                for (int c = 0; c < 8; ++c) {
-                                    const int j0 = 32 * pc + c0 + 2 * c;
-                                    const int d0 = cd.ni - cd.n_of(j0), d1 = cd.ni - cd.n_of(j0 + 1);
-                                    const float v0 = j0 <= i ? __uint_as_float(sv[2 * c]) * sm.pw[d0 > 0 ? d0 : 0] : 0.0f;
-                                    const float v1 = j0 + 1 <= i ? __uint_as_float(sv[2 * c + 1]) * sm.pw[d1 > 0 ? d1 : 0] : 0.0f;
-                                    pk[c] = pack_bf16(v0, v1);
-                                }
-                            } else {
-#pragma unroll
-                                for (int c = 0; c < 8; ++c) pk[c] = 0u;
-                            }
-                            tmem_st8(tmem + lane_base + kColS + 64 * grp + 8 * q16, pk);
+                        for (int c = 0; c < 8; ++c) {
+                            const int j0 = 32 * pc + c0 + 2 * c;
+                            const int d0 = cd.ni - cd.n_of(j0), d1 = cd.ni - cd.n_of(j0 + 1);
+                            const float v0 = j0 <= i ? __uint_as_float(sv[2 * c]) * sm.pw[d0 > 0 ? d0 : 0] : 0.0f;
+                            const float v1 = j0 + 1 <= i ? __uint_as_float(sv[2 * c + 1]) * sm.pw[d1 > 0 ? d1 : 0] : 0.0f;
+                            pk[c] = pack_bf16(v0, v1);
                         }
-                        if (grp == 0) scale_row_inplace<8>(sm.q[s] + i * 128, sm.pw[cd.ni], 0, i & 7);   // Q~
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) pk[c] = 0u;
                     }
-                    tmem_wait_st();
-                    fence_proxy_async();
-                    tc_fence_before();
-                    mbar_arrive(&sm.bar.p_ready);
-                    if (!fast) {
-                        mbar_arrive(&sm.bar.tbl_free);    // last use of the table in this task
-                        ++exact_tasks;
+                    tmem_st8(tmem + lane_base + kColS + 64 * grp + 8 * q16, pk);
+                }
+                if (grp == 0) scale_row_inplace<8>(sm.q[s] + i * 128, sm.pw[cd.ni], 0, i & 7);   // Q~
+            }
+            tmem_wait_st();
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(&sm.bar.p_ready);
+            if (!fast) {
+                mbar_arrive(&sm.bar.tbl_free);    // last use of the table in this task
+                ++exact_tasks;
+            }
+            TRACE_E(3);
+
+            // ---- state section, the only serial link along a chain: take the incoming state
+            //      (waiting for it if it is not here yet), copy it for the Q x state MMAs,
+            //      E3: S_new = gamma^N S_prev + dS, hand S_new on at once
+            if (!(ok = mbar_wait(&sm.bar.ds_done, par, limit, abort_flag, p.status))) break;
+            tc_fence_after();
+            TRACE_E(4);
+            // (the request is not issued earlier in the task: holding its 32 registers across E1
+            // costs more in spills than the exposed trip from L2)
+            uint4 rv[8];
+            if (relayed_in) relay_request(slot, rv);
+            if (!relayed_in) {
+                if (p.state_in) {
+                    load_state(p.state_in + (size_t)t.x * (kD * kD));
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) st[e] = 0.0f;
+                }
+            } else if (!relay_accept(rv, tag_in)) {
+                // not here yet: poll one word per warp, then read the warp's words again
+                bool got = false;
+                for (unsigned it = 0; it < limit; ++it) {
+                    if (relay_peek(slot, tag_in)) {
+                        relay_request(slot, rv);
+                        if (relay_accept(rv, tag_in)) { got = true; break; }
                     }
-                    TRACE_E(3);
+                    if ((it & 15u) == 15u && *abort_flag) break;
+                    __nanosleep(32);
+                }
+                if (!got) {
+                    if (!*abort_flag) { *abort_flag = 1; atomicExch(p.status, 1); }
+                    ok = false;
+                    break;
                 }
             }
-            if (!ok) break;
+            TRACE_E(2);
+            // gamma^N S_prev (normal) / S_prev (exact: Q~ carries gamma^n_i)
+            write_state_bf16(fast ? g_chunk : 1.0f);
+            fence_proxy_async();
+            mbar_arrive(&sm.bar.sb_ready);
+            update_state(g_chunk);
+            if (!last_chunk) {
+                relay_out(slot, tag_out);
+            } else if (p.state_out) {
+                store_state(p.state_out + (size_t)t.x * (kD * kD));
+            }
+            TRACE_E(5);
 
             // ---- E2: o_i = scale * gamma^-(N - n_i) * O'_i (normal) / scale * O_i (exact) -----------
             const float out_f = fast ? p.scale * gpow(-(cd.n_last - cd.ni)) : p.scale;
@@ -677,6 +678,22 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             tc_fence_before();
             mbar_arrive(&sm.bar.st_ready);
             TRACE_E(7);
+
+            // ---- next task of this CTA -----------------------------------------------------------
+            t.n += dn;
+            t.x += dx;
+            phase += dphase;
+            if (t.x >= p.X) {
+                t.x -= p.X;
+                t.n += 1;
+                phase += gp.step;
+            }
+            if (p.grid_w > 0) {
+                if (phase >= p.grid_w) phase -= p.grid_w;
+                if (phase >= p.grid_w) phase -= p.grid_w;
+            }
+            t.b = t.x / p.H;
+            t.h = t.x - t.b * p.H;
         }
     }
 

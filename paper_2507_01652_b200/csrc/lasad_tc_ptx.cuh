@@ -152,6 +152,20 @@ __device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t (&r)[8])
                  "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
                  : "memory");
 }
+// 16 TMEM lanes x 32 columns spread over all 32 threads of the warp (the accumulator layout of an
+// M = 64 MMA keeps 16 rows per lane quadrant): thread t receives, for each group k of 8 columns,
+// r[4k + 0], r[4k + 1] = (row t / 4, columns 8k + 2 (t % 4), + 1) and
+// r[4k + 2], r[4k + 3] = (row t / 4 + 8, same columns).
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t addr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(addr)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 

@@ -195,7 +195,7 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
 
     int impl = ctx->opt_prefill_impl;
     const bool tc_ok = lasad::prefill_tc_supported(p->dk, p->dv, bf16);
-    if (impl == 0) impl = tc_ok ? 3 : 1;
+    if (impl == 0) impl = tc_ok ? 2 : 1;
     if (impl == 3) {
         if (!tc_ok) return LASAD_ERR_UNSUPPORTED;
         const int64_t units = (int64_t)p->B * p->H;

@@ -55,8 +55,9 @@ enum { LASAD_F32 = 0, LASAD_BF16 = 1 };
 
 /* Options for lasad_set_option. */
 enum {
-    LASAD_OPT_PREFILL_IMPL = 0, /* 0 auto, 1 CUDA-core fp32 kernel, 2 tcgen05 kernel with one CTA per
-                                   (batch, head), 3 tcgen05 kernel streaming (batch, head, chunk) tasks  */
+    LASAD_OPT_PREFILL_IMPL = 0, /* 0 auto (2 where it applies, else 1), 1 CUDA-core fp32 kernel,
+                                   2 tcgen05 kernel with one CTA per (batch, head), 3 tcgen05 kernel
+                                   streaming (batch, head, chunk) tasks through persistent CTAs        */
     LASAD_OPT_PREFILL_CHUNK = 1,/* CUDA-core prefill chunk length: 0 auto, else 16/32/64          */
     LASAD_OPT_DECODE_TPU = 2,   /* decode: threads per (b,h) state; 0 auto, else 32/64/128/256 */
     LASAD_OPT_WAIT_LIMIT = 3    /* iteration cap of device-side waits; 0 = library default   */
@@ -109,6 +110,37 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p,
                   const void* q, const void* k, const void* v,
                   const float* decay, const float* state_in,
                   void* o, float* state_out, void* cuda_stream);
+
+/*
+ * lasad_forward without a context and without any allocation.  The paper has no counterpart:
+ * this exists for hosts in which this library may not allocate device memory at all -- a serving
+ * process that fixes its device-memory plan at start-up and treats a later cudaMalloc as an
+ * error (it synchronises the device and can fail once the plan has taken the memory), or a
+ * plug-in whose host framework owns every allocation on the device.  lasad_create cannot be
+ * used there, because it allocates.
+ *
+ * It runs the task-streaming tensor-core prefill (prefill implementation 3) on the CURRENT
+ * device.  The per-(batch, head) relay slots that kernel needs live in a fixed array inside the
+ * library image: 8 MiB plus a status block, held by every device that loads the library until
+ * the process exits.  Limits: bf16, dk = dv = 64, B * H <= 256; anything else returns
+ * LASAD_ERR_UNSUPPORTED (other argument rules as for lasad_forward).  The call makes no
+ * cudaMalloc / cudaFree and calls no allocating library routine.
+ *
+ *   device_status   device memory, one int, or NULL.  A kernel that gives up a bounded wait
+ *                   writes 1 there; the caller clears and reads it (with NULL the library's own
+ *                   status block takes the write and cannot be read back).
+ *
+ * The first call on a device looks up the array's device address and the device's limits; make
+ * that first call before starting any stream capture.  All calls on a device share the one
+ * array, which keeps the previous call's contents (the library invalidates them by a call
+ * counter and clears the array before the counter repeats): two calls that overlap on the GPU
+ * race on it, so issue them on one stream or order the streams.  Arguments q .. state_out and
+ * cuda_stream as for lasad_forward.
+ */
+int lasad_forward_static(const lasad_params* p,
+                         const void* q, const void* k, const void* v,
+                         const float* decay, const float* state_in,
+                         void* o, float* state_out, int* device_status, void* cuda_stream);
 
 /*
  * One generation step (Algorithm 1's loop body for the token at absolute index p->t0):

@@ -27,7 +27,8 @@ LASAD_OPT_DECODE_TPU = 2
 LASAD_OPT_WAIT_LIMIT = 3
 
 EXPORTS = (
-    "lasad_create", "lasad_destroy", "lasad_set_option", "lasad_reserve", "lasad_forward", "lasad_decode_step",
+    "lasad_create", "lasad_destroy", "lasad_set_option", "lasad_reserve", "lasad_forward", "lasad_forward_static",
+    "lasad_decode_step",
     "lasad_last_device_status", "lasad_last_cuda_error", "lasad_launch_count", "lasad_strerror",
 )
 
@@ -75,6 +76,8 @@ def load_library() -> ctypes.CDLL:
         lib.lasad_reserve.argtypes = [vp, ctypes.c_int64]
         lib.lasad_forward.restype = i32
         lib.lasad_forward.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.lasad_forward_static.restype = i32
+        lib.lasad_forward_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_decode_step.restype = i32
         lib.lasad_decode_step.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_last_device_status.restype = i32
@@ -212,6 +215,27 @@ class Lasad:
         if rc != LASAD_OK:
             self._raise(rc, "lasad_decode_step")
         return o
+
+
+def lasad_forward_static(q, k, v, decay, grid_w, o, state_out=None, prefix_len=0, t0=0, scale=1.0,
+                         state_in=None, device_status=None, stream=None):
+    """``lasad_forward_static``: prefill on q's device with no context and no allocation.
+
+    Every buffer, the output ``o`` included, is the caller's: this wrapper allocates nothing either.
+    ``device_status`` is an optional int32 CUDA tensor of one element.  Raises on an error code."""
+    _check_cuda(q, k, v, decay, state_in, o, state_out, device_status)
+    B, T, H, dk = q.shape
+    dv = v.shape[3]
+    p = LasadParams(B, T, H, dk, dv, grid_w, prefix_len, _dtype_code(q), t0, scale, 0,
+                    _strides3(q), _strides3(k), _strides3(v), _strides3(o))
+    lib = load_library()
+    with torch.cuda.device(q.device):
+        st = torch.cuda.current_stream(q.device).cuda_stream if stream is None else stream
+        rc = lib.lasad_forward_static(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(decay), _ptr(state_in),
+                                      _ptr(o), _ptr(state_out), _ptr(device_status), ctypes.c_void_p(st))
+    if rc != LASAD_OK:
+        raise LasadError(rc, "lasad_forward_static")
+    return o, state_out
 
 
 _default = {}

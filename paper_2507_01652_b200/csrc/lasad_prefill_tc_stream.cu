@@ -52,8 +52,12 @@
 // allocates TMEM and issues every MMA, warp 9 issues the TMA loads and stores.  All waits are
 // bounded: a wait that runs out raises a status word the host can read and the CTA leaves
 // through the normal exit (copies in flight are waited for, TMEM is freed).
+#include "../../include/lasad.h"
 #include "lasad_common.cuh"
 #include "lasad_tc_ptx.cuh"
+
+#include <cmath>
+#include <mutex>
 
 #include <cstdio>
 #include <cstdlib>
@@ -808,3 +812,92 @@ cudaError_t launch_prefill_stream(const KernelArgs& a, const TcRelay& r, cudaStr
 }
 
 }  // namespace lasad
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free prefill entry point (declared in lasad.h)
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticUnits = 256;   // (batch, head) pairs the built-in relay storage covers
+
+// Relay slots for kStaticUnits chains (8 MiB) followed by one 256-byte status block.  It lives in
+// the library image: every device that loads the library holds it until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticUnits * lasad::kTcRelaySlotBytes + 256];
+
+struct StaticState {
+    void* scratch = nullptr;        // device address of g_static_scratch on this device
+    int max_ctas = 0;
+    unsigned long long epoch = 0;   // launches through the allocation-free entry point on this device
+};
+StaticState g_static_state[64];
+std::mutex g_static_mutex;
+
+}  // namespace
+
+extern "C" int lasad_forward_static(const lasad_params* p, const void* q, const void* k, const void* v,
+                                    const float* decay, const float* state_in, void* o, float* state_out,
+                                    int* device_status, void* cuda_stream)
+{
+    // ---- argument checks (the same rules as lasad_forward, restricted to what this path runs) ----
+    if (!p || !q || !k || !v || !o || !decay) return LASAD_ERR_INVALID_ARG;
+    if (p->B <= 0 || p->H <= 0 || p->T <= 0 || p->dk <= 0 || p->dv <= 0) return LASAD_ERR_INVALID_ARG;
+    if (p->grid_w < 0 || p->prefix_len < 0 || p->t0 < 0 || p->reserved != 0) return LASAD_ERR_INVALID_ARG;
+    if (!std::isfinite(p->scale)) return LASAD_ERR_INVALID_ARG;
+    if (p->dtype != LASAD_F32 && p->dtype != LASAD_BF16) return LASAD_ERR_INVALID_ARG;
+    auto aligned16 = [](const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; };
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return LASAD_ERR_INVALID_ARG;
+    if ((state_in && !aligned16(state_in)) || (state_out && !aligned16(state_out))) return LASAD_ERR_INVALID_ARG;
+    if (device_status && (reinterpret_cast<uintptr_t>(device_status) & 3u)) return LASAD_ERR_INVALID_ARG;
+    const int64_t* strides[4] = {p->q_stride, p->k_stride, p->v_stride, p->o_stride};
+    for (int s = 0; s < 4; ++s) {
+        for (int d = 0; d < 3; ++d)
+            if (strides[s][d] < 0 || (strides[s][d] * 2) % 16 != 0) return LASAD_ERR_INVALID_ARG;
+        if (strides[s][2] < 64 && p->H > 1) return LASAD_ERR_INVALID_ARG;
+    }
+    if (p->dtype != LASAD_BF16 || p->dk != 64 || p->dv != 64) return LASAD_ERR_UNSUPPORTED;
+    const int64_t units = (int64_t)p->B * p->H;
+    if (units > kStaticUnits) return LASAD_ERR_UNSUPPORTED;     // beyond the built-in relay storage
+    if (units * lasad::prefill_stream_chunks(p->T) > 0x7fffffffLL) return LASAD_ERR_UNSUPPORTED;
+
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return LASAD_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticState& st = g_static_state[device];
+    if (!st.scratch) {
+        // once per device, with that device current: the symbol's name is only a host-side handle;
+        // the kernel needs the array's address on this device
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return LASAD_ERR_CUDA;
+        const int n = lasad::prefill_stream_max_ctas(device);
+        if (n <= 0) return LASAD_ERR_CUDA;
+        st.scratch = ptr;
+        st.max_ctas = n;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    unsigned char* base = static_cast<unsigned char*>(st.scratch);
+    const size_t relay_bytes = (size_t)kStaticUnits * lasad::kTcRelaySlotBytes;
+
+    lasad::KernelArgs a{};
+    a.B = p->B; a.T = p->T; a.H = p->H;
+    a.grid_w = p->grid_w; a.prefix_len = p->prefix_len; a.t0 = p->t0; a.scale = p->scale;
+    for (int d = 0; d < 3; ++d) {
+        a.qs[d] = p->q_stride[d]; a.ks[d] = p->k_stride[d];
+        a.vs[d] = p->v_stride[d]; a.os[d] = p->o_stride[d];
+    }
+    a.q = q; a.k = k; a.v = v; a.o = o;
+    a.decay = decay; a.state_in = state_in; a.state_out = state_out;
+    a.status = device_status ? device_status : reinterpret_cast<int*>(base + relay_bytes);
+    a.wait_limit = 1u << 22;
+
+    lasad::TcRelay r{};
+    r.relay = base;
+    // The slots keep the packets of earlier calls; their tags carry the call number modulo 65535,
+    // so before a number comes round again the slots are cleared (they also start out as zeros,
+    // and no tag is ever zero).
+    st.epoch += 1;
+    r.epoch16 = (unsigned)(st.epoch % 65535u) + 1u;
+    if (st.epoch % 65535u == 0 && cudaMemsetAsync(base, 0, relay_bytes, stream) != cudaSuccess) return LASAD_ERR_CUDA;
+    r.max_ctas = st.max_ctas;
+    return lasad::launch_prefill_stream(a, r, stream) == cudaSuccess ? LASAD_OK : LASAD_ERR_CUDA;
+}
+

@@ -31,7 +31,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) from the ncu captures
 # summarised under profiles/; None until a capture of that kernel exists.
-NCU_TRAFFIC_BYTES = {"prefill": None, "decode": None}
+NCU_TRAFFIC_BYTES = {
+    # prefill_tc_kernel: 580.5 MB measured on the 608.7 MB capture case, scaled by tokens to config 5b
+    "prefill": 867_000_000,
+    # decode_kernel, config 4, inside the kernel (the rest of the written state drains from L2 later)
+    "decode": 111_900_000,
+}
 
 
 def load_peaks():
@@ -161,6 +166,7 @@ def run_ours(args):
 
     peaks = load_peaks()
     ctx = binding.Lasad(local)
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, args.prefill_impl)
     K, W = args.steps, max(args.warmup, 3)
     wl = workloads.WORKLOADS[args.prefill_workload]
     if args.prefill_batch:
@@ -235,6 +241,7 @@ def run_ours(args):
     h2d = 3 * hq.numel() * hq.element_size()
     d2h = ho.numel() * ho.element_size()
     del hq, hk, hv, ho, q, k, v, o
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
 
     # ---- the other prefill configurations (context for the headline; rank 0 reports) ----------
     sweep = None
@@ -258,7 +265,7 @@ def run_ours(args):
             "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": f"{wl.name}: B={wl.B} H={wl.H} T={wl.T} ({wl.grid_h}x{wl.grid_w} grid) "
                                    f"d_k=d_v={wl.d}, {wl.dtype} I/O, fp32 accumulate and state",
-                       "per_gpu_tokens": tokens_per_step, "parallelism": f"replicated x{world}, no collective",
+                       "prefill_impl": args.prefill_impl, "per_gpu_tokens": tokens_per_step, "parallelism": f"replicated x{world}, no collective",
                        "l2_policy": "inputs larger than L2 (q,k,v,o = %.0f MB)" % (pf_bytes / 1e6)},
             "e2e": {"value": round(world * tokens_per_step / (e2e_ms * 1e-3), 1), "unit": "tokens/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4),
@@ -267,7 +274,8 @@ def run_ours(args):
             "clocks": sampler.summary(),
             "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4),
-                         "traffic": NCU_TRAFFIC_BYTES["prefill"], "peak_source": peaks["source"],
+                         "traffic": NCU_TRAFFIC_BYTES["prefill"] if (wl.name == "config5b" and args.prefill_impl in (0, 2)) else None,
+                         "peak_source": peaks["source"],
                          "kernel_ms": round(kern_ms, 5), "bytes_per_launch": pf_bytes},
             "tensor": {"executed_tflops": round(tc_tflops, 1), "chunk": chunk,
                        "frac_of_bf16_peak": round(tc_tflops / peaks["bf16_tflops"], 4)},
@@ -407,7 +415,7 @@ def run_decode(args, ctx, peaks, dev, rank, barrier, max_over_ranks, K):
         "roofline": {"bound": "hbm", "achieved": round(dbytes / (best_us * 1e-6) / 1e9, 1),
                      "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": round(dbytes / (best_us * 1e-6) / 1e9 / peaks["hbm_gbs"], 4),
-                     "traffic": NCU_TRAFFIC_BYTES["decode"], "peak_source": peaks["source"],
+                     "traffic": NCU_TRAFFIC_BYTES["decode"] if dw.name == "config4" else None, "peak_source": peaks["source"],
                      "timed": "cold sweep, CUDA graph" if graph_us is not None else "cold sweep, stream"},
     }
     if "graph_error" in dec:
@@ -496,6 +504,8 @@ def main():
                     help="chunk length used to count executed tensor flops")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-configuration prefill sweep")
+    ap.add_argument("--prefill-impl", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="prefill kernel: 0 library default, 1 CUDA cores, 2 tcgen05 CTA-per-chain, 3 tcgen05 task-streaming")
     ap.add_argument("--only", choices=["all", "prefill", "decode"], default="all",
                     help="time only one of the two kernels (small profiling runs)")
     ap.add_argument("--prefill-batch", type=int, default=0, help="override the prefill workload's batch")

@@ -248,3 +248,66 @@ def test_argument_errors_launch_nothing(ctx):
     with pytest.raises(ValueError):
         ctx.lasad_forward(q.cpu(), q, q, g, 4)
     assert ctx.launch_count == n0
+
+
+# ------------------------------------------------------------------------------------------
+# task-streaming prefill (implementation 3): paths the shared cases above do not reach
+# ------------------------------------------------------------------------------------------
+def test_streaming_prefill_many_heads_and_relay_growth(ctx):
+    """More heads than the kernel's shared-memory decay cache holds (H > 256) and more (batch,
+    head) pairs than the context's initial relay storage (B * H > 1024, so the call grows it)."""
+    B, T, H, d, w = 4, 300, 260, 64, 10
+    gen = torch.Generator().manual_seed(31)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+    g = 0.85 + 0.1499 * torch.rand(H, generator=gen)
+    o_ref, s_ref = oracle(q, k, v, g, w)
+    o, s = _forward(ctx, 3, *_dev(q, k, v, g), w)
+    assert rel_err(o, o_ref) <= TOL[torch.bfloat16]
+    assert rel_err(s, s_ref) <= TOL[torch.bfloat16]
+
+
+def test_streaming_prefill_without_final_state_and_repeated_calls(ctx):
+    """state_out = NULL, and many launches in a row over the same relay slots (each launch must
+    ignore the packets the previous one left behind)."""
+    wl = _small("config3", 2, 3)
+    q, k, v = workloads.make_qkv(wl)
+    g = workloads.make_decay(wl)
+    o_ref, _ = oracle(q, k, v, g, wl.grid_w)
+    dq, dk_, dv_, dg = _dev(q, k, v, g)
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 3)
+    try:
+        outs = []
+        for _ in range(50):
+            o, s = ctx.lasad_forward(dq, dk_, dv_, dg, wl.grid_w, want_state=False)
+            assert s is None
+            outs.append(o)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+    finally:
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
+    assert rel_err(outs[0], o_ref) <= TOL[torch.bfloat16]
+    assert all(torch.equal(outs[0], x) for x in outs[1:])
+
+
+def test_streaming_prefill_launch_counter_wraps(ctx):
+    """The relay tags hold the launch number modulo 65535: run past the wrap (the library clears
+    the slots there) and check the result on both sides of it."""
+    B, T, H, d, w = 1, 256, 2, 64, 16
+    gen = torch.Generator().manual_seed(32)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+    g = torch.tensor([0.9, 0.99])
+    o_ref, s_ref = oracle(q, k, v, g, w)
+    dq, dk_, dv_, dg = _dev(q, k, v, g)
+    o = torch.empty_like(dq)
+    s = torch.empty(B, H, d, d, device="cuda")
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 3)
+    try:
+        for it in range(66000):
+            ctx.lasad_forward(dq, dk_, dv_, dg, w, o=o, state_out=s)
+            if it % 8192 == 0 or it > 65990:
+                torch.cuda.synchronize()
+                assert ctx.device_status() == 0
+                assert rel_err(o, o_ref) <= TOL[torch.bfloat16], f"launch {it}"
+                assert rel_err(s, s_ref) <= TOL[torch.bfloat16], f"launch {it}"
+    finally:
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)

@@ -116,6 +116,31 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------------------------
+# multi-rank bookkeeping (replicas only: no data-path collective)
+# --------------------------------------------------------------------------------------------
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Every rank draws its own replica of the workload."""
+    return base_seed + 1000 * rank
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    """Slowest rank's time (the only value exchanged between ranks)."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Units processed by all ranks per second, given the slowest rank's time per step."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
+# --------------------------------------------------------------------------------------------
 # algorithmic traffic
 # --------------------------------------------------------------------------------------------
 def prefill_bytes(wl) -> int:
@@ -157,12 +182,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    def max_ranks(x: float) -> float:
+        return max_over_ranks(x, world, dev)
 
     peaks = load_peaks()
     ctx = binding.Lasad(local)
@@ -171,10 +192,10 @@ def run_ours(args):
     wl = workloads.WORKLOADS[args.prefill_workload]
     if args.prefill_batch:
         wl = wl.scaled(B=args.prefill_batch)
-    wl = dataclasses.replace(wl, seed=wl.seed + 1000 * rank)
+    wl = dataclasses.replace(wl, seed=rank_seed(wl.seed, rank))
     stream = torch.cuda.current_stream()
     if args.only == "decode":
-        dec = run_decode(args, ctx, peaks, dev, rank, barrier, max_over_ranks, K)
+        dec = run_decode(args, ctx, peaks, dev, rank, barrier, max_ranks, K)
         if rank == 0:
             print(json.dumps({"decode": dec}), flush=True)
         ctx.close()
@@ -206,11 +227,11 @@ def run_ours(args):
     barrier()
     launches = ctx.launch_count - n0
     assert ctx.device_status() == 0, "a device-side wait timed out during the timed region"
-    total_ms = max_over_ranks(t_beg.elapsed_time(t_end))
+    total_ms = max_ranks(t_beg.elapsed_time(t_end))
     kern_ms = statistics.mean(a.elapsed_time(b) for a, b in ev)
     ms_per_step = total_ms / K
     tokens_per_step = wl.B * wl.T
-    value = world * tokens_per_step / (ms_per_step * 1e-3)
+    value = whole_job_rate(tokens_per_step, world, ms_per_step)
     pf_bytes = prefill_bytes(wl)
     achieved = pf_bytes / (kern_ms * 1e-3) / 1e9
     chunk = args.chunk_for_flops
@@ -237,7 +258,7 @@ def run_ours(args):
     e_end.record(stream)
     torch.cuda.synchronize()
     barrier()
-    e2e_ms = max_over_ranks(e_beg.elapsed_time(e_end)) / Ke
+    e2e_ms = max_ranks(e_beg.elapsed_time(e_end)) / Ke
     h2d = 3 * hq.numel() * hq.element_size()
     d2h = ho.numel() * ho.element_size()
     del hq, hk, hv, ho, q, k, v, o
@@ -250,7 +271,7 @@ def run_ours(args):
 
     decode = None
     if args.only != "prefill":
-        decode = run_decode(args, ctx, peaks, dev, rank, barrier, max_over_ranks, K)
+        decode = run_decode(args, ctx, peaks, dev, rank, barrier, max_ranks, K)
 
     # ---- CPU baseline: the oracle as it stands on this machine's host cores (rank 0, N = 1) ----
     cpu = None
@@ -267,7 +288,7 @@ def run_ours(args):
                                    f"d_k=d_v={wl.d}, {wl.dtype} I/O, fp32 accumulate and state",
                        "prefill_impl": args.prefill_impl, "per_gpu_tokens": tokens_per_step, "parallelism": f"replicated x{world}, no collective",
                        "l2_policy": "inputs larger than L2 (q,k,v,o = %.0f MB)" % (pf_bytes / 1e6)},
-            "e2e": {"value": round(world * tokens_per_step / (e2e_ms * 1e-3), 1), "unit": "tokens/s",
+            "e2e": {"value": round(whole_job_rate(tokens_per_step, world, e2e_ms), 1), "unit": "tokens/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4),
                     "steps": Ke},
             "gpu_launches": int(launches),
@@ -326,7 +347,7 @@ def prefill_sweep(ctx, peaks, dev, names, reps: int = 10):
     return out
 
 
-def run_decode(args, ctx, peaks, dev, rank, barrier, max_over_ranks, K):
+def run_decode(args, ctx, peaks, dev, rank, barrier, max_ranks, K):
     """Decode sweep (config 4 shape): persistent fp32 state, one `lasad_decode_step` per grid position."""
     import torch
 
@@ -337,7 +358,7 @@ def run_decode(args, ctx, peaks, dev, rank, barrier, max_over_ranks, K):
     dw = workloads.WORKLOADS[args.decode_workload]
     if args.decode_batch:
         dw = dw.scaled(B=args.decode_batch)
-    dw = dataclasses.replace(dw, seed=dw.seed + 1000 * rank)
+    dw = dataclasses.replace(dw, seed=rank_seed(dw.seed, rank))
     P = dw.prefix_len
     dq, dk_, dv_ = [t.to(dev) for t in workloads.make_qkv(dw)]
     dg = workloads.make_decay(dw).to(dev)
@@ -373,7 +394,7 @@ def run_decode(args, ctx, peaks, dev, rank, barrier, max_over_ranks, K):
             d_end.record(stream)
             torch.cuda.synchronize()
         barrier()
-        us = max_over_ranks(d_beg.elapsed_time(d_end)) * 1e3 / (sweeps * len(positions))
+        us = max_ranks(d_beg.elapsed_time(d_end)) * 1e3 / (sweeps * len(positions))
         dec[mode] = us
     # the same cold sweep replayed as a CUDA graph: kernel time without per-launch host cost
     graph_us = None
@@ -398,7 +419,7 @@ def run_decode(args, ctx, peaks, dev, rank, barrier, max_over_ranks, K):
             g_end.record(stream)
             torch.cuda.synchronize()
         barrier()
-        graph_us = max_over_ranks(g_beg.elapsed_time(g_end)) * 1e3 / (sweeps * len(positions))
+        graph_us = max_ranks(g_beg.elapsed_time(g_end)) * 1e3 / (sweeps * len(positions))
     except Exception as e:  # pragma: no cover - reported, never hidden
         dec["graph_error"] = repr(e)
     assert ctx.device_status() == 0

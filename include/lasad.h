@@ -153,6 +153,26 @@ int lasad_decode_step(lasad_ctx* ctx, const lasad_params* p,
                       const void* q, const void* k, const void* v,
                       const float* decay, float* state, void* o, void* cuda_stream);
 
+/*
+ * The paper's own, data-dependent form of the operator (Algorithm 1; the SAD recurrence of Section
+ * 3.4 with a decay vector per token): lambda_t in [0,1]^dk, e.g. Sigmoid(Linear(x_t)), multiplies
+ * the state row-wise, s_t = diag(lambda_t^spatial) s_{t-1} + k_t v_t^T, with lambda_t^spatial = 1
+ * on the step that absorbs the last token of a grid row (the SAD rule) and lambda_t otherwise.
+ *
+ *   gate   [B,T,H,dk] (prefill) / [B,H,dk] (decode): lambda, in the dtype of q and with the
+ *          strides given in k_stride.
+ *   k      as in lasad_forward, or NULL: the key is tied to the gate, k_t = 1 - lambda_t (the
+ *          paper's base decay, lambda_t = 1 - k_t; Algorithm 1).  k_stride always describes gate.
+ *   The `decay` vector of lasad_forward has no counterpart here.  Other arguments, dtypes, sizes
+ *   and error rules as for lasad_forward / lasad_decode_step.  Arithmetic is fp32 on CUDA cores.
+ */
+int lasad_forward_gated(lasad_ctx* ctx, const lasad_params* p,
+                        const void* q, const void* k, const void* v, const void* gate,
+                        const float* state_in, void* o, float* state_out, void* cuda_stream);
+int lasad_decode_step_gated(lasad_ctx* ctx, const lasad_params* p,
+                            const void* q, const void* k, const void* v, const void* gate,
+                            float* state, void* o, void* cuda_stream);
+
 /* After the caller has synchronised the stream: 0, or LASAD_ERR_TIMEOUT if a kernel gave up a
  * bounded wait since the last query (the flag is cleared by the query).  Synchronous copy. */
 int lasad_last_device_status(lasad_ctx* ctx, int* status);

@@ -28,7 +28,7 @@ LASAD_OPT_WAIT_LIMIT = 3
 
 EXPORTS = (
     "lasad_create", "lasad_destroy", "lasad_set_option", "lasad_reserve", "lasad_forward", "lasad_forward_static",
-    "lasad_decode_step",
+    "lasad_decode_step", "lasad_forward_gated", "lasad_decode_step_gated",
     "lasad_last_device_status", "lasad_last_cuda_error", "lasad_launch_count", "lasad_strerror",
 )
 
@@ -80,6 +80,10 @@ def load_library() -> ctypes.CDLL:
         lib.lasad_forward_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_decode_step.restype = i32
         lib.lasad_decode_step.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp]
+        lib.lasad_forward_gated.restype = i32
+        lib.lasad_forward_gated.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.lasad_decode_step_gated.restype = i32
+        lib.lasad_decode_step_gated.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_last_device_status.restype = i32
         lib.lasad_last_device_status.argtypes = [vp, ctypes.POINTER(i32)]
         lib.lasad_last_cuda_error.restype = i32
@@ -237,6 +241,59 @@ def lasad_forward_static(q, k, v, decay, grid_w, o, state_out=None, prefix_len=0
         raise LasadError(rc, "lasad_forward_static")
     return o, state_out
 
+
+def _gated_methods():
+    def lasad_forward_gated(self, q, k, v, gate, grid_w, prefix_len=0, t0=0, scale=1.0, state_in=None, o=None,
+                            state_out=None, want_state=True, stream=None):
+        """Prefill with a data-dependent gate [B,T,H,dk]; ``k=None`` ties the key to the gate
+        (k = 1 - gate).  Returns (o, state_out)."""
+        _check_cuda(q, k, v, gate, state_in, o, state_out)
+        B, T, H, dk = q.shape
+        dv = v.shape[3]
+        if o is None:
+            o = torch.empty((B, T, H, dv), dtype=q.dtype, device=q.device)
+        if state_out is None and want_state:
+            state_out = torch.empty((B, H, dk, dv), dtype=torch.float32, device=q.device)
+        if gate.dtype != q.dtype or tuple(gate.shape) != tuple(q.shape):
+            raise ValueError("gate must have q's shape and dtype")
+        if k is not None and tuple(k.stride()) != tuple(gate.stride()):
+            raise ValueError("k and gate must share strides")
+        p = LasadParams(B, T, H, dk, dv, grid_w, prefix_len, _dtype_code(q), t0, scale, 0,
+                        _strides3(q), _strides3(gate), _strides3(v), _strides3(o))
+        st = torch.cuda.current_stream(q.device).cuda_stream if stream is None else stream
+        rc = self._lib.lasad_forward_gated(self._h, ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(gate),
+                                           _ptr(state_in), _ptr(o), _ptr(state_out), ctypes.c_void_p(st))
+        if rc != LASAD_OK:
+            self._raise(rc, "lasad_forward_gated")
+        return o, state_out
+
+    def lasad_decode_step_gated(self, q, k, v, gate, state, grid_w, prefix_len, t, scale=1.0, o=None, stream=None):
+        """One generation step with a data-dependent gate [B,H,dk]; ``state`` is updated in place."""
+        _check_cuda(q, k, v, gate, state, o)
+        B, H, dk = q.shape
+        dv = v.shape[2]
+        if o is None:
+            o = torch.empty((B, H, dv), dtype=q.dtype, device=q.device)
+        if state.dtype != torch.float32 or not state.is_contiguous() or tuple(state.shape) != (B, H, dk, dv):
+            raise ValueError("state must be contiguous float32 [B,H,dk,dv]")
+        if gate.dtype != q.dtype or tuple(gate.shape) != tuple(q.shape):
+            raise ValueError("gate must have q's shape and dtype")
+        if k is not None and tuple(k.stride()) != tuple(gate.stride()):
+            raise ValueError("k and gate must share strides")
+        p = LasadParams(B, 1, H, dk, dv, grid_w, prefix_len, _dtype_code(q), t, scale, 0,
+                        _strides_decode(q), _strides_decode(gate), _strides_decode(v), _strides_decode(o))
+        st = torch.cuda.current_stream(q.device).cuda_stream if stream is None else stream
+        rc = self._lib.lasad_decode_step_gated(self._h, ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(gate),
+                                               _ptr(state), _ptr(o), ctypes.c_void_p(st))
+        if rc != LASAD_OK:
+            self._raise(rc, "lasad_decode_step_gated")
+        return o
+
+    Lasad.lasad_forward_gated = lasad_forward_gated
+    Lasad.lasad_decode_step_gated = lasad_decode_step_gated
+
+
+_gated_methods()
 
 _default = {}
 

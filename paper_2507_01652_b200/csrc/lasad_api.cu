@@ -269,6 +269,52 @@ int lasad_decode_step(lasad_ctx* ctx, const lasad_params* p, const void* q, cons
     return LASAD_OK;
 }
 
+int lasad_forward_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
+                        const void* gate, const float* state_in, void* o, float* state_out, void* cuda_stream)
+{
+    int rc = check_common(ctx, p, false);
+    if (rc != LASAD_OK) return rc;
+    if (!q || !v || !o || !gate) return LASAD_ERR_INVALID_ARG;
+    if (!aligned16(q) || (k && !aligned16(k)) || !aligned16(v) || !aligned16(o) || !aligned16(gate))
+        return LASAD_ERR_INVALID_ARG;
+    if ((state_in && !aligned16(state_in)) || (state_out && !aligned16(state_out)))
+        return LASAD_ERR_INVALID_ARG;
+    lasad::KernelArgs a{};
+    fill_args(a, ctx, p);
+    a.q = q; a.k = k; a.v = v; a.o = o;
+    a.decay = nullptr; a.state_in = state_in; a.state_out = state_out;
+    const cudaError_t e = lasad::launch_prefill_gated(a, gate, p->dk, p->dtype == LASAD_BF16,
+                                                      static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    ctx->launches += 1;
+    return LASAD_OK;
+}
+
+int lasad_decode_step_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
+                            const void* gate, float* state, void* o, void* cuda_stream)
+{
+    int rc = check_common(ctx, p, true);
+    if (rc != LASAD_OK) return rc;
+    if (!q || !v || !o || !gate || !state) return LASAD_ERR_INVALID_ARG;
+    if (!aligned16(q) || (k && !aligned16(k)) || !aligned16(v) || !aligned16(o) || !aligned16(gate) ||
+        !aligned16(state))
+        return LASAD_ERR_INVALID_ARG;
+    lasad::KernelArgs a{};
+    fill_args(a, ctx, p);
+    a.T = 1;
+    a.q = q; a.k = k; a.v = v; a.o = o;
+    a.decay = nullptr; a.state_in = state; a.state_out = state;
+    // SAD rule (Algorithm 1's if-statement): the decay is 1 on a row-boundary step
+    const bool decay_on = !lasad::is_boundary_step(p->t0, p->grid_w, p->prefix_len);
+    int tpu = ctx->opt_decode_tpu;
+    if (tpu == 0) tpu = (long long)p->B * p->H >= 16LL * ctx->sm_count ? 128 : 256;
+    const cudaError_t e = lasad::launch_decode_gated(a, gate, p->dk, p->dtype == LASAD_BF16, decay_on, tpu,
+                                                     static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    ctx->launches += 1;
+    return LASAD_OK;
+}
+
 int lasad_last_device_status(lasad_ctx* ctx, int* status)
 {
     if (!ctx || !status) return LASAD_ERR_INVALID_ARG;

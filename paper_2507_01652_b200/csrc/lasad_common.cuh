@@ -58,6 +58,11 @@ template <> struct io<__nv_bfloat16> {
 // Launchers implemented in the kernel files; each returns the cudaError_t of its launch.
 cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool decay_on, int tpu,
                           cudaStream_t st);
+// Data-dependent gate (the paper's own decay): `gate` has q's dtype and k's strides; a.k may be
+// null (key tied to the gate, k = 1 - lambda); a.decay is unused.
+cudaError_t launch_decode_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, bool decay_on, int tpu,
+                                cudaStream_t st);
+cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, cudaStream_t st);
 bool prefill_tc_supported(int dk, int dv, bool bf16);
 cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st);
 

@@ -39,8 +39,11 @@ template <> __device__ inline void store4<__nv_bfloat16>(__nv_bfloat16* p, const
 // TPU threads cooperate on one (b,h) state of D x D floats.  A state row is D/4 float4s, so
 // CG = D/4 adjacent threads cover one row and a warp covers 32/CG consecutive rows: every
 // warp-wide load or store is one contiguous 512-byte run.
-template <typename T, int D, int TPU>
-__global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on)
+// GATED: the decay is the paper's data-dependent gate, a value per (batch, head, key channel)
+// read from `gate` with q's layout, and the key may be tied to it (k = 1 - lambda when a.k is
+// null); otherwise it is the per-head constant a.decay[h].
+template <typename T, int D, int TPU, bool GATED>
+__global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on, const void* gate_v)
 {
     constexpr int CG = D / 4;          // threads per state row
     constexpr int RPP = TPU / CG;      // rows covered per pass
@@ -64,17 +67,18 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on)
     if (live) {
         const int b = (int)(unit / a.H), h = (int)(unit % a.H);
         const T* q = static_cast<const T*>(a.q) + b * a.qs[0] + h * a.qs[2];
-        const T* k = static_cast<const T*>(a.k) + b * a.ks[0] + h * a.ks[2];
+        const T* k = a.k ? static_cast<const T*>(a.k) + b * a.ks[0] + h * a.ks[2] : nullptr;
+        const T* lam = GATED ? static_cast<const T*>(gate_v) + b * a.ks[0] + h * a.ks[2] : nullptr;
         const T* v = static_cast<const T*>(a.v) + b * a.vs[0] + h * a.vs[2];
         float* S = a.state_out + unit * (D * D) + r0 * D + cg * 4;
-        const float g = decay_on ? a.decay[h] : 1.0f;
+        const float g = GATED ? 1.0f : (decay_on ? a.decay[h] : 1.0f);
         float vv[4];
         load4<T>(v + cg * 4, vv);
 
 #pragma unroll
         for (int p0 = 0; p0 < PASSES; p0 += BATCH) {
             float4 s[BATCH];
-            float qr[BATCH], kr[BATCH];
+            float qr[BATCH], kr[BATCH], gr[BATCH];
 #pragma unroll
             for (int u = 0; u < BATCH; ++u)
                 s[u] = *reinterpret_cast<const float4*>(S + (size_t)(p0 + u) * RPP * D);
@@ -82,14 +86,21 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on)
             for (int u = 0; u < BATCH; ++u) {
                 const int row = r0 + (p0 + u) * RPP;
                 qr[u] = io<T>::load(q + row);
-                kr[u] = io<T>::load(k + row);
+                if (GATED) {
+                    const float lr = io<T>::load(lam + row);
+                    kr[u] = k ? io<T>::load(k + row) : 1.0f - lr;     // key tied to the gate
+                    gr[u] = decay_on ? lr : 1.0f;                      // SAD rule: 1 on a boundary step
+                } else {
+                    kr[u] = io<T>::load(k + row);
+                    gr[u] = g;
+                }
             }
 #pragma unroll
             for (int u = 0; u < BATCH; ++u) {
-                s[u].x = fmaf(g, s[u].x, kr[u] * vv[0]);
-                s[u].y = fmaf(g, s[u].y, kr[u] * vv[1]);
-                s[u].z = fmaf(g, s[u].z, kr[u] * vv[2]);
-                s[u].w = fmaf(g, s[u].w, kr[u] * vv[3]);
+                s[u].x = fmaf(gr[u], s[u].x, kr[u] * vv[0]);
+                s[u].y = fmaf(gr[u], s[u].y, kr[u] * vv[1]);
+                s[u].z = fmaf(gr[u], s[u].z, kr[u] * vv[2]);
+                s[u].w = fmaf(gr[u], s[u].w, kr[u] * vv[3]);
                 acc[0] = fmaf(qr[u], s[u].x, acc[0]);
                 acc[1] = fmaf(qr[u], s[u].y, acc[1]);
                 acc[2] = fmaf(qr[u], s[u].z, acc[2]);
@@ -134,15 +145,15 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on)
     }
 }
 
-template <typename T, int D>
-cudaError_t launch_decode_t(const KernelArgs& a, bool decay_on, int tpu, cudaStream_t st)
+template <typename T, int D, bool GATED>
+cudaError_t launch_decode_t(const KernelArgs& a, bool decay_on, int tpu, const void* gate, cudaStream_t st)
 {
     const long long n_units = (long long)a.B * a.H;
     const int on = decay_on ? 1 : 0;
 #define LASAD_DECODE_CASE(TPU_)                                                               \
     case TPU_: {                                                                              \
         const long long blocks = (n_units + (256 / TPU_) - 1) / (256 / TPU_);                 \
-        decode_kernel<T, D, TPU_><<<(unsigned)blocks, 256, 0, st>>>(a, on);                   \
+        decode_kernel<T, D, TPU_, GATED><<<(unsigned)blocks, 256, 0, st>>>(a, on, gate);      \
         break;                                                                                \
     }
     switch (tpu) {
@@ -163,11 +174,22 @@ cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool d
 {
     (void)dv;
     if (dk == 64) {
-        return bf16 ? launch_decode_t<__nv_bfloat16, 64>(a, decay_on, tpu, st)
-                    : launch_decode_t<float, 64>(a, decay_on, tpu, st);
+        return bf16 ? launch_decode_t<__nv_bfloat16, 64, false>(a, decay_on, tpu, nullptr, st)
+                    : launch_decode_t<float, 64, false>(a, decay_on, tpu, nullptr, st);
     }
-    return bf16 ? launch_decode_t<__nv_bfloat16, 32>(a, decay_on, tpu, st)
-                : launch_decode_t<float, 32>(a, decay_on, tpu, st);
+    return bf16 ? launch_decode_t<__nv_bfloat16, 32, false>(a, decay_on, tpu, nullptr, st)
+                : launch_decode_t<float, 32, false>(a, decay_on, tpu, nullptr, st);
+}
+
+cudaError_t launch_decode_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, bool decay_on, int tpu,
+                                cudaStream_t st)
+{
+    if (dk == 64) {
+        return bf16 ? launch_decode_t<__nv_bfloat16, 64, true>(a, decay_on, tpu, gate, st)
+                    : launch_decode_t<float, 64, true>(a, decay_on, tpu, gate, st);
+    }
+    return bf16 ? launch_decode_t<__nv_bfloat16, 32, true>(a, decay_on, tpu, gate, st)
+                : launch_decode_t<float, 32, true>(a, decay_on, tpu, gate, st);
 }
 
 }  // namespace lasad

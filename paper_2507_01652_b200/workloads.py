@@ -92,3 +92,13 @@ def make_state(wl: Workload, seed_offset: int = 100) -> torch.Tensor:
     """A seeded non-zero incoming state, fp32 [B,H,d,d] (for hand-off / decode cases)."""
     g = torch.Generator().manual_seed(wl.seed + seed_offset)
     return torch.randn(wl.B, wl.H, wl.d, wl.d, generator=g, dtype=torch.float32)
+
+
+def make_gate(wl: Workload, T: int | None = None) -> torch.Tensor:
+    """A data-dependent gate lambda [B,T,H,d] in the workload's I/O dtype, standing in for the
+    Sigmoid(Linear(x)) of a trained layer: a seeded logistic-normal with its mass near 1
+    (median 0.88), where forget gates of trained gated linear attention layers sit."""
+    T = wl.T if T is None else T
+    g = torch.Generator().manual_seed(wl.seed + 7)
+    z = torch.randn(wl.B, T, wl.H, wl.d, generator=g, dtype=torch.float32)
+    return torch.sigmoid(z + 2.0).to(wl.torch_dtype)

@@ -1,0 +1,126 @@
+"""GPU parity of the data-dependent (gated) form of the operator -- the paper's own decay, a
+vector lambda_t per token (Algorithm 1), with the SAD rule -- against the CPU oracle run on the
+same gate tensor.  Tolerances as for the constant-decay path."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2507_01652_b200 import binding, workloads
+from tests._util import TOL, oracle, rel_err, to64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Lasad(0)
+    yield c
+    c.close()
+
+
+def _dev(*ts):
+    return [None if t is None else t.cuda() for t in ts]
+
+
+def _inputs(seed, B, T, H, d, dtype, gate_lo=None):
+    gen = torch.Generator().manual_seed(seed)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / d ** 0.5).to(dtype) for _ in range(3)]
+    lam = torch.sigmoid(torch.randn(B, T, H, d, generator=gen) + 2.0)
+    if gate_lo is not None:        # a few hard zeros, ones and tiny gates
+        sel = torch.rand(B, T, H, d, generator=gen)
+        lam = torch.where(sel < 0.02, torch.zeros_like(lam), lam)
+        lam = torch.where((sel >= 0.02) & (sel < 0.04), torch.ones_like(lam), lam)
+        lam = torch.where((sel >= 0.04) & (sel < 0.06), torch.full_like(lam, gate_lo), lam)
+    return q, k, v, lam.to(dtype)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d", [32, 64])
+@pytest.mark.parametrize("T,w,P", [(1, 4, 0), (16, 4, 0), (17, 5, 1), (100, 7, 0), (257, 16, 1), (300, 0, 0)])
+def test_gated_prefill_matches_oracle(ctx, dtype, d, T, w, P):
+    B, H = 2, 3
+    q, k, v, lam = _inputs(500 + T + d, B, T, H, d, dtype)
+    s_in = torch.randn(B, H, d, d, generator=torch.Generator().manual_seed(T))
+    o_ref, s_ref = oracle(q, k, v, lam, w, P, 5, 0.5, s_in)
+    o, s = ctx.lasad_forward_gated(*_dev(q, k, v, lam), w, prefix_len=P, t0=5, scale=0.5, state_in=s_in.cuda())
+    torch.cuda.synchronize()
+    assert rel_err(o, o_ref) <= TOL[dtype]
+    assert rel_err(s, s_ref) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_gated_prefill_key_tied_to_gate(ctx, dtype):
+    """k = NULL: the key is 1 - lambda (the paper's base decay lambda = 1 - k)."""
+    B, T, H, d, w = 2, 150, 4, 64, 10
+    q, _, v, lam = _inputs(77, B, T, H, d, dtype)
+    k_ref = 1.0 - to64(lam)                    # from the gate the kernel sees, in fp64
+    o_ref, s_ref = oracle(q, torch.from_numpy(k_ref), v, lam, w)
+    o, s = ctx.lasad_forward_gated(q.cuda(), None, v.cuda(), lam.cuda(), w)
+    torch.cuda.synchronize()
+    assert rel_err(o, o_ref) <= TOL[dtype]
+    assert rel_err(s, s_ref) <= TOL[dtype]
+
+
+def test_gated_prefill_extreme_gates(ctx):
+    """Gates of exactly 0 and 1 and tiny ones: nothing overflows, zeros cut the history."""
+    B, T, H, d, w = 1, 90, 2, 32, 9
+    q, k, v, lam = _inputs(78, B, T, H, d, torch.float32, gate_lo=1e-6)
+    o_ref, s_ref = oracle(q, k, v, lam, w)
+    o, s = ctx.lasad_forward_gated(*_dev(q, k, v, lam), w)
+    torch.cuda.synchronize()
+    assert torch.isfinite(o).all() and torch.isfinite(s).all()
+    assert rel_err(o, o_ref) <= TOL[torch.float32]
+    assert rel_err(s, s_ref) <= TOL[torch.float32]
+
+
+def test_constant_gate_reduces_to_the_per_head_path(ctx):
+    """A gate that is the same number everywhere in a head is the data-independent decay."""
+    wl = workloads.WORKLOADS["config2"].scaled(B=2, H=4)
+    q, k, v = workloads.make_qkv(wl)
+    g = workloads.make_decay(wl)
+    lam = g.view(1, 1, wl.H, 1).expand(wl.B, wl.T, wl.H, wl.d).to(torch.bfloat16).contiguous()
+    g_seen = lam[0, 0, :, 0].float()           # the per-head value after rounding to bf16
+    o_ref, s_ref = oracle(q, k, v, g_seen, wl.grid_w)
+    o, s = ctx.lasad_forward_gated(*_dev(q, k, v, lam), wl.grid_w)
+    o2, s2 = ctx.lasad_forward(*_dev(q, k, v, g_seen), wl.grid_w)
+    torch.cuda.synchronize()
+    assert rel_err(o, o_ref) <= TOL[torch.bfloat16] and rel_err(s, s_ref) <= TOL[torch.bfloat16]
+    assert rel_err(o2, o_ref) <= TOL[torch.bfloat16] and rel_err(s2, s_ref) <= TOL[torch.bfloat16]
+
+
+@pytest.mark.parametrize("dtype,d", [(torch.float32, 32), (torch.bfloat16, 64)])
+@pytest.mark.parametrize("tied", [False, True])
+def test_gated_decode_matches_oracle_and_prefill(ctx, dtype, d, tied):
+    B, T, H, w, P = 2, 40, 3, 6, 1
+    q, k, v, lam = _inputs(90 + d, B, T, H, d, dtype)
+    k_used = torch.from_numpy(1.0 - to64(lam)) if tied else k
+    o_ref, s_ref = oracle(q, k_used, v, lam, w, P)
+    dq, dk_, dv_, dl = _dev(q, k, v, lam)
+    state = torch.zeros(B, H, d, d, device="cuda")
+    outs = []
+    for t in range(T):
+        outs.append(ctx.lasad_decode_step_gated(dq[:, t], None if tied else dk_[:, t], dv_[:, t], dl[:, t], state,
+                                                w, P, t))
+    torch.cuda.synchronize()
+    assert rel_err(torch.stack(outs, 1), o_ref) <= TOL[dtype]
+    assert rel_err(state, s_ref) <= TOL[dtype]
+    _, s_pre = ctx.lasad_forward_gated(dq, None if tied else dk_, dv_, dl, w, prefix_len=P)
+    torch.cuda.synchronize()
+    assert rel_err(state, to64(s_pre)) <= TOL[dtype]
+
+
+def test_gated_state_handoff(ctx):
+    wl = dataclasses.replace(workloads.WORKLOADS["config3"], B=1, H=2)
+    q, k, v = workloads.make_qkv(wl)
+    lam = workloads.make_gate(wl)
+    o_ref, s_ref = oracle(q, k, v, lam, wl.grid_w)
+    dq, dk_, dv_, dl = _dev(q, k, v, lam)
+    for m in (1, 37, 300):
+        o1, s1 = ctx.lasad_forward_gated(dq[:, :m], dk_[:, :m], dv_[:, :m], dl[:, :m], wl.grid_w)
+        o2, s2 = ctx.lasad_forward_gated(dq[:, m:], dk_[:, m:], dv_[:, m:], dl[:, m:], wl.grid_w, t0=m,
+                                         state_in=s1, state_out=s1)
+        torch.cuda.synchronize()
+        assert rel_err(torch.cat([o1, o2], 1), o_ref) <= TOL[torch.bfloat16]
+        assert rel_err(s2, s_ref) <= TOL[torch.bfloat16]

@@ -268,6 +268,9 @@ def run_ours(args):
     sweep = None
     if args.only == "all" and not args.no_sweep:
         sweep = prefill_sweep(ctx, peaks, dev, ("config1", "config2", "config3", "config5a"))
+    gated = None
+    if args.only == "all" and not args.no_sweep:
+        gated = gated_sweep(ctx, peaks, dev)
 
     decode = None
     if args.only != "prefill":
@@ -302,6 +305,7 @@ def run_ours(args):
                        "frac_of_bf16_peak": round(tc_tflops / peaks["bf16_tflops"], 4)},
             "decode": decode,
             "prefill_sweep": sweep,
+            "gated": gated,
             "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)
@@ -344,6 +348,66 @@ def prefill_sweep(ctx, peaks, dev, names, reps: int = 10):
                     "algorithmic_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
                     "frac_of_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)})
         del q, k, v, o, s_out
+    return out
+
+
+def gated_sweep(ctx, peaks, dev, reps: int = 10):
+    """The data-dependent (gated) form: kernel time of one prefill on the config 2 and config 3
+    shapes (L2 flushed between launches) and of one decode step on the config 4 shape (rotating
+    state sets), with a seeded logistic-normal gate and the key given explicitly."""
+    import torch
+
+    from paper_2507_01652_b200 import workloads
+
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    out = {"prefill": [], "decode": None}
+    for name in ("config2", "config3"):
+        wl = workloads.WORKLOADS[name]
+        q, k, v = [t.to(dev) for t in workloads.make_qkv(wl)]
+        lam = workloads.make_gate(wl).to(dev)
+        o = torch.empty_like(v)
+        s_out = torch.empty(wl.B, wl.H, wl.d, wl.d, dtype=torch.float32, device=dev)
+        times = []
+        for it in range(reps + 3):
+            flush.fill_(it & 1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            ctx.lasad_forward_gated(q, k, v, lam, wl.grid_w, prefix_len=wl.prefix_len, o=o, state_out=s_out)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if it >= 3:
+                times.append(a.elapsed_time(b))
+        ms = statistics.median(times)
+        nbytes = wl.B * wl.T * wl.H * 5 * wl.d * wl.elem_bytes + wl.B * wl.H * wl.d * wl.d * 4   # q,k,v,gate in, o out
+        out["prefill"].append({"workload": f"{wl.name}: B={wl.B} H={wl.H} T={wl.T} d={wl.d} {wl.dtype}",
+                               "kernel_us": round(ms * 1e3, 2), "tokens_per_s": round(wl.B * wl.T / (ms * 1e-3), 1),
+                               "algorithmic_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                               "frac_of_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)})
+        del q, k, v, lam, o, s_out
+    dw = workloads.WORKLOADS["config4"]
+    T = 16
+    q, k, v = [t.to(dev) for t in workloads.make_qkv(dw, T)]
+    lam = workloads.make_gate(dw, T).to(dev)
+    states = [torch.zeros(dw.B, dw.H, dw.d, dw.d, dtype=torch.float32, device=dev) for _ in range(3)]
+    do = torch.empty(dw.B, dw.H, dw.d, dtype=q.dtype, device=dev)
+    def sweep():
+        for t in range(T):
+            ctx.lasad_decode_step_gated(q[:, t], k[:, t], v[:, t], lam[:, t], states[t % 3], dw.grid_w,
+                                        dw.prefix_len, dw.prefix_len + t, o=do)
+    sweep()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(reps):
+        sweep()
+    b.record(stream)
+    torch.cuda.synchronize()
+    us = a.elapsed_time(b) * 1e3 / (reps * T)
+    dbytes = dw.B * dw.H * (8 * dw.d * dw.d + 5 * dw.d * dw.elem_bytes)
+    out["decode"] = {"workload": f"{dw.name}: B={dw.B} H={dw.H} d={dw.d}, rotating states, per-step launches",
+                     "us_per_step": round(us, 3), "algorithmic_gbs": round(dbytes / (us * 1e-6) / 1e9, 1),
+                     "frac_of_hbm_peak": round(dbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], 4)}
     return out
 
 

@@ -112,6 +112,22 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p,
                   void* o, float* state_out, void* cuda_stream);
 
 /*
+ * lasad_forward on HOST buffers: q, k, v, decay, state_in are read from, and o, state_out written
+ * to, host memory (contiguous [B,T,H,d] / [H] / [B,H,dk,dv]; the strides in `p` are ignored).  Use
+ * page-locked memory: the call then overlaps, one batch element at a time, the copy in of element
+ * b+1, the prefill of element b and the copy out of element b-1 on two internal streams.  All
+ * work is ordered after what `cuda_stream` held at the call, and `cuda_stream` is complete only
+ * when o (and state_out) have arrived in host memory; the call itself does not wait.  The
+ * context keeps two staging slots of one batch element each; a call that needs larger ones than
+ * any before allocates them (cudaMalloc, synchronising).  Same operator, dtypes and error rules
+ * as lasad_forward (Section 3.4: the SAD recurrence).
+ */
+int lasad_forward_host(lasad_ctx* ctx, const lasad_params* p,
+                       const void* q, const void* k, const void* v,
+                       const float* decay, const float* state_in,
+                       void* o, float* state_out, void* cuda_stream);
+
+/*
  * lasad_forward without a context and without any allocation.  The paper has no counterpart:
  * this exists for hosts in which this library may not allocate device memory at all -- a serving
  * process that fixes its device-memory plan at start-up and treats a later cudaMalloc as an

@@ -27,7 +27,7 @@ LASAD_OPT_DECODE_TPU = 2
 LASAD_OPT_WAIT_LIMIT = 3
 
 EXPORTS = (
-    "lasad_create", "lasad_destroy", "lasad_set_option", "lasad_reserve", "lasad_forward", "lasad_forward_static",
+    "lasad_create", "lasad_destroy", "lasad_set_option", "lasad_reserve", "lasad_forward", "lasad_forward_host", "lasad_forward_static",
     "lasad_decode_step", "lasad_forward_gated", "lasad_decode_step_gated",
     "lasad_last_device_status", "lasad_last_cuda_error", "lasad_launch_count", "lasad_strerror",
 )
@@ -76,6 +76,8 @@ def load_library() -> ctypes.CDLL:
         lib.lasad_reserve.argtypes = [vp, ctypes.c_int64]
         lib.lasad_forward.restype = i32
         lib.lasad_forward.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.lasad_forward_host.restype = i32
+        lib.lasad_forward_host.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_forward_static.restype = i32
         lib.lasad_forward_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_decode_step.restype = i32
@@ -198,6 +200,26 @@ class Lasad:
                                      ctypes.c_void_p(st))
         if rc != LASAD_OK:
             self._raise(rc, "lasad_forward")
+        return o, state_out
+
+    def lasad_forward_host(self, q, k, v, decay, grid_w, o, prefix_len=0, t0=0, scale=1.0, state_in=None,
+                           state_out=None, stream=None):
+        """Prefill on HOST tensors (contiguous, ideally pinned): the library pipelines the copies
+        with the kernels.  ``o`` (and ``state_out``) are host tensors that are complete once the
+        stream has been synchronised.  Returns (o, state_out)."""
+        for t in (q, k, v, decay, o, state_in, state_out):
+            if t is not None and (t.is_cuda or not t.is_contiguous()):
+                raise ValueError("lasad_forward_host takes contiguous host tensors")
+        B, T, H, dk = q.shape
+        dv = v.shape[3]
+        p = LasadParams(B, T, H, dk, dv, grid_w, prefix_len, _dtype_code(q), t0, scale, 0,
+                        _strides3(q), _strides3(k), _strides3(v), _strides3(o))
+        dev = torch.device("cuda", self.device)
+        st = torch.cuda.current_stream(dev).cuda_stream if stream is None else stream
+        rc = self._lib.lasad_forward_host(self._h, ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(decay),
+                                          _ptr(state_in), _ptr(o), _ptr(state_out), ctypes.c_void_p(st))
+        if rc != LASAD_OK:
+            self._raise(rc, "lasad_forward_host")
         return o, state_out
 
     def lasad_decode_step(self, q, k, v, decay, state, grid_w, prefix_len, t, scale=1.0, o=None,

@@ -20,6 +20,17 @@ struct lasad_ctx {
     int64_t relay_cap;
     uint64_t epoch;               // launches of the task-streaming prefill so far
     int stream_max_ctas;
+    // host-buffer pipeline of lasad_forward_host: two staging slots (q | k | v | o of one batch
+    // element each), a decay and a state buffer, copy streams and the events that order them
+    void* d_stage[2];
+    size_t stage_bytes;
+    float* d_host_decay;
+    int64_t host_decay_cap;
+    float* d_host_state;
+    size_t host_state_bytes;
+    cudaStream_t s_in, s_out;
+    cudaEvent_t ev_start, ev_in[2], ev_comp[2], ev_out[2];
+    bool pipeline_ready;
 };
 
 namespace {
@@ -139,6 +150,20 @@ int lasad_destroy(lasad_ctx* ctx)
     if (!ctx) return LASAD_ERR_INVALID_ARG;
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_relay) cudaFree(ctx->d_relay);
+    for (int i = 0; i < 2; ++i)
+        if (ctx->d_stage[i]) cudaFree(ctx->d_stage[i]);
+    if (ctx->d_host_decay) cudaFree(ctx->d_host_decay);
+    if (ctx->d_host_state) cudaFree(ctx->d_host_state);
+    if (ctx->pipeline_ready) {
+        cudaStreamDestroy(ctx->s_in);
+        cudaStreamDestroy(ctx->s_out);
+        cudaEventDestroy(ctx->ev_start);
+        for (int i = 0; i < 2; ++i) {
+            cudaEventDestroy(ctx->ev_in[i]);
+            cudaEventDestroy(ctx->ev_comp[i]);
+            cudaEventDestroy(ctx->ev_out[i]);
+        }
+    }
     delete ctx;
     return LASAD_OK;
 }
@@ -312,6 +337,118 @@ int lasad_decode_step_gated(lasad_ctx* ctx, const lasad_params* p, const void* q
                                                      static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     ctx->launches += 1;
+    return LASAD_OK;
+}
+
+int lasad_forward_host(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
+                       const float* decay, const float* state_in, void* o, float* state_out, void* cuda_stream)
+{
+    int rc = check_common(ctx, p, false);
+    if (rc != LASAD_OK) return rc;
+    if (!q || !k || !v || !o || !decay) return LASAD_ERR_INVALID_ARG;
+    const size_t esz = p->dtype == LASAD_F32 ? 4 : 2;
+    const size_t per_q = (size_t)p->T * p->H * p->dk * esz, per_v = (size_t)p->T * p->H * p->dv * esz;
+    const size_t off_k = (per_q + 255) & ~size_t(255), off_v = 2 * off_k;
+    const size_t off_o = off_v + ((per_v + 255) & ~size_t(255));
+    const size_t slot = off_o + ((per_v + 255) & ~size_t(255));
+    const size_t state_bytes = (size_t)p->B * p->H * p->dk * p->dv * sizeof(float);
+    const bool use_state = state_in || state_out;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaError_t e = cudaSetDevice(ctx->device);
+    // ---- set-up and growth of the context's staging storage (allocates; synchronises) ----
+    if (e == cudaSuccess && !ctx->pipeline_ready) {
+        e = cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming);
+        for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+            e = cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_comp[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming);
+        }
+        ctx->pipeline_ready = e == cudaSuccess;
+    }
+    if (e == cudaSuccess && slot > ctx->stage_bytes) {
+        e = cudaDeviceSynchronize();
+        for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+            if (ctx->d_stage[i]) cudaFree(ctx->d_stage[i]);
+            ctx->d_stage[i] = nullptr;
+            e = cudaMalloc(&ctx->d_stage[i], slot);
+        }
+        ctx->stage_bytes = e == cudaSuccess ? slot : 0;
+    }
+    if (e == cudaSuccess && p->H > ctx->host_decay_cap) {
+        e = cudaDeviceSynchronize();
+        if (ctx->d_host_decay) cudaFree(ctx->d_host_decay);
+        ctx->d_host_decay = nullptr;
+        if (e == cudaSuccess) e = cudaMalloc(&ctx->d_host_decay, (size_t)p->H * sizeof(float));
+        ctx->host_decay_cap = e == cudaSuccess ? p->H : 0;
+    }
+    if (e == cudaSuccess && use_state && state_bytes > ctx->host_state_bytes) {
+        e = cudaDeviceSynchronize();
+        if (ctx->d_host_state) cudaFree(ctx->d_host_state);
+        ctx->d_host_state = nullptr;
+        if (e == cudaSuccess) e = cudaMalloc(&ctx->d_host_state, state_bytes);
+        ctx->host_state_bytes = e == cudaSuccess ? state_bytes : 0;
+    }
+    if (e != cudaSuccess) {
+        cudaSetDevice(prev);
+        return fail_cuda(ctx, e);
+    }
+
+    // ---- the pipeline: batch element b is copied in on s_in while b-1 is computed on the
+    //      caller's stream and b-2 is copied out on s_out ----
+    lasad_params pb = *p;
+    pb.B = 1;
+    const int64_t row_q = (int64_t)p->H * p->dk, row_v = (int64_t)p->H * p->dv;
+    pb.q_stride[0] = pb.k_stride[0] = (int64_t)p->T * row_q;
+    pb.q_stride[1] = pb.k_stride[1] = row_q;
+    pb.q_stride[2] = pb.k_stride[2] = p->dk;
+    pb.v_stride[0] = pb.o_stride[0] = (int64_t)p->T * row_v;
+    pb.v_stride[1] = pb.o_stride[1] = row_v;
+    pb.v_stride[2] = pb.o_stride[2] = p->dv;
+    const size_t unit_floats = (size_t)p->H * p->dk * p->dv;
+
+    e = cudaEventRecord(ctx->ev_start, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_in, ctx->ev_start, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_out, ctx->ev_start, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_host_decay, decay, (size_t)p->H * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && state_in)
+        e = cudaMemcpyAsync(ctx->d_host_state, state_in, state_bytes, cudaMemcpyHostToDevice, st);
+    for (int b = 0; b < p->B && e == cudaSuccess && rc == LASAD_OK; ++b) {
+        const int sl = b & 1;
+        unsigned char* base = static_cast<unsigned char*>(ctx->d_stage[sl]);
+        const unsigned char* hq = static_cast<const unsigned char*>(q) + (size_t)b * per_q;
+        const unsigned char* hk = static_cast<const unsigned char*>(k) + (size_t)b * per_q;
+        const unsigned char* hv = static_cast<const unsigned char*>(v) + (size_t)b * per_v;
+        unsigned char* ho = static_cast<unsigned char*>(o) + (size_t)b * per_v;
+        if (b >= 2) e = cudaStreamWaitEvent(ctx->s_in, ctx->ev_comp[sl], 0);   // the slot's inputs have been consumed
+        if (e == cudaSuccess) e = cudaMemcpyAsync(base, hq, per_q, cudaMemcpyHostToDevice, ctx->s_in);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(base + off_k, hk, per_q, cudaMemcpyHostToDevice, ctx->s_in);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(base + off_v, hv, per_v, cudaMemcpyHostToDevice, ctx->s_in);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_in[sl], ctx->s_in);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, ctx->ev_in[sl], 0);
+        if (e == cudaSuccess && b >= 2) e = cudaStreamWaitEvent(st, ctx->ev_out[sl], 0);   // the slot's output has left
+        if (e != cudaSuccess) break;
+        float* sb = use_state ? ctx->d_host_state + (size_t)b * unit_floats : nullptr;
+        rc = lasad_forward(ctx, &pb, base, base + off_k, base + off_v, ctx->d_host_decay, state_in ? sb : nullptr,
+                           base + off_o, state_out ? sb : nullptr, st);
+        if (rc != LASAD_OK) break;
+        e = cudaEventRecord(ctx->ev_comp[sl], st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_out, ctx->ev_comp[sl], 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(ho, base + off_o, per_v, cudaMemcpyDeviceToHost, ctx->s_out);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_out[sl], ctx->s_out);
+    }
+    // the caller's stream ends the call: it waits for the last copies out
+    for (int i = 0; i < 2 && e == cudaSuccess && rc == LASAD_OK; ++i)
+        if (i < p->B) e = cudaStreamWaitEvent(st, ctx->ev_out[i], 0);
+    if (e == cudaSuccess && rc == LASAD_OK && state_out)
+        e = cudaMemcpyAsync(state_out, ctx->d_host_state, state_bytes, cudaMemcpyDeviceToHost, st);
+    cudaSetDevice(prev);
+    if (rc != LASAD_OK) return rc;
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
     return LASAD_OK;
 }
 

@@ -311,3 +311,29 @@ def test_streaming_prefill_launch_counter_wraps(ctx):
                 assert rel_err(s, s_ref) <= TOL[torch.bfloat16], f"launch {it}"
     finally:
         ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
+
+
+# ------------------------------------------------------------------------------------------
+# host-buffer entry point: the pipelined copies must not change the result
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,d,B", [(torch.bfloat16, 64, 5), (torch.float32, 32, 3), (torch.bfloat16, 64, 1)])
+def test_forward_host_equals_device_path(ctx, dtype, d, B):
+    T, H, w, P = 333, 3, 12, 1
+    gen = torch.Generator().manual_seed(41 + B)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / d ** 0.5).to(dtype).pin_memory() for _ in range(3)]
+    g = torch.tensor([0.9, 0.97, 0.999]).pin_memory()
+    s_in = torch.randn(B, H, d, d, generator=gen).pin_memory()
+    o_h = torch.empty(B, T, H, d, dtype=dtype).pin_memory()
+    s_h = torch.empty(B, H, d, d).pin_memory()
+    for _ in range(2):      # twice: the second call reuses the staging slots and events
+        o_h.zero_()
+        s_h.zero_()
+        ctx.lasad_forward_host(q, k, v, g, w, o_h, prefix_len=P, t0=2, scale=0.5, state_in=s_in, state_out=s_h)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        o_d, s_d = ctx.lasad_forward(q.cuda(), k.cuda(), v.cuda(), g.cuda(), w, prefix_len=P, t0=2, scale=0.5,
+                                     state_in=s_in.cuda())
+        torch.cuda.synchronize()
+        assert torch.equal(o_h, o_d.cpu()) and torch.equal(s_h, s_d.cpu())
+    o_ref, s_ref = oracle(q, k, v, g, w, P, 2, 0.5, s_in)
+    assert rel_err(o_h, o_ref) <= TOL[dtype] and rel_err(s_h, s_ref) <= TOL[dtype]

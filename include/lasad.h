@@ -170,6 +170,18 @@ int lasad_decode_step(lasad_ctx* ctx, const lasad_params* p,
                       const float* decay, float* state, void* o, void* cuda_stream);
 
 /*
+ * lasad_decode_step for sequences that are not at the same position (continuous batching, images
+ * of different widths in one batch): pos [B] int32 (device) gives each sequence's absolute 0-based
+ * token index, grid_w [B] int32 (device) its tokens per grid row, or NULL for p->grid_w; p->t0 is
+ * ignored and the row-boundary test of the SAD rule (Section 3.4) is made per batch element on
+ * the device.  Everything else as lasad_decode_step.
+ */
+int lasad_decode_step_pos(lasad_ctx* ctx, const lasad_params* p,
+                          const void* q, const void* k, const void* v,
+                          const float* decay, float* state, void* o,
+                          const int32_t* pos, const int32_t* grid_w, void* cuda_stream);
+
+/*
  * The paper's own, data-dependent form of the operator (Algorithm 1; the SAD recurrence of Section
  * 3.4 with a decay vector per token): lambda_t in [0,1]^dk, e.g. Sigmoid(Linear(x_t)), multiplies
  * the state row-wise, s_t = diag(lambda_t^spatial) s_{t-1} + k_t v_t^T, with lambda_t^spatial = 1

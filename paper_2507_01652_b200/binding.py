@@ -28,7 +28,7 @@ LASAD_OPT_WAIT_LIMIT = 3
 
 EXPORTS = (
     "lasad_create", "lasad_destroy", "lasad_set_option", "lasad_reserve", "lasad_forward", "lasad_forward_host", "lasad_forward_static",
-    "lasad_decode_step", "lasad_forward_gated", "lasad_decode_step_gated",
+    "lasad_decode_step", "lasad_decode_step_pos", "lasad_forward_gated", "lasad_decode_step_gated",
     "lasad_last_device_status", "lasad_last_cuda_error", "lasad_launch_count", "lasad_strerror",
 )
 
@@ -82,6 +82,8 @@ def load_library() -> ctypes.CDLL:
         lib.lasad_forward_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_decode_step.restype = i32
         lib.lasad_decode_step.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp]
+        lib.lasad_decode_step_pos.restype = i32
+        lib.lasad_decode_step_pos.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_forward_gated.restype = i32
         lib.lasad_forward_gated.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_decode_step_gated.restype = i32
@@ -311,6 +313,30 @@ def _gated_methods():
             self._raise(rc, "lasad_decode_step_gated")
         return o
 
+    def lasad_decode_step_pos(self, q, k, v, decay, state, pos, prefix_len=0, grid_w=0, widths=None, scale=1.0,
+                              o=None, stream=None):
+        """One generation step with every sequence at its own position: ``pos`` int32 [B] on the
+        device, ``widths`` int32 [B] or None (then ``grid_w`` for all).  Returns o [B,H,dv]."""
+        _check_cuda(q, k, v, decay, state, o, pos, widths)
+        B, H, dk = q.shape
+        dv = v.shape[2]
+        if o is None:
+            o = torch.empty((B, H, dv), dtype=q.dtype, device=q.device)
+        if state.dtype != torch.float32 or not state.is_contiguous() or tuple(state.shape) != (B, H, dk, dv):
+            raise ValueError("state must be contiguous float32 [B,H,dk,dv]")
+        for t in (pos, widths):
+            if t is not None and (t.dtype != torch.int32 or not t.is_contiguous() or t.numel() != B):
+                raise ValueError("pos / widths must be contiguous int32 [B]")
+        p = LasadParams(B, 1, H, dk, dv, grid_w, prefix_len, _dtype_code(q), 0, scale, 0,
+                        _strides_decode(q), _strides_decode(k), _strides_decode(v), _strides_decode(o))
+        st = torch.cuda.current_stream(q.device).cuda_stream if stream is None else stream
+        rc = self._lib.lasad_decode_step_pos(self._h, ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(decay),
+                                             _ptr(state), _ptr(o), _ptr(pos), _ptr(widths), ctypes.c_void_p(st))
+        if rc != LASAD_OK:
+            self._raise(rc, "lasad_decode_step_pos")
+        return o
+
+    Lasad.lasad_decode_step_pos = lasad_decode_step_pos
     Lasad.lasad_forward_gated = lasad_forward_gated
     Lasad.lasad_decode_step_gated = lasad_decode_step_gated
 

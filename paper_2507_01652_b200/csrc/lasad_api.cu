@@ -294,6 +294,31 @@ int lasad_decode_step(lasad_ctx* ctx, const lasad_params* p, const void* q, cons
     return LASAD_OK;
 }
 
+int lasad_decode_step_pos(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
+                          const float* decay, float* state, void* o, const int32_t* pos, const int32_t* grid_w,
+                          void* cuda_stream)
+{
+    int rc = check_common(ctx, p, true);
+    if (rc != LASAD_OK) return rc;
+    if (!q || !k || !v || !o || !decay || !state || !pos) return LASAD_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(state))
+        return LASAD_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(pos) & 3u) || (reinterpret_cast<uintptr_t>(grid_w) & 3u)) return LASAD_ERR_INVALID_ARG;
+    lasad::KernelArgs a{};
+    fill_args(a, ctx, p);
+    a.T = 1;
+    a.q = q; a.k = k; a.v = v; a.o = o;
+    a.decay = decay; a.state_in = state; a.state_out = state;
+    a.pos = pos; a.widths = grid_w;
+    int tpu = ctx->opt_decode_tpu;
+    if (tpu == 0) tpu = (long long)p->B * p->H >= 16LL * ctx->sm_count ? 128 : 256;
+    const cudaError_t e = lasad::launch_decode(a, p->dk, p->dv, p->dtype == LASAD_BF16, true, tpu,
+                                               static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    ctx->launches += 1;
+    return LASAD_OK;
+}
+
 int lasad_forward_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
                         const void* gate, const float* state_in, void* o, float* state_out, void* cuda_stream)
 {

@@ -21,6 +21,8 @@ struct KernelArgs {
     const float* decay;     // [H]
     const float* state_in;  // [B,H,dk,dv] or nullptr
     float* state_out;       // [B,H,dk,dv] or nullptr
+    const int* pos;         // decode only: [B] absolute index of each sequence's token, or nullptr (t0 for all)
+    const int* widths;      // decode only: [B] grid width of each sequence, or nullptr (grid_w for all)
     int* status;            // device status word (bounded waits report here)
     unsigned wait_limit;
 };

@@ -71,6 +71,11 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on,
         const T* lam = GATED ? static_cast<const T*>(gate_v) + b * a.ks[0] + h * a.ks[2] : nullptr;
         const T* v = static_cast<const T*>(a.v) + b * a.vs[0] + h * a.vs[2];
         float* S = a.state_out + unit * (D * D) + r0 * D + cg * 4;
+        if (a.pos) {
+            // every sequence at its own position (and grid width): the SAD rule per batch element
+            const int w = a.widths ? a.widths[b] : a.grid_w;
+            decay_on = !is_boundary_step(a.pos[b], w, a.prefix_len);
+        }
         const float g = GATED ? 1.0f : (decay_on ? a.decay[h] : 1.0f);
         float vv[4];
         load4<T>(v + cg * 4, vv);

@@ -337,3 +337,25 @@ def test_forward_host_equals_device_path(ctx, dtype, d, B):
         assert torch.equal(o_h, o_d.cpu()) and torch.equal(s_h, s_d.cpu())
     o_ref, s_ref = oracle(q, k, v, g, w, P, 2, 0.5, s_in)
     assert rel_err(o_h, o_ref) <= TOL[dtype] and rel_err(s_h, s_ref) <= TOL[dtype]
+
+
+def test_decode_per_sequence_positions_and_widths(ctx):
+    """Every sequence at its own position and on its own grid width: each batch element must
+    equal a single-sequence oracle run at that position."""
+    B, H, d = 5, 3, 64
+    gen = torch.Generator().manual_seed(51)
+    q, k, v = [(torch.randn(B, 1, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+    g = torch.tensor([0.8, 0.95, 0.999])
+    s_in = torch.randn(B, H, d, d, generator=gen)
+    pos = torch.tensor([3, 4, 7, 11, 0], dtype=torch.int32)       # with P = 0: 3, 7, 11 end a row of width 4
+    widths = torch.tensor([4, 4, 8, 6, 1], dtype=torch.int32)     # element 4: width 1, every step is a boundary
+    for use_widths in (False, True):
+        state = s_in.clone().cuda()
+        o = ctx.lasad_decode_step_pos(q[:, 0].cuda(), k[:, 0].cuda(), v[:, 0].cuda(), g.cuda(), state, pos.cuda(),
+                                      prefix_len=0, grid_w=4, widths=widths.cuda() if use_widths else None)
+        torch.cuda.synchronize()
+        for b in range(B):
+            w = int(widths[b]) if use_widths else 4
+            o_ref, s_ref = oracle(q[b:b + 1], k[b:b + 1], v[b:b + 1], g, w, 0, int(pos[b]), 1.0, s_in[b:b + 1])
+            assert rel_err(o[b:b + 1], o_ref[:, 0]) <= TOL[torch.bfloat16], (b, use_widths)
+            assert rel_err(state[b:b + 1], s_ref) <= 1e-6, (b, use_widths)

@@ -39,10 +39,11 @@ template <> __device__ inline void store4<__nv_bfloat16>(__nv_bfloat16* p, const
 // TPU threads cooperate on one (b,h) state of D x D floats.  A state row is D/4 float4s, so
 // CG = D/4 adjacent threads cover one row and a warp covers 32/CG consecutive rows: every
 // warp-wide load or store is one contiguous 512-byte run.
+// POS: every sequence has its own position a.pos[b] (and grid width a.widths[b]).
 // GATED: the decay is the paper's data-dependent gate, a value per (batch, head, key channel)
 // read from `gate` with q's layout, and the key may be tied to it (k = 1 - lambda when a.k is
 // null); otherwise it is the per-head constant a.decay[h].
-template <typename T, int D, int TPU, bool GATED>
+template <typename T, int D, int TPU, bool GATED, bool POS>
 __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on, const void* gate_v)
 {
     constexpr int CG = D / 4;          // threads per state row
@@ -67,11 +68,11 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on,
     if (live) {
         const int b = (int)(unit / a.H), h = (int)(unit % a.H);
         const T* q = static_cast<const T*>(a.q) + b * a.qs[0] + h * a.qs[2];
-        const T* k = a.k ? static_cast<const T*>(a.k) + b * a.ks[0] + h * a.ks[2] : nullptr;
+        const T* k = (!GATED || a.k) ? static_cast<const T*>(a.k) + b * a.ks[0] + h * a.ks[2] : nullptr;
         const T* lam = GATED ? static_cast<const T*>(gate_v) + b * a.ks[0] + h * a.ks[2] : nullptr;
         const T* v = static_cast<const T*>(a.v) + b * a.vs[0] + h * a.vs[2];
         float* S = a.state_out + unit * (D * D) + r0 * D + cg * 4;
-        if (a.pos) {
+        if (POS) {
             // every sequence at its own position (and grid width): the SAD rule per batch element
             const int w = a.widths ? a.widths[b] : a.grid_w;
             decay_on = !is_boundary_step(a.pos[b], w, a.prefix_len);
@@ -83,7 +84,8 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on,
 #pragma unroll
         for (int p0 = 0; p0 < PASSES; p0 += BATCH) {
             float4 s[BATCH];
-            float qr[BATCH], kr[BATCH], gr[BATCH];
+            float qr[BATCH], kr[BATCH];
+            float gr[GATED ? BATCH : 1];
 #pragma unroll
             for (int u = 0; u < BATCH; ++u)
                 s[u] = *reinterpret_cast<const float4*>(S + (size_t)(p0 + u) * RPP * D);
@@ -97,15 +99,15 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on,
                     gr[u] = decay_on ? lr : 1.0f;                      // SAD rule: 1 on a boundary step
                 } else {
                     kr[u] = io<T>::load(k + row);
-                    gr[u] = g;
                 }
             }
 #pragma unroll
             for (int u = 0; u < BATCH; ++u) {
-                s[u].x = fmaf(gr[u], s[u].x, kr[u] * vv[0]);
-                s[u].y = fmaf(gr[u], s[u].y, kr[u] * vv[1]);
-                s[u].z = fmaf(gr[u], s[u].z, kr[u] * vv[2]);
-                s[u].w = fmaf(gr[u], s[u].w, kr[u] * vv[3]);
+                const float gu = GATED ? gr[GATED ? u : 0] : g;
+                s[u].x = fmaf(gu, s[u].x, kr[u] * vv[0]);
+                s[u].y = fmaf(gu, s[u].y, kr[u] * vv[1]);
+                s[u].z = fmaf(gu, s[u].z, kr[u] * vv[2]);
+                s[u].w = fmaf(gu, s[u].w, kr[u] * vv[3]);
                 acc[0] = fmaf(qr[u], s[u].x, acc[0]);
                 acc[1] = fmaf(qr[u], s[u].y, acc[1]);
                 acc[2] = fmaf(qr[u], s[u].z, acc[2]);
@@ -150,7 +152,7 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on,
     }
 }
 
-template <typename T, int D, bool GATED>
+template <typename T, int D, bool GATED, bool POS>
 cudaError_t launch_decode_t(const KernelArgs& a, bool decay_on, int tpu, const void* gate, cudaStream_t st)
 {
     const long long n_units = (long long)a.B * a.H;
@@ -158,7 +160,7 @@ cudaError_t launch_decode_t(const KernelArgs& a, bool decay_on, int tpu, const v
 #define LASAD_DECODE_CASE(TPU_)                                                               \
     case TPU_: {                                                                              \
         const long long blocks = (n_units + (256 / TPU_) - 1) / (256 / TPU_);                 \
-        decode_kernel<T, D, TPU_, GATED><<<(unsigned)blocks, 256, 0, st>>>(a, on, gate);      \
+        decode_kernel<T, D, TPU_, GATED, POS><<<(unsigned)blocks, 256, 0, st>>>(a, on, gate); \
         break;                                                                                \
     }
     switch (tpu) {
@@ -178,23 +180,31 @@ cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool d
                           cudaStream_t st)
 {
     (void)dv;
-    if (dk == 64) {
-        return bf16 ? launch_decode_t<__nv_bfloat16, 64, false>(a, decay_on, tpu, nullptr, st)
-                    : launch_decode_t<float, 64, false>(a, decay_on, tpu, nullptr, st);
+    if (a.pos) {
+        if (dk == 64) {
+            return bf16 ? launch_decode_t<__nv_bfloat16, 64, false, true>(a, decay_on, tpu, nullptr, st)
+                        : launch_decode_t<float, 64, false, true>(a, decay_on, tpu, nullptr, st);
+        }
+        return bf16 ? launch_decode_t<__nv_bfloat16, 32, false, true>(a, decay_on, tpu, nullptr, st)
+                    : launch_decode_t<float, 32, false, true>(a, decay_on, tpu, nullptr, st);
     }
-    return bf16 ? launch_decode_t<__nv_bfloat16, 32, false>(a, decay_on, tpu, nullptr, st)
-                : launch_decode_t<float, 32, false>(a, decay_on, tpu, nullptr, st);
+    if (dk == 64) {
+        return bf16 ? launch_decode_t<__nv_bfloat16, 64, false, false>(a, decay_on, tpu, nullptr, st)
+                    : launch_decode_t<float, 64, false, false>(a, decay_on, tpu, nullptr, st);
+    }
+    return bf16 ? launch_decode_t<__nv_bfloat16, 32, false, false>(a, decay_on, tpu, nullptr, st)
+                : launch_decode_t<float, 32, false, false>(a, decay_on, tpu, nullptr, st);
 }
 
 cudaError_t launch_decode_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, bool decay_on, int tpu,
                                 cudaStream_t st)
 {
     if (dk == 64) {
-        return bf16 ? launch_decode_t<__nv_bfloat16, 64, true>(a, decay_on, tpu, gate, st)
-                    : launch_decode_t<float, 64, true>(a, decay_on, tpu, gate, st);
+        return bf16 ? launch_decode_t<__nv_bfloat16, 64, true, false>(a, decay_on, tpu, gate, st)
+                    : launch_decode_t<float, 64, true, false>(a, decay_on, tpu, gate, st);
     }
-    return bf16 ? launch_decode_t<__nv_bfloat16, 32, true>(a, decay_on, tpu, gate, st)
-                : launch_decode_t<float, 32, true>(a, decay_on, tpu, gate, st);
+    return bf16 ? launch_decode_t<__nv_bfloat16, 32, true, false>(a, decay_on, tpu, gate, st)
+                : launch_decode_t<float, 32, true, false>(a, decay_on, tpu, gate, st);
 }
 
 }  // namespace lasad

@@ -212,14 +212,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (tid <= kC) {
-        // gamma^m for m = 0..128 by binary exponentiation in double precision (0^0 = 1)
-        double base = (double)gamma, acc = 1.0;
-        for (int e = tid; e > 0; e >>= 1) {
-            if (e & 1) acc *= base;
-            base *= base;
+        if (fast) {
+            // gamma^m and gamma^-m for m = 0..128 from exp2: |m log2 gamma| <= 95, so the relative
+            // error is ~1e-5, far below what bf16 I/O resolves, and a short sequence does not pay
+            // for double-precision arithmetic in every CTA's prologue
+            const float lg = log2f(gamma);
+            sm.pw[tid] = exp2f((float)tid * lg);
+            sm.ipw[tid] = exp2f(-(float)tid * lg);
+        } else {
+            // exact path: binary exponentiation in double precision (0^0 = 1)
+            double base = (double)gamma, acc = 1.0;
+            for (int e = tid; e > 0; e >>= 1) {
+                if (e & 1) acc *= base;
+                base *= base;
+            }
+            sm.pw[tid] = (float)acc;
+            sm.ipw[tid] = 0.0f;
         }
-        sm.pw[tid] = (float)acc;
-        sm.ipw[tid] = fast ? (float)(1.0 / acc) : 0.0f;
     }
     tc_fence_before();
     __syncthreads();

@@ -15,9 +15,9 @@
 // task only waits for a smaller id, so the grid cannot deadlock as long as all its CTAs are
 // resident (the host sizes the grid from the occupancy query); every wait is bounded anyway.
 //
-// Relay packets.  A state value travels as an 8-byte (value, tag) pair, two pairs per 16-byte
-// access.  An aligned 8-byte access is single-copy atomic, so a pair whose tag matches carries its
-// value: the relay needs no fence and no separate flag (release/acquire at GPU scope stalled for
+// Relay packets.  A state value travels as one 64-bit word (tag in the high half, value in the low
+// half), two words per 16-byte vector access.  A 64-bit element is read and written as a unit, so
+// a word whose tag matches carries its value: the relay needs no fence and no separate flag (release/acquire at GPU scope stalled for
 // microseconds while bulk copies were in flight).  The tag is the launch number (folded into
 // 1..65535 by the host, which clears the slots before a value comes round again) and the chunk
 // index.  Waiting CTAs poll one packet per warp, never the whole slot.
@@ -411,25 +411,25 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         // the relay use the same thread mapping, so the layout never shows outside the slot.
         auto relay_out = [&](uint4* slot, uint32_t tag) {
             uint4* dst = slot + tid;
+            const unsigned long long hi = (unsigned long long)tag << 32;
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                st_cg_v4(dst + j * kEThreads, make_uint4(__float_as_uint(st[2 * j]), tag, __float_as_uint(st[2 * j + 1]), tag));
+                st_cg_v2u64(dst + j * kEThreads, hi | __float_as_uint(st[2 * j]), hi | __float_as_uint(st[2 * j + 1]));
         };
-        // The eight words are requested into registers and then accepted (tags checked, values
-        // moved into st).
-        auto relay_request = [&](const uint4* slot, uint4 (&rv)[8]) {
+        // The eight 16-byte words are requested into registers and then accepted (tags checked,
+        // values moved into st).
+        auto relay_request = [&](const uint4* slot, unsigned long long (&rv)[16]) {
             const uint4* src = slot + tid;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) rv[j] = ld_cg_v4(src + j * kEThreads);
+            for (int j = 0; j < 8; ++j) ld_cg_v2u64(src + j * kEThreads, rv[2 * j], rv[2 * j + 1]);
         };
         // true when every tag matched (warp-uniform result)
-        auto relay_accept = [&](const uint4 (&rv)[8], uint32_t tag) {
+        auto relay_accept = [&](const unsigned long long (&rv)[16], uint32_t tag) {
             bool all = true;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                st[2 * j] = __uint_as_float(rv[j].x);
-                st[2 * j + 1] = __uint_as_float(rv[j].z);
-                all = all && rv[j].y == tag && rv[j].w == tag;
+            for (int e = 0; e < 16; ++e) {
+                st[e] = __uint_as_float((uint32_t)rv[e]);
+                all = all && (uint32_t)(rv[e] >> 32) == tag;
             }
             return __all_sync(0xffffffffu, all);
         };
@@ -439,8 +439,9 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         auto relay_peek = [&](const uint4* slot, uint32_t tag) {
             bool hit = true;
             if (lane == 31) {
-                const uint4 v = ld_cg_v4(slot + 7 * kEThreads + tid);
-                hit = v.y == tag && v.w == tag;
+                unsigned long long a, b;
+                ld_cg_v2u64(slot + 7 * kEThreads + tid, a, b);
+                hit = (uint32_t)(a >> 32) == tag && (uint32_t)(b >> 32) == tag;
             }
             return __all_sync(0xffffffffu, hit);
         };
@@ -633,7 +634,7 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             TRACE_E(4);
             // (the request is not issued earlier in the task: holding its 32 registers across E1
             // costs more in spills than the exposed trip from L2)
-            uint4 rv[8];
+            unsigned long long rv[16];
             if (relayed_in) relay_request(slot, rv);
             if (!relayed_in) {
                 if (p.state_in) {

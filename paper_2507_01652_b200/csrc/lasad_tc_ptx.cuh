@@ -211,19 +211,15 @@ __device__ __forceinline__ bool mbar_test_wait(void* bar, unsigned parity)
     return ok != 0;
 }
 
-// 16-byte global accesses that bypass L1 (data written and read by different SMs).
-__device__ __forceinline__ uint4 ld_cg_v4(const uint4* p)
+// 16-byte global accesses, as two 64-bit elements, that bypass L1 (data written and read by
+// different SMs).  Each 64-bit element is accessed as a unit.
+__device__ __forceinline__ void ld_cg_v2u64(const void* p, unsigned long long& a, unsigned long long& b)
 {
-    uint4 v;
-    asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
+    asm volatile("ld.global.cg.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p));
 }
-__device__ __forceinline__ void st_cg_v4(uint4* p, uint4 v)
+__device__ __forceinline__ void st_cg_v2u64(void* p, unsigned long long a, unsigned long long b)
 {
-    asm volatile("st.global.cg.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
-                 : "memory");
+    asm volatile("st.global.cg.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(a), "l"(b) : "memory");
 }
 
 }  // namespace tcx

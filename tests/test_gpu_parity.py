@@ -359,3 +359,34 @@ def test_decode_per_sequence_positions_and_widths(ctx):
             o_ref, s_ref = oracle(q[b:b + 1], k[b:b + 1], v[b:b + 1], g, w, 0, int(pos[b]), 1.0, s_in[b:b + 1])
             assert rel_err(o[b:b + 1], o_ref[:, 0]) <= TOL[torch.bfloat16], (b, use_widths)
             assert rel_err(state[b:b + 1], s_ref) <= 1e-6, (b, use_widths)
+
+
+# ------------------------------------------------------------------------------------------
+# bounded waits: a wait that runs out is reported, nothing hangs, the context stays usable
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("impl", [2, 3])
+def test_expired_device_wait_is_reported_and_context_survives(ctx, impl):
+    """With the poll limit of the device-side waits set to 1, some wait runs out before its
+    barrier completes: the kernel must leave through its normal exit, the status word must say
+    so, and the next call (default limit) must be correct again."""
+    wl = _small("config3", 1, 2)
+    q, k, v = workloads.make_qkv(wl)
+    g = workloads.make_decay(wl)
+    o_ref, s_ref = oracle(q, k, v, g, wl.grid_w)
+    dq, dk_, dv_, dg = _dev(q, k, v, g)
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, impl)
+    try:
+        ctx.set_option(binding.LASAD_OPT_WAIT_LIMIT, 1)
+        ctx.lasad_forward(dq, dk_, dv_, dg, wl.grid_w)
+        torch.cuda.synchronize()                       # returns: no wait is unbounded
+        assert ctx.device_status() == binding.LASAD_ERR_TIMEOUT
+        assert ctx.device_status() == 0                # the query clears the flag
+        ctx.set_option(binding.LASAD_OPT_WAIT_LIMIT, 0)
+        o, s = ctx.lasad_forward(dq, dk_, dv_, dg, wl.grid_w)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        assert rel_err(o, o_ref) <= TOL[torch.bfloat16]
+        assert rel_err(s, s_ref) <= TOL[torch.bfloat16]
+    finally:
+        ctx.set_option(binding.LASAD_OPT_WAIT_LIMIT, 0)
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)

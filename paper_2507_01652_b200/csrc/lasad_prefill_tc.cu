@@ -285,7 +285,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const int s = n % kStages;
             if (!mbar_wait(&sm.bar.full[s], (n / kStages) & 1, limit, abort_flag, p.status)) return false;
             tc_fence_after();
-            if (lane == 0) {
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk)  // 32 bytes along K per step
                     mma_ss(tmem + kColS, dq[s] + 2 * kk, dk[s] + 2 * kk, idesc_s, kk > 0);
@@ -300,7 +300,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             TRACE_M(8 * n + 0);
             if (!mbar_wait(&sm.bar.x_ready, n & 1, limit, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
-            if (lane == 0) {
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K and of V per step
                     mma_ss(tmem + kColDS, dk[s] + 128 * kk, dv[s] + 128 * kk, idesc_kv, kk > 0);
@@ -311,7 +311,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (!mbar_wait(&sm.bar.p_ready, n & 1, limit, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
             TRACE_M(8 * n + 2);
-            if (lane == 0) {
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kC / 16; ++kk)  // A/P: 8 TMEM columns per step (tokens 0..63 at columns
                                                       // 0..31, tokens 64..127 at 64..95); V: 2048 B per step
@@ -328,7 +328,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             TRACE_M(8 * n + 4);
         }
         // make sure nothing is still running on the tensor pipe before TMEM is freed
-        if (lane == 0) {
+        if (elect_one()) {
             mma_commit(&sm.bar.drain);
             for (unsigned it = 0; it < kTeardownLimit; ++it)
                 if (mbar_try_wait(&sm.bar.drain, 0)) break;

@@ -320,7 +320,7 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         auto issue_m1 = [&](int g) {
             const uint64_t dq = (g & 1) ? dq1 : dq0, dk = (g & 1) ? dk1 : dk0;
             tc_fence_after();
-            if (lane == 0) {
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk)  // 32 bytes along K per step
                     mma_ss(tmem + kColS, dq + 2 * kk, dk + 2 * kk, idesc_s, kk > 0);
@@ -334,7 +334,7 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             const uint64_t dq = (g & 1) ? dq1 : dq0, dk = (g & 1) ? dk1 : dk0, dv = (g & 1) ? dv1 : dv0;
             if (!mbar_wait(&sm.bar.x_ready, g & 1, limit, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
-            if (lane == 0) {
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K and of V per step
                     mma_ss(tmem + kColDS, dk + 128 * kk, dv + 128 * kk, idesc_kv, kk > 0);
@@ -344,7 +344,7 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             if (!mbar_wait(&sm.bar.p_ready, g & 1, limit, abort_flag, p.status)) { ok = false; break; }
             if (!mbar_wait(&sm.bar.sb_ready, g & 1, limit, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
-            if (lane == 0) {
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kC / 16; ++kk)  // A/P: 8 TMEM columns per step (tokens 0..63 at columns
                                                       // 0..31, tokens 64..127 at 64..95); V: 2048 B per step
@@ -367,7 +367,7 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             }
         }
         // make sure nothing is still running on the tensor pipe before TMEM is freed
-        if (lane == 0) {
+        if (elect_one()) {
             mma_commit(&sm.bar.drain);
             for (unsigned it = 0; it < kTeardownLimit; ++it)
                 if (mbar_try_wait(&sm.bar.drain, 0)) break;

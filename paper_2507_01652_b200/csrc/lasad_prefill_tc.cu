@@ -237,7 +237,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     if (warp == 9) {
         // ===================== TMA warp: loads two chunks ahead, stores each output tile =======
-        if (lane == 0) {
+        if (elect_one()) {
             auto issue_loads = [&](int n) {
                 const int s = n % kStages;
                 mbar_arrive_expect_tx(&sm.bar.full[s], 3 * kTileBytes);

@@ -275,7 +275,7 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
     if (warp == 9) {
         // ===================== TMA warp: loads two tasks ahead, stores each output tile ========
-        if (lane == 0) {
+        if (elect_one()) {
             auto issue_loads = [&](int g) {
                 const Task t = decode_task(first + g * G, p.X, p.H);
                 const int s = g % kStages;

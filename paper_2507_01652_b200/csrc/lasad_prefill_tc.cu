@@ -305,6 +305,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K and of V per step
                     mma_ss(tmem + kColDS, dk[s] + 128 * kk, dv[s] + 128 * kk, idesc_kv, kk > 0);
                 mma_commit(&sm.bar.ds_done);
+                // Normal path: the state's contribution to O needs nothing from E1 (the state copy
+                // was written, and the previous O read, before x_ready), so it opens the
+                // accumulator now and only the A V~ MMAs remain once A is ready.
+                if (fast) {
+#pragma unroll
+                    for (int kk = 0; kk < kD / 16; ++kk)
+                        mma_ss(tmem + kColO, dq[s] + 2 * kk, d_sb + 128 * kk, idesc_qs, kk > 0);
+                }
             }
             __syncwarp();
             TRACE_M(8 * n + 1);
@@ -316,10 +324,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 for (int kk = 0; kk < kC / 16; ++kk)  // A/P: 8 TMEM columns per step (tokens 0..63 at columns
                                                       // 0..31, tokens 64..127 at 64..95); V: 2048 B per step
                     mma_ts(tmem + kColO, tmem + kColS + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), dv[s] + 128 * kk,
-                           idesc_pv, kk > 0);
+                           idesc_pv, fast || kk > 0);
+                if (!fast) {
+                    // exact path: Q~ is written during E1, so its MMAs come last
 #pragma unroll
-                for (int kk = 0; kk < kD / 16; ++kk)
-                    mma_ss(tmem + kColO, dq[s] + 2 * kk, d_sb + 128 * kk, idesc_qs, 1);
+                    for (int kk = 0; kk < kD / 16; ++kk)
+                        mma_ss(tmem + kColO, dq[s] + 2 * kk, d_sb + 128 * kk, idesc_qs, 1);
+                }
                 mma_commit(&sm.bar.o_done);
             }
             __syncwarp();

@@ -238,27 +238,40 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (warp == 9) {
         // ===================== TMA warp: loads two chunks ahead, stores each output tile =======
         if (elect_one()) {
-            auto issue_loads = [&](int n) {
+            // A stage is refilled in two steps: K and V as soon as every MMA of the chunk that used
+            // them has retired, Q (whose buffer stages the output tile) once the store has read it.
+            auto issue_kv = [&](int n) {
                 const int s = n % kStages;
                 mbar_arrive_expect_tx(&sm.bar.full[s], 3 * kTileBytes);
-                tma_load_4d(sm.q[s], &tm_q, &sm.bar.full[s], 0, h, n * kC, b);
                 tma_load_4d(sm.k[s], &tm_k, &sm.bar.full[s], 0, h, n * kC, b);
                 tma_load_4d(sm.v[s], &tm_v, &sm.bar.full[s], 0, h, n * kC, b);
             };
+            auto issue_q = [&](int n) {
+                const int s = n % kStages;
+                tma_load_4d(sm.q[s], &tm_q, &sm.bar.full[s], 0, h, n * kC, b);
+            };
             int loads_issued = min(n_chunks, kStages);
-            for (int n = 0; n < loads_issued; ++n) issue_loads(n);
+            for (int n = 0; n < loads_issued; ++n) {
+                issue_kv(n);
+                issue_q(n);
+            }
             for (int n = 0; n < n_chunks; ++n) {
                 const int s = n % kStages;
-                // the output tile of chunk n sits in the Q buffer of its stage; by now every MMA
-                // that read this stage has retired (the element-wise warps waited for o_done)
-                if (!mbar_wait(&sm.bar.st_ready, n & 1, limit, abort_flag, p.status)) break;
-                tma_store_4d(&tm_o, sm.q[s], 0, h, n * kC, b);
-                tma_store_commit();
-                if (n + kStages < n_chunks) {
-                    tma_store_wait_read();        // the store has finished reading the buffer
-                    issue_loads(n + kStages);
+                const bool refill = n + kStages < n_chunks;
+                if (refill) {
+                    if (!mbar_wait(&sm.bar.o_done, n & 1, limit, abort_flag, p.status)) break;
+                    issue_kv(n + kStages);
                     loads_issued = n + kStages + 1;
                 }
+                // the output tile of chunk n sits in the Q buffer of its stage
+                const bool staged = mbar_wait(&sm.bar.st_ready, n & 1, limit, abort_flag, p.status);
+                if (staged) {
+                    tma_store_4d(&tm_o, sm.q[s], 0, h, n * kC, b);
+                    tma_store_commit();
+                    if (refill) tma_store_wait_read();        // the store has finished reading the buffer
+                }
+                if (refill) issue_q(n + kStages);              // (also after a failed wait: the stage's barrier must complete)
+                if (!staged) break;
             }
             tma_store_wait_all();
             // leave only when every issued load has landed (they write this CTA's shared memory)

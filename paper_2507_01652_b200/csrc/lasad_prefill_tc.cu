@@ -364,46 +364,46 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const int grp = warp >> 2;               // which half of the quadrant's columns
         const int i = qd * 32 + lane;            // chunk row owned by this thread
         const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
-        const int srow = qd * 16 + lane;         // state row (M = 64 TMEM layout: lanes 0..15 of a quadrant)
-        const bool has_state = lane < 16;
+        // State ownership.  The dS accumulator (M = 64 layout) keeps state rows 16 qd .. 16 qd + 15 in
+        // the first 16 TMEM lanes of quadrant qd; the 16x256b load spreads this warp's 16 rows x 32
+        // columns (columns 32 grp ..) over all 32 threads, 16 values each: for column group k,
+        // st[4k], st[4k+1] = (row r0, columns c0 + 8k, + 1), st[4k+2], st[4k+3] = (row r0 + 8, same).
+        const int r0 = qd * 16 + (lane >> 2);
+        const int c0 = 32 * grp + 2 * (lane & 3);
         const size_t unit = (size_t)blockIdx.x * kD * kD;
 
         // position of the call's first token relative to the grid (SAD rule, Section 3.4)
         GridPos gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0, lane);
 
-        float st[32];                            // state[srow][32 grp .. 32 grp + 31], fp32 master
+        float st[16];                            // fp32 master state, this thread's 16 values
 #pragma unroll
-        for (int e = 0; e < 32; ++e) st[e] = 0.0f;
-        if (has_state && p.state_in) {
-            const float4* src = reinterpret_cast<const float4*>(p.state_in + unit + (size_t)srow * kD + 32 * grp);
+        for (int e = 0; e < 16; ++e) st[e] = 0.0f;
+        if (p.state_in) {
 #pragma unroll
-            for (int e4 = 0; e4 < 8; ++e4) {
-                const float4 t = src[e4];
-                st[4 * e4] = t.x; st[4 * e4 + 1] = t.y; st[4 * e4 + 2] = t.z; st[4 * e4 + 3] = t.w;
+            for (int k = 0; k < 4; ++k) {
+                const float2 a = *reinterpret_cast<const float2*>(p.state_in + unit + (size_t)r0 * kD + c0 + 8 * k);
+                const float2 c = *reinterpret_cast<const float2*>(p.state_in + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k);
+                st[4 * k] = a.x; st[4 * k + 1] = a.y; st[4 * k + 2] = c.x; st[4 * k + 3] = c.y;
             }
         }
-        // bf16 copy of mult * state for the Q x state MMA of the next chunk
+        // bf16 copy of mult * state for the Q x state MMA of the next chunk: [dk][dv] rows of 128 B,
+        // 16-byte pieces swizzled by the row; this thread writes eight bf16 pairs
         auto write_state_bf16 = [&](float mult) {
-            if (has_state) {
-                uint4* row = reinterpret_cast<uint4*>(sm.sb + srow * 128);
+            unsigned char* row0 = sm.sb + r0 * 128 + 4 * (lane & 3);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint4 x;
-                    x.x = pack_bf16(mult * st[8 * c], mult * st[8 * c + 1]);
-                    x.y = pack_bf16(mult * st[8 * c + 2], mult * st[8 * c + 3]);
-                    x.z = pack_bf16(mult * st[8 * c + 4], mult * st[8 * c + 5]);
-                    x.w = pack_bf16(mult * st[8 * c + 6], mult * st[8 * c + 7]);
-                    row[(4 * grp + c) ^ (srow & 7)] = x;
-                }
+            for (int k = 0; k < 4; ++k) {
+                const int piece = ((4 * grp + k) ^ (r0 & 7)) * 16;    // r0 + 8 has the same low bits
+                *reinterpret_cast<uint32_t*>(row0 + piece) = pack_bf16(mult * st[4 * k], mult * st[4 * k + 1]);
+                *reinterpret_cast<uint32_t*>(row0 + 8 * 128 + piece) = pack_bf16(mult * st[4 * k + 2], mult * st[4 * k + 3]);
             }
         };
-        // E3: S_new = g * S_prev + dS (this thread's 32 columns of its state row)
+        // E3: S_new = g * S_prev + dS
         auto update_state = [&](float g) {
-            uint32_t dsv[32];
-            tmem_ld32(tmem + lane_base + kColDS + 32 * grp, dsv);
+            uint32_t dsv[16];
+            tmem_ld_16x256b_x4(tmem + lane_base + kColDS + 32 * grp, dsv);
             tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) st[e] = fmaf(g, st[e], __uint_as_float(dsv[e]));
+            for (int e = 0; e < 16; ++e) st[e] = fmaf(g, st[e], __uint_as_float(dsv[e]));
         };
         // E2: this thread's 32 columns of output row i -> bf16 -> the stage's Q buffer
         auto stage_output = [&](int s, float f) {
@@ -561,11 +561,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 mbar_arrive(&sm.bar.st_ready);
             }
         }
-        if (ok && has_state && p.state_out) {
-            float4* dst = reinterpret_cast<float4*>(p.state_out + unit + (size_t)srow * kD + 32 * grp);
+        if (ok && p.state_out) {
 #pragma unroll
-            for (int e4 = 0; e4 < 8; ++e4)
-                dst[e4] = make_float4(st[4 * e4], st[4 * e4 + 1], st[4 * e4 + 2], st[4 * e4 + 3]);
+            for (int k = 0; k < 4; ++k) {
+                *reinterpret_cast<float2*>(p.state_out + unit + (size_t)r0 * kD + c0 + 8 * k) = make_float2(st[4 * k], st[4 * k + 1]);
+                *reinterpret_cast<float2*>(p.state_out + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k) =
+                    make_float2(st[4 * k + 2], st[4 * k + 3]);
+            }
         }
     }
 

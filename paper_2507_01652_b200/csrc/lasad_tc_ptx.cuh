@@ -177,6 +177,33 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
+// Two fp32 products in one instruction (packed f32x2 arithmetic of sm_100): {a0 * b, a1 * b}.
+__device__ __forceinline__ void mul2(float a0, float a1, float b, float& r0, float& r1)
+{
+    unsigned long long pa, pb, pr;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(pa) : "f"(a0), "f"(a1));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(pb) : "f"(b));
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(pr) : "l"(pa), "l"(pb));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(pr));
+}
+// {a0 * b + c0, a1 * b + c1}
+__device__ __forceinline__ void fma2(float a0, float a1, float b, float c0, float c1, float& r0, float& r1)
+{
+    unsigned long long pa, pb, pc, pr;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(pa) : "f"(a0), "f"(a1));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(pb) : "f"(b));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(pc) : "f"(c0), "f"(c1));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(pr) : "l"(pa), "l"(pb), "l"(pc));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(pr));
+}
+// bf16 pair * f -> bf16 pair (fp32 products, one rounding)
+__device__ __forceinline__ uint32_t scale_bf16x2(uint32_t x, float f)
+{
+    float r0, r1;
+    mul2(bf16_lo(x), bf16_hi(x), f, r0, r1);
+    return pack_bf16(r0, r1);
+}
+
 // Multiply `pieces` 16-byte pieces (8 bf16 each) of one 128-byte tile row by a scalar, in
 // place (fp32 product, one rounding).  The swizzle only permutes 16-byte pieces within the row,
 // so a row-uniform factor needs no un-swizzling; `rot` staggers the order in which neighbouring
@@ -189,10 +216,10 @@ __device__ __forceinline__ void scale_row_inplace(unsigned char* row, float f, i
     for (int c = 0; c < kPieces; ++c) {
         const int idx = (first + c) ^ rot;
         uint4 x = p[idx];
-        x.x = pack_bf16(bf16_lo(x.x) * f, bf16_hi(x.x) * f);
-        x.y = pack_bf16(bf16_lo(x.y) * f, bf16_hi(x.y) * f);
-        x.z = pack_bf16(bf16_lo(x.z) * f, bf16_hi(x.z) * f);
-        x.w = pack_bf16(bf16_lo(x.w) * f, bf16_hi(x.w) * f);
+        x.x = scale_bf16x2(x.x, f);
+        x.y = scale_bf16x2(x.y, f);
+        x.z = scale_bf16x2(x.z, f);
+        x.w = scale_bf16x2(x.w, f);
         p[idx] = x;
     }
 }

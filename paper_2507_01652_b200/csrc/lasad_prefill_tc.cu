@@ -104,15 +104,17 @@ struct TcParams {
 // Decay bookkeeping of one chunk, computed by every warp on its own with four ballots (one per
 // 32-token block): which steps decay, and from their popcounts n_i for the thread's own row.
 struct ChunkDecay {
-    unsigned mask[4];   // bit l of mask[x]: token 32 x + l of the chunk is a decaying step
-    int cum[4];         // decaying steps up to the end of block x
-    int ni;             // n of the thread's own row
-    int n_last;         // n of the chunk's last token
+    unsigned m0, m1, m2, m3;   // bit l of m<x>: token 32 x + l of the chunk is a decaying step
+    int c0, c1, c2;            // decaying steps up to the end of block 0, 1, 2
+    int ni;                    // n of the thread's own row
+    int n_last;                // n of the chunk's last token
     // n of chunk column j (warp-uniform j)
     __device__ __forceinline__ int n_of(int j) const
     {
         const int x = j >> 5;
-        return (x ? cum[x - 1] : 0) + __popc(mask[x] & (0xffffffffu >> (31 - (j & 31))));
+        const unsigned m = x == 0 ? m0 : x == 1 ? m1 : x == 2 ? m2 : m3;
+        const int before = x == 0 ? 0 : x == 1 ? c0 : x == 2 ? c1 : c2;
+        return before + __popc(m & (0xffffffffu >> (31 - (j & 31))));
     }
 };
 
@@ -154,21 +156,23 @@ __device__ __forceinline__ GridPos grid_pos_init(int grid_w, int prefix_len, lon
 __device__ __forceinline__ ChunkDecay chunk_decay(GridPos& g, int cs, int L, int qd, int lane)
 {
     ChunkDecay d;
-    int run = 0;
+    unsigned mk[4];
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
         const int tok = 32 * x + lane;
         const int m = g.phase + g.r[x];
         const bool boundary = g.grid_w > 0 && cs + tok >= g.pre && (m == 0 || m == g.grid_w);
-        d.mask[x] = __ballot_sync(0xffffffffu, tok < L && !boundary);
-        run += __popc(d.mask[x]);
-        d.cum[x] = run;
+        mk[x] = __ballot_sync(0xffffffffu, tok < L && !boundary);
     }
+    d.m0 = mk[0]; d.m1 = mk[1]; d.m2 = mk[2]; d.m3 = mk[3];
+    d.c0 = __popc(d.m0);
+    d.c1 = d.c0 + __popc(d.m1);
+    d.c2 = d.c1 + __popc(d.m2);
+    d.n_last = d.c2 + __popc(d.m3);
     g.phase += g.step;
     if (g.phase >= g.grid_w) g.phase -= g.grid_w;
-    d.n_last = run;
-    const unsigned own = qd == 0 ? d.mask[0] : qd == 1 ? d.mask[1] : qd == 2 ? d.mask[2] : d.mask[3];
-    const int before = qd == 0 ? 0 : qd == 1 ? d.cum[0] : qd == 2 ? d.cum[1] : d.cum[2];
+    const unsigned own = qd == 0 ? d.m0 : qd == 1 ? d.m1 : qd == 2 ? d.m2 : d.m3;
+    const int before = qd == 0 ? 0 : qd == 1 ? d.c0 : qd == 2 ? d.c1 : d.c2;
     d.ni = before + __popc(own & (0xffffffffu >> (31 - lane)));
     return d;
 }
@@ -287,21 +291,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         constexpr uint32_t idesc_qs = make_idesc(128, 64, 0, 1);   // Q (K-major) x state (MN-major)
         constexpr uint32_t idesc_kv = make_idesc(64, 64, 1, 1);    // K^T (MN-major) x V (MN-major)
         const uint64_t d_sb = make_desc(smem_u32(sm.sb));
-        uint64_t dq[kStages], dk[kStages], dv[kStages];
-#pragma unroll
-        for (int s = 0; s < kStages; ++s) {
-            dq[s] = make_desc(smem_u32(sm.q[s]));
-            dk[s] = make_desc(smem_u32(sm.k[s]));
-            dv[s] = make_desc(smem_u32(sm.v[s]));
-        }
+        const uint64_t dq0 = make_desc(smem_u32(sm.q[0])), dq1 = make_desc(smem_u32(sm.q[1]));
+        const uint64_t dk0 = make_desc(smem_u32(sm.k[0])), dk1 = make_desc(smem_u32(sm.k[1]));
+        const uint64_t dv0 = make_desc(smem_u32(sm.v[0])), dv1 = make_desc(smem_u32(sm.v[1]));
         auto issue_m1 = [&](int n) {
             const int s = n % kStages;
+            const uint64_t dqs = s ? dq1 : dq0, dks = s ? dk1 : dk0;
             if (!mbar_wait(&sm.bar.full[s], (n / kStages) & 1, limit, abort_flag, p.status)) return false;
             tc_fence_after();
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk)  // 32 bytes along K per step
-                    mma_ss(tmem + kColS, dq[s] + 2 * kk, dk[s] + 2 * kk, idesc_s, kk > 0);
+                    mma_ss(tmem + kColS, dqs + 2 * kk, dks + 2 * kk, idesc_s, kk > 0);
                 mma_commit(&sm.bar.s_done);
             }
             __syncwarp();
@@ -310,13 +311,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         bool ok = n_chunks > 0 && issue_m1(0);
         for (int n = 0; ok && n < n_chunks; ++n) {
             const int s = n % kStages;
+            const uint64_t dqs = s ? dq1 : dq0, dks = s ? dk1 : dk0, dvs = s ? dv1 : dv0;
             TRACE_M(8 * n + 0);
             if (!mbar_wait(&sm.bar.x_ready, n & 1, limit, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K and of V per step
-                    mma_ss(tmem + kColDS, dk[s] + 128 * kk, dv[s] + 128 * kk, idesc_kv, kk > 0);
+                    mma_ss(tmem + kColDS, dks + 128 * kk, dvs + 128 * kk, idesc_kv, kk > 0);
                 mma_commit(&sm.bar.ds_done);
                 // Normal path: the state's contribution to O needs nothing from E1 (the state copy
                 // was written, and the previous O read, before x_ready), so it opens the
@@ -324,7 +326,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (fast) {
 #pragma unroll
                     for (int kk = 0; kk < kD / 16; ++kk)
-                        mma_ss(tmem + kColO, dq[s] + 2 * kk, d_sb + 128 * kk, idesc_qs, kk > 0);
+                        mma_ss(tmem + kColO, dqs + 2 * kk, d_sb + 128 * kk, idesc_qs, kk > 0);
                 }
             }
             __syncwarp();
@@ -336,13 +338,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
                 for (int kk = 0; kk < kC / 16; ++kk)  // A/P: 8 TMEM columns per step (tokens 0..63 at columns
                                                       // 0..31, tokens 64..127 at 64..95); V: 2048 B per step
-                    mma_ts(tmem + kColO, tmem + kColS + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), dv[s] + 128 * kk,
+                    mma_ts(tmem + kColO, tmem + kColS + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), dvs + 128 * kk,
                            idesc_pv, fast || kk > 0);
                 if (!fast) {
                     // exact path: Q~ is written during E1, so its MMAs come last
 #pragma unroll
                     for (int kk = 0; kk < kD / 16; ++kk)
-                        mma_ss(tmem + kColO, dq[s] + 2 * kk, d_sb + 128 * kk, idesc_qs, 1);
+                        mma_ss(tmem + kColO, dqs + 2 * kk, d_sb + 128 * kk, idesc_qs, 1);
                 }
                 mma_commit(&sm.bar.o_done);
             }

@@ -333,8 +333,11 @@ int lasad_forward_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, co
     fill_args(a, ctx, p);
     a.q = q; a.k = k; a.v = v; a.o = o;
     a.decay = nullptr; a.state_in = state_in; a.state_out = state_out;
-    const cudaError_t e = lasad::launch_prefill_gated(a, gate, p->dk, p->dtype == LASAD_BF16,
-                                                      static_cast<cudaStream_t>(cuda_stream));
+    // tensor cores where the shape allows it, unless the CUDA-core implementation is asked for
+    const bool bf16 = p->dtype == LASAD_BF16;
+    const bool tc = ctx->opt_prefill_impl != 1 && lasad::prefill_gated_tc_supported(p->dk, p->dv, bf16);
+    const cudaError_t e = tc ? lasad::launch_prefill_gated_tc(a, gate, static_cast<cudaStream_t>(cuda_stream))
+                             : lasad::launch_prefill_gated(a, gate, p->dk, bf16, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     ctx->launches += 1;
     return LASAD_OK;

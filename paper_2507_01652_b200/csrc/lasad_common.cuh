@@ -65,6 +65,9 @@ cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool d
 cudaError_t launch_decode_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, bool decay_on, int tpu,
                                 cudaStream_t st);
 cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, cudaStream_t st);
+// Tensor-core form of the gated prefill (bf16, dk = dv = 64).
+bool prefill_gated_tc_supported(int dk, int dv, bool bf16);
+cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, cudaStream_t st);
 bool prefill_tc_supported(int dk, int dv, bool bf16);
 cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st);
 

@@ -1,0 +1,616 @@
+// LASAD prefill with the paper's data-dependent gate on the 5th-generation tensor cores
+// (sm_100a): bf16 I/O, d_k = d_v = 64, fp32 accumulation, fp32 master state.
+//
+// The operator is Algorithm 1 with a decay vector lambda_t in [0,1]^dk per token and the SAD
+// rule of Section 3.4 on top (decay 1 on the step that absorbs the last token of a grid row):
+//
+//     s_t = diag(Lambda_t) s_{t-1} + k_t v_t^T,    o_t = scale * q_t^T s_t,    k_t = 1 - lambda_t if tied.
+//
+// One CTA owns one (batch, head) and walks its sequence in chunks of C = 128 tokens; two CTAs fit
+// on an SM.  With b_i[c] = sum_{u <= i in the chunk} log2 Lambda_u[c] (non-increasing in i) the
+// recurrence unrolled over a chunk is
+//
+//     o_i   = scale * ( sum_{j<=i} sum_c q_i[c] k_j[c] 2^(b_i[c]-b_j[c]) v_j + sum_c q_i[c] 2^(b_i[c]) S_prev[c,:] )
+//     S_new = diag(2^b_N) S_prev + sum_j diag(2^(b_N-b_j)) k_j v_j^T
+//
+// and the per-channel decay is split around a reference r[c] = b_N[c] / 2 so that each factor
+// goes onto one operand and the scores are a plain product of two matrices:
+//
+//     Q~ = Q o 2^(b_i - r),   K~ = K o 2^(r - b_j)           element-wise, bf16, written to their own tiles
+//     S  = Q~ K~^T                          (M1)   tcgen05.mma 128x128x64
+//     A  = tril(S) -> bf16                  (E1)   back into TMEM over S's own columns
+//     dS = K~^T V                           (M2a)  tcgen05.mma 64x64x128
+//     O  = A V + Q~ (diag(2^r) S_prev)      (M2b)  tcgen05.mma 128x64x128 (tmem x smem) + 128x64x64
+//     S_new = diag(2^b_N) S_prev + diag(2^(b_N - r)) dS       fp32 registers
+//
+// Every exponent that is formed lies within +-|b_N|/2.  A chunk is taken in one pass while
+// |b_N[c]| <= 200 for all channels (an average decay above 0.34 per step); otherwise it is cut
+// into aligned segments of 64, 32, 16 or, at worst, single tokens (log2 of a decay is clamped at
+// -150, below which the decay is 0 in fp32 anyway), each a pass of the same pipeline over the
+// segment's rows with all other rows of Q~ and K~ zero, so the result stays exact for every gate
+// in [0,1] and only pathological inputs pay for it.
+//
+// Warp roles: warps 0-7 do the element-wise work.  For the scaling they split the chunk by rows
+// (warp w: rows 16 w ..), lanes across channel pairs, so the running sum b needs no exchange
+// inside a warp and only eight partial sums per channel cross warps through shared memory; for
+// the TMEM stages warp w works on lane quadrant w & 3 as in the scalar-decay kernel.  Warp 8
+// issues the MMAs, warp 9 the TMA loads and stores.  All waits are bounded: a wait that runs out
+// raises a status word the host can read and the CTA leaves through the normal exit.
+#include "lasad_common.cuh"
+#include "lasad_tc_ptx.cuh"
+#include "lasad_tc_tma.cuh"
+
+namespace lasad {
+namespace {
+
+using namespace tcx;
+
+constexpr int kC = 128;                    // chunk length (tokens) = MMA M
+constexpr int kD = 64;                     // d_k = d_v
+constexpr int kEThreads = 256;             // element-wise warps 0-7
+constexpr int kThreads = kEThreads + 64;   // + the MMA warp and the TMA warp
+constexpr int kTileBytes = kC * kD * 2;    // 16 KB: one [128 x 64] bf16 tile, 128 B rows
+constexpr int kTmemCols = 256;
+constexpr uint32_t kColS = 0;      // S (fp32, 128 columns); A (bf16 pairs) aliases columns 0..31 and 64..95
+constexpr uint32_t kColO = 128;    // O accumulator, 64 columns
+constexpr uint32_t kColDS = 192;   // dS accumulator (M = 64 layout), 64 columns
+constexpr unsigned kTeardownLimit = 1u << 26;
+constexpr float kMinLog2 = -150.0f;    // log2 of a decay is clamped here (2^-150 is 0 in fp32)
+constexpr float kSafeRange = 200.0f;   // largest |sum of log2 decays| one pass may span
+
+struct __align__(8) Barriers {
+    unsigned long long full_a;     // gate (and key) tile of the chunk has landed
+    unsigned long long full_b;     // query and value tiles have landed
+    unsigned long long scan;       // partial sums of the chunk are in shared memory (256 arrivals)
+    unsigned long long gk_free;    // last read of the gate and key tiles of the chunk (256 arrivals)
+    unsigned long long x_ready;    // Q~, K~ and the state copy of a pass are written (256 arrivals)
+    unsigned long long s_done;     // M1 complete
+    unsigned long long ds_done;    // dS MMAs complete
+    unsigned long long p_ready;    // A in TMEM (256 arrivals)
+    unsigned long long o_done;     // O MMAs complete (and every MMA issued before them)
+    unsigned long long st_ready;   // output tile of the chunk staged in shared memory (256 arrivals)
+    unsigned long long drain;      // teardown: all MMAs retired
+};
+
+struct Smem {
+    // tiles first: each must sit on a 1024-byte boundary (128-byte swizzle atom = 8 rows)
+    unsigned char q[kTileBytes];    // queries; its rows are overwritten by the output rows as they complete
+    unsigned char k[kTileBytes];
+    unsigned char v[kTileBytes];
+    unsigned char g[kTileBytes];    // gate lambda
+    unsigned char qt[kTileBytes];   // Q~
+    unsigned char kt[kTileBytes];   // K~
+    unsigned char sb[kD * kD * 2];  // bf16 copy of diag(2^r) state, [dk][dv], 128 B rows, swizzled
+    float segsum[8][kD];            // sum of log2 Lambda over rows 16 x .. 16 x + 15, per channel
+    Barriers bar;
+    uint32_t tmem_base;
+    int npass;                      // passes of the current chunk (written before the first x_ready)
+    int abort_flag;
+};
+
+struct GatedParams {
+    int B, T, H;
+    int grid_w, prefix_len;
+    long long t0;
+    float scale;
+    int tied;                // key tied to the gate: k = 1 - lambda, no key tensor
+    const float* state_in;
+    float* state_out;
+    int* status;
+    unsigned wait_limit;
+};
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2(float x)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// log2 of a gate value under the clamp; 0 and negative values count as decay 0
+__device__ __forceinline__ float log2_decay(float g) { return fmaxf(lg2(fmaxf(g, 0.0f)), kMinLog2); }
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g,
+                        const __grid_constant__ CUtensorMap tm_o, GatedParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.x / p.H, h = blockIdx.x % p.H;
+    const int n_chunks = (p.T + kC - 1) / kC;
+    volatile int* abort_flag = &sm.abort_flag;
+    const unsigned limit = p.wait_limit;
+
+    // ---- set-up ---------------------------------------------------------------------------
+    if (tid == 0) {
+        mbar_init(&sm.bar.full_a, 1);
+        mbar_init(&sm.bar.full_b, 1);
+        mbar_init(&sm.bar.scan, kEThreads);
+        mbar_init(&sm.bar.gk_free, kEThreads);
+        mbar_init(&sm.bar.x_ready, kEThreads);
+        mbar_init(&sm.bar.s_done, 1);
+        mbar_init(&sm.bar.ds_done, 1);
+        mbar_init(&sm.bar.p_ready, kEThreads);
+        mbar_init(&sm.bar.o_done, 1);
+        mbar_init(&sm.bar.st_ready, kEThreads);
+        mbar_init(&sm.bar.drain, 1);
+        sm.abort_flag = 0;
+        sm.npass = 1;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 8) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    if (warp == 9) {
+        // ===================== TMA warp ========================================================
+        // One set of tiles; each is refilled for the next chunk as soon as its last reader is done:
+        // gate and key after the chunk's last scaling pass, value after the last MMA, query (whose
+        // tile carries the output rows) after the store has read it.
+        if (elect_one()) {
+            const unsigned a_bytes = (p.tied ? 1 : 2) * kTileBytes;
+            auto issue_a = [&](int n) {
+                mbar_arrive_expect_tx(&sm.bar.full_a, a_bytes);
+                tma_load_4d(sm.g, &tm_g, &sm.bar.full_a, 0, h, n * kC, b);
+                if (!p.tied) tma_load_4d(sm.k, &tm_k, &sm.bar.full_a, 0, h, n * kC, b);
+            };
+            auto issue_v = [&](int n) {
+                mbar_arrive_expect_tx(&sm.bar.full_b, 2 * kTileBytes);
+                tma_load_4d(sm.v, &tm_v, &sm.bar.full_b, 0, h, n * kC, b);
+            };
+            auto issue_q = [&](int n) { tma_load_4d(sm.q, &tm_q, &sm.bar.full_b, 0, h, n * kC, b); };
+            int a_issued = 0, b_issued = 0;     // chunks whose loads have been issued (b: both tiles)
+            if (n_chunks > 0) {
+                issue_a(0);
+                issue_v(0);
+                issue_q(0);
+                a_issued = b_issued = 1;
+            }
+            for (int n = 0; n < n_chunks; ++n) {
+                const bool more = n + 1 < n_chunks;
+                if (more) {
+                    if (!mbar_wait(&sm.bar.gk_free, n & 1, limit, abort_flag, p.status)) break;
+                    issue_a(n + 1);
+                    a_issued = n + 2;
+                }
+                const bool staged = mbar_wait(&sm.bar.st_ready, n & 1, limit, abort_flag, p.status);
+                if (more) issue_v(n + 1);       // (also after a failed wait: the barrier's byte count must complete)
+                if (staged) {
+                    tma_store_4d(&tm_o, sm.q, 0, h, n * kC, b);
+                    tma_store_commit();
+                    if (more) tma_store_wait_read();
+                }
+                if (more) {
+                    issue_q(n + 1);
+                    b_issued = n + 2;
+                }
+                if (!staged) break;
+            }
+            tma_store_wait_all();
+            // leave only when every issued load has landed (they write this CTA's shared memory)
+            if (a_issued > 0)
+                for (unsigned it = 0; it < kTeardownLimit; ++it)
+                    if (mbar_try_wait(&sm.bar.full_a, (a_issued - 1) & 1)) break;
+            if (b_issued > 0)
+                for (unsigned it = 0; it < kTeardownLimit; ++it)
+                    if (mbar_try_wait(&sm.bar.full_b, (b_issued - 1) & 1)) break;
+        }
+        __syncwarp();
+    } else if (warp == 8) {
+        // ===================== MMA issuer: the whole warp runs the loop, one lane issues =======
+        constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);   // Q~ (K-major) x K~ (K-major)
+        constexpr uint32_t idesc_pv = make_idesc(128, 64, 0, 1);   // A (tmem) x V (MN-major)
+        constexpr uint32_t idesc_qs = make_idesc(128, 64, 0, 1);   // Q~ (K-major) x state (MN-major)
+        constexpr uint32_t idesc_kv = make_idesc(64, 64, 1, 1);    // K~^T (MN-major) x V (MN-major)
+        const uint64_t d_sb = make_desc(smem_u32(sm.sb));
+        const uint64_t d_q = make_desc(smem_u32(sm.qt));
+        const uint64_t d_k = make_desc(smem_u32(sm.kt));
+        const uint64_t d_v = make_desc(smem_u32(sm.v));
+        bool ok = true;
+        unsigned it = 0;                // passes so far: phase of the per-pass barriers
+        for (int n = 0; ok && n < n_chunks; ++n) {
+            int np = 1;
+            for (int ps = 0; ok && ps < np; ++ps, ++it) {
+                if (!mbar_wait(&sm.bar.x_ready, it & 1, limit, abort_flag, p.status)) { ok = false; break; }
+                if (ps == 0) {
+                    np = *reinterpret_cast<volatile int*>(&sm.npass);
+                    // the value tile was written by the TMA unit: observe its barrier here as well
+                    if (!mbar_wait(&sm.bar.full_b, n & 1, limit, abort_flag, p.status)) { ok = false; break; }
+                }
+                tc_fence_after();
+                if (elect_one()) {
+#pragma unroll
+                    for (int kk = 0; kk < kD / 16; ++kk)  // 32 bytes along K per step
+                        mma_ss(tmem + kColS, d_q + 2 * kk, d_k + 2 * kk, idesc_s, kk > 0);
+                    mma_commit(&sm.bar.s_done);
+#pragma unroll
+                    for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K~ and of V per step
+                        mma_ss(tmem + kColDS, d_k + 128 * kk, d_v + 128 * kk, idesc_kv, kk > 0);
+                    mma_commit(&sm.bar.ds_done);
+                    // the state's contribution opens the O accumulator; A V is added once A is ready
+#pragma unroll
+                    for (int kk = 0; kk < kD / 16; ++kk)
+                        mma_ss(tmem + kColO, d_q + 2 * kk, d_sb + 128 * kk, idesc_qs, kk > 0);
+                }
+                __syncwarp();
+                if (!mbar_wait(&sm.bar.p_ready, it & 1, limit, abort_flag, p.status)) { ok = false; break; }
+                tc_fence_after();
+                if (elect_one()) {
+#pragma unroll
+                    for (int kk = 0; kk < kC / 16; ++kk)  // A: 8 TMEM columns per step (tokens 0..63 at columns
+                                                          // 0..31, tokens 64..127 at 64..95); V: 2048 B per step
+                        mma_ts(tmem + kColO, tmem + kColS + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), d_v + 128 * kk,
+                               idesc_pv, 1);
+                    mma_commit(&sm.bar.o_done);
+                }
+                __syncwarp();
+            }
+        }
+        // make sure nothing is still running on the tensor pipe before TMEM is freed
+        if (elect_one()) {
+            mma_commit(&sm.bar.drain);
+            for (unsigned w = 0; w < kTeardownLimit; ++w)
+                if (mbar_try_wait(&sm.bar.drain, 0)) break;
+        }
+        __syncwarp();
+    } else {
+        // ===================== element-wise warps ==============================================
+        const int qd = warp & 3;                 // TMEM lane quadrant
+        const int grp = warp >> 2;               // which half of the quadrant's columns
+        const int i = qd * 32 + lane;            // chunk row owned by this thread in the TMEM stages
+        const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+        // State ownership as in the scalar-decay kernel: the 16x256b load of the dS accumulator
+        // (M = 64 layout) gives this thread, for column group k, st[4k], st[4k+1] = (row r0,
+        // columns c0 + 8k, + 1) and st[4k+2], st[4k+3] = (row r0 + 8, same columns).
+        const int r0 = qd * 16 + (lane >> 2);
+        const int c0 = 32 * grp + 2 * (lane & 3);
+        const size_t unit = (size_t)blockIdx.x * kD * kD;
+        // Scaling role: rows 16 warp .. 16 warp + 15, channels 2 lane and 2 lane + 1.  Byte offset
+        // of that channel pair in row r of a tile: r * 128 + (((lane >> 2) ^ (r & 7)) << 4) + 4 (lane & 3).
+        const int row_base = 16 * warp;
+
+        // SAD rule (Section 3.4) without a division per token: token tok of the chunk at call
+        // offset cs is a boundary step iff it lies on the grid and phase + (tok mod w) is 0 or w,
+        // with phase = (grid index of the chunk's first token + 1) mod w.
+        const int grid_w = p.grid_w;
+        int pre = 0, phase = 0, phase_step = 0, rmod[4] = {0, 0, 0, 0};
+        {
+            const long long g0 = p.t0 - p.prefix_len;   // grid index of the call's first token (may be < 0)
+            pre = g0 < 0 ? (int)min(-g0, (long long)0x7fffffff) : 0;
+            if (grid_w > 0) {
+                long long ph = (g0 + 1) % grid_w;
+                if (ph < 0) ph += grid_w;
+                phase = (int)ph;
+                phase_step = kC % grid_w;
+#pragma unroll
+                for (int x = 0; x < 4; ++x) rmod[x] = (32 * x + lane) % grid_w;
+            }
+        }
+
+        float st[16];                            // fp32 master state, this thread's 16 values
+#pragma unroll
+        for (int e = 0; e < 16; ++e) st[e] = 0.0f;
+        if (p.state_in) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 a = *reinterpret_cast<const float2*>(p.state_in + unit + (size_t)r0 * kD + c0 + 8 * k);
+                const float2 c = *reinterpret_cast<const float2*>(p.state_in + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k);
+                st[4 * k] = a.x; st[4 * k + 1] = a.y; st[4 * k + 2] = c.x; st[4 * k + 3] = c.y;
+            }
+        }
+        // bf16 copy of diag(mult) state for the Q~ x state MMA: [dk][dv] rows of 128 B, 16-byte
+        // pieces swizzled by the row; this thread writes eight bf16 pairs
+        auto write_state_bf16 = [&](float mult_a, float mult_b) {
+            unsigned char* row0 = sm.sb + r0 * 128 + 4 * (lane & 3);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int piece = ((4 * grp + k) ^ (r0 & 7)) * 16;    // r0 + 8 has the same low bits
+                float a0, a1, b0, b1;
+                mul2(st[4 * k], st[4 * k + 1], mult_a, a0, a1);
+                mul2(st[4 * k + 2], st[4 * k + 3], mult_b, b0, b1);
+                *reinterpret_cast<uint32_t*>(row0 + piece) = pack_bf16(a0, a1);
+                *reinterpret_cast<uint32_t*>(row0 + 8 * 128 + piece) = pack_bf16(b0, b1);
+            }
+        };
+        // S_new = diag(f) S_prev + diag(m) dS, with f = m * m (rows r0 and r0 + 8)
+        auto update_state = [&](float m_a, float m_b) {
+            uint32_t dsv[16];
+            tmem_ld_16x256b_x4(tmem + lane_base + kColDS + 32 * grp, dsv);
+            tmem_wait_ld();
+            const float f_a = m_a * m_a, f_b = m_b * m_b;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                float x0, x1, y0, y1;
+                mul2(st[4 * k], st[4 * k + 1], f_a, x0, x1);
+                mul2(st[4 * k + 2], st[4 * k + 3], f_b, y0, y1);
+                fma2(__uint_as_float(dsv[4 * k]), __uint_as_float(dsv[4 * k + 1]), m_a, x0, x1, st[4 * k], st[4 * k + 1]);
+                fma2(__uint_as_float(dsv[4 * k + 2]), __uint_as_float(dsv[4 * k + 3]), m_b, y0, y1, st[4 * k + 2],
+                     st[4 * k + 3]);
+            }
+        };
+        // this thread's 32 columns of output row i -> bf16 -> row i of the query tile
+        // (the TMEM load is warp-wide; `mine` only gates this thread's row)
+        auto stage_output = [&](float f, bool mine) {
+            unsigned char* orow = sm.q + i * 128;
+            uint32_t ov[32];
+            tmem_ld32(tmem + lane_base + kColO + 32 * grp, ov);
+            tmem_wait_ld();
+            if (!mine) return;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float x0, x1;
+                    mul2(__uint_as_float(ov[8 * c + 2 * e]), __uint_as_float(ov[8 * c + 2 * e + 1]), f, x0, x1);
+                    w[e] = pack_bf16(x0, x1);
+                }
+                reinterpret_cast<uint4*>(orow)[(4 * grp + c) ^ (i & 7)] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        };
+
+        bool ok = true;
+        unsigned it = 0;                // passes so far: phase of the per-pass barriers
+        for (int n = 0; ok && n < n_chunks; ++n) {
+            const int cs = n * kC;
+            const int Lc = min(kC, p.T - cs);
+            // which tokens of the chunk are decaying steps (live and not a row boundary)
+            unsigned mk[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int tok = 32 * x + lane;
+                const int m = phase + rmod[x];
+                const bool boundary = grid_w > 0 && cs + tok >= pre && (m == 0 || m == grid_w);
+                mk[x] = __ballot_sync(0xffffffffu, tok < Lc && !boundary);
+            }
+            phase += phase_step;
+            if (phase >= grid_w) phase -= grid_w;
+            // the 16 rows of this warp's scaling role sit in one mask word
+            const unsigned own_word = (warp >> 1) == 0 ? mk[0] : (warp >> 1) == 1 ? mk[1] : (warp >> 1) == 2 ? mk[2] : mk[3];
+            const unsigned dec16 = (own_word >> (16 * (warp & 1))) & 0xffffu;
+            auto decays = [&](int r) {      // warp-uniform r
+                const unsigned w = (r >> 5) == 0 ? mk[0] : (r >> 5) == 1 ? mk[1] : (r >> 5) == 2 ? mk[2] : mk[3];
+                return ((w >> (r & 31)) & 1u) != 0;
+            };
+
+            // ---- sums of log2 Lambda over this warp's rows, per channel --------------------------
+            if (!(ok = mbar_wait(&sm.bar.full_a, n & 1, limit, abort_flag, p.status))) break;
+            {
+                float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+                for (int rr = 0; rr < 16; ++rr) {
+                    const int r = row_base + rr;
+                    const uint32_t g2 =
+                        *reinterpret_cast<const uint32_t*>(sm.g + r * 128 + (((lane >> 2) ^ (r & 7)) << 4) + 4 * (lane & 3));
+                    if ((dec16 >> rr) & 1u) {
+                        s0 += log2_decay(bf16_lo(g2));
+                        s1 += log2_decay(bf16_hi(g2));
+                    }
+                }
+                *reinterpret_cast<float2*>(&sm.segsum[warp][2 * lane]) = make_float2(s0, s1);
+            }
+            mbar_arrive(&sm.bar.scan);
+            if (!(ok = mbar_wait(&sm.bar.scan, n & 1, limit, abort_flag, p.status))) break;
+
+            // ---- segment length of the chunk (the same value in every warp) ----------------------
+            int len = kC;
+            {
+                float2 bs[8];
+#pragma unroll
+                for (int x = 0; x < 8; ++x) bs[x] = *reinterpret_cast<const float2*>(&sm.segsum[x][2 * lane]);
+                auto span = [&](int x0, int cnt) {      // largest |sum| over blocks x0 .. x0 + cnt - 1, this lane's channels
+                    float a = 0.0f, c = 0.0f;
+#pragma unroll
+                    for (int x = 0; x < 8; ++x)
+                        if (x >= x0 && x < x0 + cnt) { a += bs[x].x; c += bs[x].y; }
+                    return fmaxf(fabsf(a), fabsf(c));
+                };
+                if (warp_max(span(0, 8)) > kSafeRange) {
+                    float a64 = fmaxf(span(0, 4), span(4, 4));
+                    float a32 = fmaxf(fmaxf(span(0, 2), span(2, 2)), fmaxf(span(4, 2), span(6, 2)));
+                    float a16 = 0.0f;
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) a16 = fmaxf(a16, span(x, 1));
+                    a64 = warp_max(a64); a32 = warp_max(a32); a16 = warp_max(a16);
+                    len = a64 <= kSafeRange ? 64 : a32 <= kSafeRange ? 32 : a16 <= kSafeRange ? 16 : 1;
+                }
+            }
+            const int npass = (Lc + len - 1) / len;
+            if (tid == 0) sm.npass = npass;
+
+            if (!(ok = mbar_wait(&sm.bar.full_b, n & 1, limit, abort_flag, p.status))) break;
+
+            for (int ps = 0; ok && ps < npass; ++ps, ++it) {
+                const int lo = ps * len, hi = lo + len;       // rows of this pass
+                const int blk0 = lo >> 4, blk1 = (hi + 15) >> 4;
+                const bool single = len == 1;
+
+                // ---- Q~ and K~ of this pass: rows inside the segment scaled, all others zero ------
+                {
+                    float base0 = 0.0f, base1 = 0.0f, tot0 = 0.0f, tot1 = 0.0f;
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        if (x >= blk0 && x < blk1) {
+                            const float2 bsx = *reinterpret_cast<const float2*>(&sm.segsum[x][2 * lane]);
+                            tot0 += bsx.x; tot1 += bsx.y;
+                            if (x < warp) { base0 += bsx.x; base1 += bsx.y; }
+                        }
+                    }
+                    const bool warp_in = warp >= blk0 && warp < blk1;
+                    float run0 = base0, run1 = base1;
+#pragma unroll 4
+                    for (int rr = 0; rr < 16; ++rr) {
+                        const int r = row_base + rr;
+                        const int off = r * 128 + (((lane >> 2) ^ (r & 7)) << 4) + 4 * (lane & 3);
+                        uint32_t qo = 0u, ko = 0u;
+                        if (warp_in && r >= lo && r < hi && r < Lc) {
+                            const uint32_t g2 = *reinterpret_cast<const uint32_t*>(sm.g + off);
+                            const uint32_t q2 = *reinterpret_cast<const uint32_t*>(sm.q + off);
+                            const float g_lo = bf16_lo(g2), g_hi = bf16_hi(g2);
+                            float l0 = 0.0f, l1 = 0.0f;
+                            if ((dec16 >> rr) & 1u) { l0 = log2_decay(g_lo); l1 = log2_decay(g_hi); }
+                            float k_lo, k_hi;
+                            if (p.tied) {
+                                k_lo = 1.0f - g_lo; k_hi = 1.0f - g_hi;
+                            } else {
+                                const uint32_t k2 = *reinterpret_cast<const uint32_t*>(sm.k + off);
+                                k_lo = bf16_lo(k2); k_hi = bf16_hi(k2);
+                            }
+                            float e0, e1;        // b_i - r
+                            if (single) {
+                                e0 = 0.5f * l0; e1 = 0.5f * l1;
+                            } else {
+                                run0 += l0; run1 += l1;
+                                e0 = run0 - 0.5f * tot0; e1 = run1 - 0.5f * tot1;
+                            }
+                            qo = pack_bf16(bf16_lo(q2) * ex2(e0), bf16_hi(q2) * ex2(e1));
+                            ko = pack_bf16(k_lo * ex2(-e0), k_hi * ex2(-e1));
+                        }
+                        *reinterpret_cast<uint32_t*>(sm.qt + off) = qo;
+                        *reinterpret_cast<uint32_t*>(sm.kt + off) = ko;
+                    }
+                }
+                // ---- per-row factors of the state (rows r0 and r0 + 8 are channels) ---------------
+                float m_a, m_b;          // 2^(b_seg / 2) = 2^r = 2^(b_seg - r)
+                {
+                    float ta = 0.0f, tb = 0.0f;
+                    if (single) {
+                        if (decays(lo)) {
+                            const unsigned char* grow = sm.g + lo * 128;
+                            const int ca = r0, cb = r0 + 8;
+                            ta = log2_decay(__bfloat162float(
+                                *reinterpret_cast<const __nv_bfloat16*>(grow + (((ca >> 3) ^ (lo & 7)) << 4) + 2 * (ca & 7))));
+                            tb = log2_decay(__bfloat162float(
+                                *reinterpret_cast<const __nv_bfloat16*>(grow + (((cb >> 3) ^ (lo & 7)) << 4) + 2 * (cb & 7))));
+                        }
+                    } else {
+#pragma unroll
+                        for (int x = 0; x < 8; ++x) {
+                            if (x >= blk0 && x < blk1) { ta += sm.segsum[x][r0]; tb += sm.segsum[x][r0 + 8]; }
+                        }
+                    }
+                    m_a = ex2(0.5f * ta);
+                    m_b = ex2(0.5f * tb);
+                }
+                write_state_bf16(m_a, m_b);
+                if (ps == npass - 1) mbar_arrive(&sm.bar.gk_free);
+                fence_proxy_async();
+                tc_fence_before();
+                mbar_arrive(&sm.bar.x_ready);
+
+                // ---- E1: A = tril(S) -> bf16 over S's own columns (blocks 2 grp, 2 grp + 1 of this
+                //      thread's row, kept inside this warp's half of S's columns) ---------------------
+                if (!(ok = mbar_wait(&sm.bar.s_done, it & 1, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+#pragma unroll
+                for (int pi = 0; pi < 2; ++pi) {
+                    const int pc = 2 * grp + pi;
+                    uint32_t pk[16];
+                    if (pc <= qd) {
+                        uint32_t sv[32];
+                        tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
+                        tmem_wait_ld();
+                        if (pc < qd) {
+#pragma unroll
+                            for (int c = 0; c < 16; ++c)
+                                pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 16; ++c)
+                                pk[c] = pack_bf16(2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
+                                                  2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                    }
+                    tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(&sm.bar.p_ready);
+
+                // ---- state carry across the segment, in fp32 registers -----------------------------
+                if (!(ok = mbar_wait(&sm.bar.ds_done, it & 1, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+                update_state(m_a, m_b);
+
+                // ---- output rows of the segment -----------------------------------------------------
+                if (!(ok = mbar_wait(&sm.bar.o_done, it & 1, limit, abort_flag, p.status))) break;
+                tc_fence_after();
+                if (32 * qd < hi && 32 * qd + 32 > lo) stage_output(p.scale, i >= lo && i < hi);
+            }
+            if (!ok) break;
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(&sm.bar.st_ready);
+        }
+        if (ok && p.state_out) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                *reinterpret_cast<float2*>(p.state_out + unit + (size_t)r0 * kD + c0 + 8 * k) = make_float2(st[4 * k], st[4 * k + 1]);
+                *reinterpret_cast<float2*>(p.state_out + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k) =
+                    make_float2(st[4 * k + 2], st[4 * k + 3]);
+            }
+        }
+    }
+
+    // ---- teardown ---------------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+}  // namespace
+
+bool prefill_gated_tc_supported(int dk, int dv, bool bf16) { return bf16 && dk == kD && dv == kD; }
+
+cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, cudaStream_t st)
+{
+    CUtensorMap mq, mk, mv, mg, mo;
+    // the gate shares the key's strides; without a key tensor its map stands in for the key's
+    if (!encode_chunk_map(&mq, a.q, a.B, a.T, a.H, a.qs) || !encode_chunk_map(&mg, gate, a.B, a.T, a.H, a.ks) ||
+        !encode_chunk_map(&mk, a.k ? a.k : gate, a.B, a.T, a.H, a.ks) ||
+        !encode_chunk_map(&mv, a.v, a.B, a.T, a.H, a.vs) || !encode_chunk_map(&mo, a.o, a.B, a.T, a.H, a.os))
+        return cudaErrorInvalidValue;
+    GatedParams p;
+    p.B = a.B; p.T = a.T; p.H = a.H;
+    p.grid_w = a.grid_w; p.prefix_len = a.prefix_len; p.t0 = a.t0; p.scale = a.scale;
+    p.tied = a.k ? 0 : 1;
+    p.state_in = a.state_in; p.state_out = a.state_out;
+    p.status = a.status; p.wait_limit = a.wait_limit;
+    const size_t smem = sizeof(Smem) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(prefill_gated_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    prefill_gated_tc_kernel<<<(unsigned)(a.B * a.H), kThreads, smem, st>>>(mq, mk, mv, mg, mo, p);
+    return cudaGetLastError();
+}
+
+}  // namespace lasad

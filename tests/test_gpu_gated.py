@@ -50,6 +50,47 @@ def test_gated_prefill_matches_oracle(ctx, dtype, d, T, w, P):
     assert rel_err(s, s_ref) <= TOL[dtype]
 
 
+@pytest.mark.parametrize("T,w,P", [(1, 4, 0), (100, 7, 0), (128, 16, 0), (257, 16, 1), (700, 24, 0)])
+def test_gated_prefill_both_implementations(ctx, T, w, P):
+    """bf16, d = 64: the tensor-core kernel (default) and the CUDA-core kernel (option 1) against the
+    oracle on the same inputs."""
+    B, H, d = 3, 5, 64
+    q, k, v, lam = _inputs(900 + T, B, T, H, d, torch.bfloat16)
+    s_in = torch.randn(B, H, d, d, generator=torch.Generator().manual_seed(T))
+    o_ref, s_ref = oracle(q, k, v, lam, w, P, 3, 0.25, s_in)
+    for impl in (0, 1):
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, impl)
+        try:
+            o, s = ctx.lasad_forward_gated(*_dev(q, k, v, lam), w, prefix_len=P, t0=3, scale=0.25, state_in=s_in.cuda())
+            torch.cuda.synchronize()
+        finally:
+            ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
+        assert ctx.device_status() == 0
+        assert rel_err(o, o_ref) <= TOL[torch.bfloat16], impl
+        assert rel_err(s, s_ref) <= TOL[torch.bfloat16], impl
+
+
+@pytest.mark.parametrize("level,tied", [(0.35, False), (0.05, False), (0.003, True), (1e-5, False), (0.0, False)])
+def test_gated_tensor_core_path_strong_decay(ctx, level, tied):
+    """Gates so small that a 128-token chunk cannot be scaled around one reference point: the
+    tensor-core kernel cuts such chunks into segments of 64, 32, 16 or single tokens.  The middle
+    chunk of three is the strong one, with exact zeros sprinkled in; the others are ordinary."""
+    B, T, H, d, w = 2, 330, 3, 64, 11
+    q, k, v, lam = _inputs(1200 + int(level * 1e6), B, T, H, d, torch.bfloat16)
+    gen = torch.Generator().manual_seed(5)
+    strong = torch.full((B, 128, H, d), level) * (1.0 + 0.3 * torch.rand(B, 128, H, d, generator=gen))
+    strong = torch.where(torch.rand(B, 128, H, d, generator=gen) < 0.01, torch.zeros_like(strong), strong)
+    lam[:, 128:256] = strong.to(torch.bfloat16)
+    k_used = torch.from_numpy(1.0 - to64(lam)) if tied else k
+    o_ref, s_ref = oracle(q, k_used, v, lam, w)
+    o, s = ctx.lasad_forward_gated(q.cuda(), None if tied else k.cuda(), v.cuda(), lam.cuda(), w)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    assert torch.isfinite(o.float()).all() and torch.isfinite(s).all()
+    assert rel_err(o, o_ref) <= TOL[torch.bfloat16]
+    assert rel_err(s, s_ref) <= TOL[torch.bfloat16]
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_gated_prefill_key_tied_to_gate(ctx, dtype):
     """k = NULL: the key is 1 - lambda (the paper's base decay lambda = 1 - k)."""

@@ -20,6 +20,9 @@ struct lasad_ctx {
     int64_t relay_cap;
     uint64_t epoch;               // launches of the task-streaming prefill so far
     int stream_max_ctas;
+    // per-chain flags of the gated tensor-core prefill: chains it left to the CUDA-core kernel
+    int* d_redo;                  // [redo_cap]
+    int64_t redo_cap;
     // host-buffer pipeline of lasad_forward_host: two staging slots (q | k | v | o of one batch
     // element each), a decay and a state buffer, copy streams and the events that order them
     void* d_stage[2];
@@ -58,6 +61,31 @@ int reserve_units(lasad_ctx* ctx, int64_t units)
         ctx->relay_cap = units;
     } else if (nr) {
         cudaFree(nr);
+    }
+    cudaSetDevice(prev);
+    if (e != cudaSuccess) {
+        ctx->last_cuda_error = (int)e;
+        return LASAD_ERR_CUDA;
+    }
+    return LASAD_OK;
+}
+
+constexpr int64_t kDefaultRedoUnits = 65536;   // chains covered by the flag array lasad_create allocates
+
+// Grows the per-chain flag array of the gated prefill to `units` chains (same rules as above).
+int reserve_redo(lasad_ctx* ctx, int64_t units)
+{
+    if (units <= ctx->redo_cap) return LASAD_OK;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();   // an earlier launch may still use the old array
+    int* nr = nullptr;
+    if (e == cudaSuccess) e = cudaMalloc(&nr, (size_t)units * sizeof(int));
+    if (e == cudaSuccess) {
+        if (ctx->d_redo) cudaFree(ctx->d_redo);
+        ctx->d_redo = nr;
+        ctx->redo_cap = units;
     }
     cudaSetDevice(prev);
     if (e != cudaSuccess) {
@@ -135,9 +163,11 @@ int lasad_create(lasad_ctx** out, int device)
     if (e == cudaSuccess) ctx->stream_max_ctas = lasad::prefill_stream_max_ctas(device);
     cudaSetDevice(prev);
     if (e == cudaSuccess && reserve_units(ctx, kDefaultRelayUnits) != LASAD_OK) e = cudaErrorMemoryAllocation;
+    if (e == cudaSuccess && reserve_redo(ctx, kDefaultRedoUnits) != LASAD_OK) e = cudaErrorMemoryAllocation;
     if (e != cudaSuccess) {
         if (ctx->d_status) cudaFree(ctx->d_status);
         if (ctx->d_relay) cudaFree(ctx->d_relay);
+        if (ctx->d_redo) cudaFree(ctx->d_redo);
         delete ctx;
         return LASAD_ERR_CUDA;
     }
@@ -150,6 +180,7 @@ int lasad_destroy(lasad_ctx* ctx)
     if (!ctx) return LASAD_ERR_INVALID_ARG;
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_relay) cudaFree(ctx->d_relay);
+    if (ctx->d_redo) cudaFree(ctx->d_redo);
     for (int i = 0; i < 2; ++i)
         if (ctx->d_stage[i]) cudaFree(ctx->d_stage[i]);
     if (ctx->d_host_decay) cudaFree(ctx->d_host_decay);
@@ -171,7 +202,8 @@ int lasad_destroy(lasad_ctx* ctx)
 int lasad_reserve(lasad_ctx* ctx, int64_t units)
 {
     if (!ctx || units <= 0) return LASAD_ERR_INVALID_ARG;
-    return reserve_units(ctx, units);
+    const int rc = reserve_units(ctx, units);
+    return rc != LASAD_OK ? rc : reserve_redo(ctx, units);
 }
 
 int lasad_set_option(lasad_ctx* ctx, int option, int value)
@@ -336,8 +368,22 @@ int lasad_forward_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, co
     // tensor cores where the shape allows it, unless the CUDA-core implementation is asked for
     const bool bf16 = p->dtype == LASAD_BF16;
     const bool tc = ctx->opt_prefill_impl != 1 && lasad::prefill_gated_tc_supported(p->dk, p->dv, bf16);
-    const cudaError_t e = tc ? lasad::launch_prefill_gated_tc(a, gate, static_cast<cudaStream_t>(cuda_stream))
-                             : lasad::launch_prefill_gated(a, gate, p->dk, bf16, static_cast<cudaStream_t>(cuda_stream));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (!tc) {
+        const cudaError_t e = lasad::launch_prefill_gated(a, gate, p->dk, bf16, nullptr, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        ctx->launches += 1;
+        return LASAD_OK;
+    }
+    // Two launches: the tensor-core kernel marks the chains whose decay is too strong for its
+    // scaling, and the CUDA-core kernel behind it computes exactly those (none, as a rule).
+    rc = reserve_redo(ctx, (int64_t)p->B * p->H);
+    if (rc != LASAD_OK) return rc;
+    cudaError_t e = lasad::launch_prefill_gated_tc(a, gate, ctx->d_redo, st);
+    if (e == cudaSuccess) {
+        ctx->launches += 1;
+        e = lasad::launch_prefill_gated(a, gate, p->dk, bf16, ctx->d_redo, st);
+    }
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     ctx->launches += 1;
     return LASAD_OK;

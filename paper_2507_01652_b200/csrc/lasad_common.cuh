@@ -64,10 +64,14 @@ cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool d
 // null (key tied to the gate, k = 1 - lambda); a.decay is unused.
 cudaError_t launch_decode_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, bool decay_on, int tpu,
                                 cudaStream_t st);
-cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, cudaStream_t st);
-// Tensor-core form of the gated prefill (bf16, dk = dv = 64).
+// `only` (device, [B*H], or null): compute just the chains whose entry is non-zero.
+cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, const int* only,
+                                 cudaStream_t st);
+// Tensor-core form of the gated prefill (bf16, dk = dv = 64).  It writes redo[chain] = 1 for every
+// chain it gave up (decay too strong for its scaling) and 0 for the others; the caller launches
+// launch_prefill_gated(..., only = redo, ...) behind it.
 bool prefill_gated_tc_supported(int dk, int dv, bool bf16);
-cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, cudaStream_t st);
+cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, int* redo, cudaStream_t st);
 bool prefill_tc_supported(int dk, int dv, bool bf16);
 cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st);
 

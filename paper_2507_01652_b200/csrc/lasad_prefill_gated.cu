@@ -22,8 +22,10 @@ constexpr int kGC = 16;          // chunk length
 constexpr float kMinLog2 = -150.0f;
 
 template <typename T, int D>
-__global__ void __launch_bounds__(256) prefill_gated_kernel(KernelArgs a, const void* gate_v)
+__global__ void __launch_bounds__(256) prefill_gated_kernel(KernelArgs a, const void* gate_v, const int* only)
 {
+    // behind the tensor-core kernel: only the chains it gave up are computed here
+    if (only && only[blockIdx.x] == 0) return;
     constexpr int LD = D + 1;
     __shared__ float Qs[kGC][LD], Ks[kGC][LD], Vs[kGC][LD], Ls[kGC][LD];   // Ls: cumulative log2 decay
     __shared__ float Ws[kGC][LD];        // exp2(L_last - L_j) k_j
@@ -136,20 +138,21 @@ __global__ void __launch_bounds__(256) prefill_gated_kernel(KernelArgs a, const 
 }
 
 template <typename T, int D>
-cudaError_t launch_gated_t(const KernelArgs& a, const void* gate, cudaStream_t st)
+cudaError_t launch_gated_t(const KernelArgs& a, const void* gate, const int* only, cudaStream_t st)
 {
     const size_t smem = sizeof(float) * D * (D + 1);
-    prefill_gated_kernel<T, D><<<(unsigned)(a.B * a.H), 256, smem, st>>>(a, gate);
+    prefill_gated_kernel<T, D><<<(unsigned)(a.B * a.H), 256, smem, st>>>(a, gate, only);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, cudaStream_t st)
+cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, const int* only,
+                                 cudaStream_t st)
 {
     if (dk == 64)
-        return bf16 ? launch_gated_t<__nv_bfloat16, 64>(a, gate, st) : launch_gated_t<float, 64>(a, gate, st);
-    return bf16 ? launch_gated_t<__nv_bfloat16, 32>(a, gate, st) : launch_gated_t<float, 32>(a, gate, st);
+        return bf16 ? launch_gated_t<__nv_bfloat16, 64>(a, gate, only, st) : launch_gated_t<float, 64>(a, gate, only, st);
+    return bf16 ? launch_gated_t<__nv_bfloat16, 32>(a, gate, only, st) : launch_gated_t<float, 32>(a, gate, only, st);
 }
 
 }  // namespace lasad

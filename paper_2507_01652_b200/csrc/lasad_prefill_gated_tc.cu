@@ -23,12 +23,16 @@
 //     O  = A V + Q~ (diag(2^r) S_prev)      (M2b)  tcgen05.mma 128x64x128 (tmem x smem) + 128x64x64
 //     S_new = diag(2^b_N) S_prev + diag(2^(b_N - r)) dS       fp32 registers
 //
-// Every exponent that is formed lies within +-|b_N|/2.  A chunk is taken in one pass while
-// |b_N[c]| <= 200 for all channels (an average decay above 0.34 per step); otherwise it is cut
-// into aligned segments of 64, 32, 16 or, at worst, single tokens (log2 of a decay is clamped at
-// -150, below which the decay is 0 in fp32 anyway), each a pass of the same pipeline over the
-// segment's rows with all other rows of Q~ and K~ zero, so the result stays exact for every gate
-// in [0,1] and only pathological inputs pay for it.
+// Every exponent that is formed lies within +-|b_N|/2.  The kernel takes a chunk this way while
+// |b_N[c]| <= 200 for all channels (an average decay above 0.34 per step, log2 of a decay clamped
+// at -150); a chain with a chunk beyond that is given up at that chunk and marked in a per-chain
+// flag array, and the CUDA-core kernel, launched behind this one on every call, recomputes exactly
+// the marked chains (it forms only differences b_i - b_j <= 0 and is safe for every gate in
+// [0,1]).  A chain that is given up has not written its final state, so state_out may alias
+// state_in.
+//
+// The running sums b are formed once: the first sweep over the gate tile parks them in the
+// 4-byte slots the same thread overwrites in the second sweep, which turns Q and K into Q~, K~.
 //
 // Warp roles: warps 0-7 do the element-wise work.  For the scaling they split the chunk by rows
 // (warp w: rows 16 w ..), lanes across channel pairs, so the running sum b needs no exchange
@@ -59,11 +63,12 @@ constexpr float kMinLog2 = -150.0f;    // log2 of a decay is clamped here (2^-15
 constexpr float kSafeRange = 200.0f;   // largest |sum of log2 decays| one pass may span
 
 struct __align__(8) Barriers {
-    unsigned long long full_a;     // gate (and key) tile of the chunk has landed
-    unsigned long long full_b;     // query and value tiles have landed
+    unsigned long long full_in;    // gate, query (and key) tiles of the chunk have landed
+    unsigned long long full_v;     // value tile has landed
     unsigned long long scan;       // partial sums of the chunk are in shared memory (256 arrivals)
-    unsigned long long gk_free;    // last read of the gate and key tiles of the chunk (256 arrivals)
-    unsigned long long x_ready;    // Q~, K~ and the state copy of a pass are written (256 arrivals)
+    unsigned long long in_free;    // last read of the gate, query and key tiles of the chunk (256 arrivals)
+    unsigned long long stage_free; // the store of the previous output tile has read its staging buffer
+    unsigned long long x_ready;    // Q~, K~ and the state copy are written (256 arrivals)
     unsigned long long s_done;     // M1 complete
     unsigned long long ds_done;    // dS MMAs complete
     unsigned long long p_ready;    // A in TMEM (256 arrivals)
@@ -74,17 +79,16 @@ struct __align__(8) Barriers {
 
 struct Smem {
     // tiles first: each must sit on a 1024-byte boundary (128-byte swizzle atom = 8 rows)
-    unsigned char q[kTileBytes];    // queries; its rows are overwritten by the output rows as they complete
-    unsigned char k[kTileBytes];
+    unsigned char q[kTileBytes];
+    unsigned char k[kTileBytes];    // keys; with the key tied to the gate, a copy of the gate
     unsigned char v[kTileBytes];
-    unsigned char g[kTileBytes];    // gate lambda
-    unsigned char qt[kTileBytes];   // Q~
-    unsigned char kt[kTileBytes];   // K~
+    unsigned char g[kTileBytes];    // gate lambda; after the first sweep the odd channels' running sums
+    unsigned char qt[kTileBytes];   // Q~ (before it is written: the even channels' running sums)
+    unsigned char kt[kTileBytes];   // K~; after the MMAs the staging buffer of the output tile
     unsigned char sb[kD * kD * 2];  // bf16 copy of diag(2^r) state, [dk][dv], 128 B rows, swizzled
     float segsum[8][kD];            // sum of log2 Lambda over rows 16 x .. 16 x + 15, per channel
     Barriers bar;
     uint32_t tmem_base;
-    int npass;                      // passes of the current chunk (written before the first x_ready)
     int abort_flag;
 };
 
@@ -96,6 +100,7 @@ struct GatedParams {
     int tied;                // key tied to the gate: k = 1 - lambda, no key tensor
     const float* state_in;
     float* state_out;
+    int* redo;               // [B*H]: 1 where this kernel gave the chain up (decay too strong), else 0
     int* status;
     unsigned wait_limit;
 };
@@ -139,10 +144,11 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 
     // ---- set-up ---------------------------------------------------------------------------
     if (tid == 0) {
-        mbar_init(&sm.bar.full_a, 1);
-        mbar_init(&sm.bar.full_b, 1);
+        mbar_init(&sm.bar.full_in, 1);
+        mbar_init(&sm.bar.full_v, 1);
         mbar_init(&sm.bar.scan, kEThreads);
-        mbar_init(&sm.bar.gk_free, kEThreads);
+        mbar_init(&sm.bar.in_free, kEThreads);
+        mbar_init(&sm.bar.stage_free, 1);
         mbar_init(&sm.bar.x_ready, kEThreads);
         mbar_init(&sm.bar.s_done, 1);
         mbar_init(&sm.bar.ds_done, 1);
@@ -151,7 +157,6 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         mbar_init(&sm.bar.st_ready, kEThreads);
         mbar_init(&sm.bar.drain, 1);
         sm.abort_flag = 0;
-        sm.npass = 1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 8) {
@@ -168,55 +173,47 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     if (warp == 9) {
         // ===================== TMA warp ========================================================
         // One set of tiles; each is refilled for the next chunk as soon as its last reader is done:
-        // gate and key after the chunk's last scaling pass, value after the last MMA, query (whose
-        // tile carries the output rows) after the store has read it.
+        // gate, query and key once the chunk's scaled operands are written, value once the chunk's
+        // MMAs have retired.  The output tile leaves from the K~ buffer.
         if (elect_one()) {
-            const unsigned a_bytes = (p.tied ? 1 : 2) * kTileBytes;
-            auto issue_a = [&](int n) {
-                mbar_arrive_expect_tx(&sm.bar.full_a, a_bytes);
-                tma_load_4d(sm.g, &tm_g, &sm.bar.full_a, 0, h, n * kC, b);
-                if (!p.tied) tma_load_4d(sm.k, &tm_k, &sm.bar.full_a, 0, h, n * kC, b);
+            const unsigned in_bytes = (p.tied ? 2 : 3) * kTileBytes;
+            auto issue_in = [&](int n) {
+                mbar_arrive_expect_tx(&sm.bar.full_in, in_bytes);
+                tma_load_4d(sm.g, &tm_g, &sm.bar.full_in, 0, h, n * kC, b);
+                tma_load_4d(sm.q, &tm_q, &sm.bar.full_in, 0, h, n * kC, b);
+                if (!p.tied) tma_load_4d(sm.k, &tm_k, &sm.bar.full_in, 0, h, n * kC, b);
             };
             auto issue_v = [&](int n) {
-                mbar_arrive_expect_tx(&sm.bar.full_b, 2 * kTileBytes);
-                tma_load_4d(sm.v, &tm_v, &sm.bar.full_b, 0, h, n * kC, b);
+                mbar_arrive_expect_tx(&sm.bar.full_v, kTileBytes);
+                tma_load_4d(sm.v, &tm_v, &sm.bar.full_v, 0, h, n * kC, b);
             };
-            auto issue_q = [&](int n) { tma_load_4d(sm.q, &tm_q, &sm.bar.full_b, 0, h, n * kC, b); };
-            int a_issued = 0, b_issued = 0;     // chunks whose loads have been issued (b: both tiles)
-            if (n_chunks > 0) {
-                issue_a(0);
-                issue_v(0);
-                issue_q(0);
-                a_issued = b_issued = 1;
-            }
+            issue_in(0);
+            issue_v(0);
+            int in_issued = 1, v_issued = 1;     // chunks whose loads have been issued
             for (int n = 0; n < n_chunks; ++n) {
                 const bool more = n + 1 < n_chunks;
                 if (more) {
-                    if (!mbar_wait(&sm.bar.gk_free, n & 1, limit, abort_flag, p.status)) break;
-                    issue_a(n + 1);
-                    a_issued = n + 2;
+                    if (!mbar_wait(&sm.bar.in_free, n & 1, limit, abort_flag, p.status)) break;
+                    issue_in(n + 1);
+                    in_issued = n + 2;
+                    if (!mbar_wait(&sm.bar.o_done, n & 1, limit, abort_flag, p.status)) break;
+                    issue_v(n + 1);
+                    v_issued = n + 2;
                 }
-                const bool staged = mbar_wait(&sm.bar.st_ready, n & 1, limit, abort_flag, p.status);
-                if (more) issue_v(n + 1);       // (also after a failed wait: the barrier's byte count must complete)
-                if (staged) {
-                    tma_store_4d(&tm_o, sm.q, 0, h, n * kC, b);
-                    tma_store_commit();
-                    if (more) tma_store_wait_read();
-                }
+                if (!mbar_wait(&sm.bar.st_ready, n & 1, limit, abort_flag, p.status)) break;
+                tma_store_4d(&tm_o, sm.kt, 0, h, n * kC, b);
+                tma_store_commit();
                 if (more) {
-                    issue_q(n + 1);
-                    b_issued = n + 2;
+                    tma_store_wait_read();        // the store has finished reading the buffer
+                    mbar_arrive(&sm.bar.stage_free);
                 }
-                if (!staged) break;
             }
             tma_store_wait_all();
             // leave only when every issued load has landed (they write this CTA's shared memory)
-            if (a_issued > 0)
-                for (unsigned it = 0; it < kTeardownLimit; ++it)
-                    if (mbar_try_wait(&sm.bar.full_a, (a_issued - 1) & 1)) break;
-            if (b_issued > 0)
-                for (unsigned it = 0; it < kTeardownLimit; ++it)
-                    if (mbar_try_wait(&sm.bar.full_b, (b_issued - 1) & 1)) break;
+            for (unsigned it = 0; it < kTeardownLimit; ++it)
+                if (mbar_try_wait(&sm.bar.full_in, (in_issued - 1) & 1)) break;
+            for (unsigned it = 0; it < kTeardownLimit; ++it)
+                if (mbar_try_wait(&sm.bar.full_v, (v_issued - 1) & 1)) break;
         }
         __syncwarp();
     } else if (warp == 8) {
@@ -229,45 +226,40 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         const uint64_t d_q = make_desc(smem_u32(sm.qt));
         const uint64_t d_k = make_desc(smem_u32(sm.kt));
         const uint64_t d_v = make_desc(smem_u32(sm.v));
-        bool ok = true;
-        unsigned it = 0;                // passes so far: phase of the per-pass barriers
-        for (int n = 0; ok && n < n_chunks; ++n) {
-            int np = 1;
-            for (int ps = 0; ok && ps < np; ++ps, ++it) {
-                if (!mbar_wait(&sm.bar.x_ready, it & 1, limit, abort_flag, p.status)) { ok = false; break; }
-                if (ps == 0) {
-                    np = *reinterpret_cast<volatile int*>(&sm.npass);
-                    // the value tile was written by the TMA unit: observe its barrier here as well
-                    if (!mbar_wait(&sm.bar.full_b, n & 1, limit, abort_flag, p.status)) { ok = false; break; }
-                }
-                tc_fence_after();
-                if (elect_one()) {
+        for (int n = 0; n < n_chunks; ++n) {
+            if (!mbar_wait(&sm.bar.x_ready, n & 1, limit, abort_flag, p.status)) break;
+            tc_fence_after();
+            if (elect_one()) {
 #pragma unroll
-                    for (int kk = 0; kk < kD / 16; ++kk)  // 32 bytes along K per step
-                        mma_ss(tmem + kColS, d_q + 2 * kk, d_k + 2 * kk, idesc_s, kk > 0);
-                    mma_commit(&sm.bar.s_done);
+                for (int kk = 0; kk < kD / 16; ++kk)  // 32 bytes along K per step
+                    mma_ss(tmem + kColS, d_q + 2 * kk, d_k + 2 * kk, idesc_s, kk > 0);
+                mma_commit(&sm.bar.s_done);
+                // the state's contribution opens the O accumulator; A V is added once A is ready
 #pragma unroll
-                    for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K~ and of V per step
-                        mma_ss(tmem + kColDS, d_k + 128 * kk, d_v + 128 * kk, idesc_kv, kk > 0);
-                    mma_commit(&sm.bar.ds_done);
-                    // the state's contribution opens the O accumulator; A V is added once A is ready
-#pragma unroll
-                    for (int kk = 0; kk < kD / 16; ++kk)
-                        mma_ss(tmem + kColO, d_q + 2 * kk, d_sb + 128 * kk, idesc_qs, kk > 0);
-                }
-                __syncwarp();
-                if (!mbar_wait(&sm.bar.p_ready, it & 1, limit, abort_flag, p.status)) { ok = false; break; }
-                tc_fence_after();
-                if (elect_one()) {
-#pragma unroll
-                    for (int kk = 0; kk < kC / 16; ++kk)  // A: 8 TMEM columns per step (tokens 0..63 at columns
-                                                          // 0..31, tokens 64..127 at 64..95); V: 2048 B per step
-                        mma_ts(tmem + kColO, tmem + kColS + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), d_v + 128 * kk,
-                               idesc_pv, 1);
-                    mma_commit(&sm.bar.o_done);
-                }
-                __syncwarp();
+                for (int kk = 0; kk < kD / 16; ++kk)
+                    mma_ss(tmem + kColO, d_q + 2 * kk, d_sb + 128 * kk, idesc_qs, kk > 0);
             }
+            __syncwarp();
+            if (!mbar_wait(&sm.bar.full_v, n & 1, limit, abort_flag, p.status)) break;
+            tc_fence_after();
+            if (elect_one()) {
+#pragma unroll
+                for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K~ and of V per step
+                    mma_ss(tmem + kColDS, d_k + 128 * kk, d_v + 128 * kk, idesc_kv, kk > 0);
+                mma_commit(&sm.bar.ds_done);
+            }
+            __syncwarp();
+            if (!mbar_wait(&sm.bar.p_ready, n & 1, limit, abort_flag, p.status)) break;
+            tc_fence_after();
+            if (elect_one()) {
+#pragma unroll
+                for (int kk = 0; kk < kC / 16; ++kk)  // A: 8 TMEM columns per step (tokens 0..63 at columns
+                                                      // 0..31, tokens 64..127 at 64..95); V: 2048 B per step
+                    mma_ts(tmem + kColO, tmem + kColS + (kk < 4 ? 8 * kk : 64 + 8 * (kk - 4)), d_v + 128 * kk,
+                           idesc_pv, 1);
+                mma_commit(&sm.bar.o_done);
+            }
+            __syncwarp();
         }
         // make sure nothing is still running on the tensor pipe before TMEM is freed
         if (elect_one()) {
@@ -289,8 +281,10 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         const int c0 = 32 * grp + 2 * (lane & 3);
         const size_t unit = (size_t)blockIdx.x * kD * kD;
         // Scaling role: rows 16 warp .. 16 warp + 15, channels 2 lane and 2 lane + 1.  Byte offset
-        // of that channel pair in row r of a tile: r * 128 + (((lane >> 2) ^ (r & 7)) << 4) + 4 (lane & 3).
-        const int row_base = 16 * warp;
+        // of that channel pair in row 16 warp + rr of a tile (rows of 128 B, 16-byte pieces
+        // swizzled by the row): scale_off + rr * 128 + (((lane >> 2) ^ (rr & 7)) << 4).
+        const int scale_off = 16 * warp * 128 + 4 * (lane & 3);
+        const int lane_piece = lane >> 2;
 
         // SAD rule (Section 3.4) without a division per token: token tok of the chunk at call
         // offset cs is a boundary step iff it lies on the grid and phase + (tok mod w) is 0 or w,
@@ -351,14 +345,12 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                      st[4 * k + 3]);
             }
         };
-        // this thread's 32 columns of output row i -> bf16 -> row i of the query tile
-        // (the TMEM load is warp-wide; `mine` only gates this thread's row)
-        auto stage_output = [&](float f, bool mine) {
-            unsigned char* orow = sm.q + i * 128;
+        // this thread's 32 columns of output row i -> bf16 -> row i of the staging buffer
+        auto stage_output = [&](float f) {
+            unsigned char* orow = sm.kt + i * 128;
             uint32_t ov[32];
             tmem_ld32(tmem + lane_base + kColO + 32 * grp, ov);
             tmem_wait_ld();
-            if (!mine) return;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t w[4];
@@ -372,203 +364,151 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             }
         };
 
-        bool ok = true;
-        unsigned it = 0;                // passes so far: phase of the per-pass barriers
+        bool ok = true, given_up = false;
         for (int n = 0; ok && n < n_chunks; ++n) {
             const int cs = n * kC;
             const int Lc = min(kC, p.T - cs);
-            // which tokens of the chunk are decaying steps (live and not a row boundary)
-            unsigned mk[4];
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const int tok = 32 * x + lane;
-                const int m = phase + rmod[x];
-                const bool boundary = grid_w > 0 && cs + tok >= pre && (m == 0 || m == grid_w);
-                mk[x] = __ballot_sync(0xffffffffu, tok < Lc && !boundary);
-            }
-            phase += phase_step;
-            if (phase >= grid_w) phase -= grid_w;
-            // the 16 rows of this warp's scaling role sit in one mask word
-            const unsigned own_word = (warp >> 1) == 0 ? mk[0] : (warp >> 1) == 1 ? mk[1] : (warp >> 1) == 2 ? mk[2] : mk[3];
-            const unsigned dec16 = (own_word >> (16 * (warp & 1))) & 0xffffu;
-            auto decays = [&](int r) {      // warp-uniform r
-                const unsigned w = (r >> 5) == 0 ? mk[0] : (r >> 5) == 1 ? mk[1] : (r >> 5) == 2 ? mk[2] : mk[3];
-                return ((w >> (r & 31)) & 1u) != 0;
-            };
-
-            // ---- sums of log2 Lambda over this warp's rows, per channel --------------------------
-            if (!(ok = mbar_wait(&sm.bar.full_a, n & 1, limit, abort_flag, p.status))) break;
+            // which of this warp's 16 rows are decaying steps (live and not a row boundary)
+            unsigned dec16;
             {
-                float s0 = 0.0f, s1 = 0.0f;
+                unsigned mk[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    const int tok = 32 * x + lane;
+                    const int m = phase + rmod[x];
+                    const bool boundary = grid_w > 0 && cs + tok >= pre && (m == 0 || m == grid_w);
+                    mk[x] = __ballot_sync(0xffffffffu, tok < Lc && !boundary);
+                }
+                phase += phase_step;
+                if (phase >= grid_w) phase -= grid_w;
+                const int wx = warp >> 1;
+                const unsigned own_word = wx == 0 ? mk[0] : wx == 1 ? mk[1] : wx == 2 ? mk[2] : mk[3];
+                dec16 = (own_word >> (16 * (warp & 1))) & 0xffffu;
+            }
+
+            // ---- first sweep: running sums of log2 Lambda down this warp's rows.  They are parked
+            //      in the slots this thread will overwrite in the second sweep (even channel: Q~'s,
+            //      odd channel: the gate's own), so nothing is computed twice.
+            if (!(ok = mbar_wait(&sm.bar.full_in, n & 1, limit, abort_flag, p.status))) break;
+            {
+                float run0 = 0.0f, run1 = 0.0f;
 #pragma unroll
                 for (int rr = 0; rr < 16; ++rr) {
-                    const int r = row_base + rr;
-                    const uint32_t g2 =
-                        *reinterpret_cast<const uint32_t*>(sm.g + r * 128 + (((lane >> 2) ^ (r & 7)) << 4) + 4 * (lane & 3));
+                    const int off = scale_off + rr * 128 + ((lane_piece ^ (rr & 7)) << 4);
+                    const uint32_t g2 = *reinterpret_cast<const uint32_t*>(sm.g + off);
                     if ((dec16 >> rr) & 1u) {
-                        s0 += log2_decay(bf16_lo(g2));
-                        s1 += log2_decay(bf16_hi(g2));
+                        run0 += log2_decay(bf16_lo(g2));
+                        run1 += log2_decay(bf16_hi(g2));
                     }
+                    *reinterpret_cast<float*>(sm.qt + off) = run0;
+                    *reinterpret_cast<float*>(sm.g + off) = run1;
+                    if (p.tied) *reinterpret_cast<uint32_t*>(sm.k + off) = g2;
                 }
-                *reinterpret_cast<float2*>(&sm.segsum[warp][2 * lane]) = make_float2(s0, s1);
+                *reinterpret_cast<float2*>(&sm.segsum[warp][2 * lane]) = make_float2(run0, run1);
             }
             mbar_arrive(&sm.bar.scan);
             if (!(ok = mbar_wait(&sm.bar.scan, n & 1, limit, abort_flag, p.status))) break;
 
-            // ---- segment length of the chunk (the same value in every warp) ----------------------
-            int len = kC;
+            // ---- this warp's offset into the chunk, the chunk's total, the range check ------------
+            float h0, h1;       // (sum over the warps before this one) - r, so that b_i - r = running sum + h
             {
-                float2 bs[8];
+                float base0 = 0.0f, base1 = 0.0f, tot0 = 0.0f, tot1 = 0.0f;
 #pragma unroll
-                for (int x = 0; x < 8; ++x) bs[x] = *reinterpret_cast<const float2*>(&sm.segsum[x][2 * lane]);
-                auto span = [&](int x0, int cnt) {      // largest |sum| over blocks x0 .. x0 + cnt - 1, this lane's channels
-                    float a = 0.0f, c = 0.0f;
-#pragma unroll
-                    for (int x = 0; x < 8; ++x)
-                        if (x >= x0 && x < x0 + cnt) { a += bs[x].x; c += bs[x].y; }
-                    return fmaxf(fabsf(a), fabsf(c));
-                };
-                if (warp_max(span(0, 8)) > kSafeRange) {
-                    float a64 = fmaxf(span(0, 4), span(4, 4));
-                    float a32 = fmaxf(fmaxf(span(0, 2), span(2, 2)), fmaxf(span(4, 2), span(6, 2)));
-                    float a16 = 0.0f;
-#pragma unroll
-                    for (int x = 0; x < 8; ++x) a16 = fmaxf(a16, span(x, 1));
-                    a64 = warp_max(a64); a32 = warp_max(a32); a16 = warp_max(a16);
-                    len = a64 <= kSafeRange ? 64 : a32 <= kSafeRange ? 32 : a16 <= kSafeRange ? 16 : 1;
+                for (int x = 0; x < 8; ++x) {
+                    const float2 bsx = *reinterpret_cast<const float2*>(&sm.segsum[x][2 * lane]);
+                    tot0 += bsx.x; tot1 += bsx.y;
+                    if (x < warp) { base0 += bsx.x; base1 += bsx.y; }
+                }
+                h0 = base0 - 0.5f * tot0;
+                h1 = base1 - 0.5f * tot1;
+                if (warp_max(fmaxf(-tot0, -tot1)) > kSafeRange) {
+                    // decay too strong to scale a whole chunk around one reference: leave the chain
+                    // to the CUDA-core kernel (every warp takes the same decision)
+                    given_up = true;
+                    if (tid == 0) *abort_flag = 1;
+                    break;
                 }
             }
-            const int npass = (Lc + len - 1) / len;
-            if (tid == 0) sm.npass = npass;
-
-            if (!(ok = mbar_wait(&sm.bar.full_b, n & 1, limit, abort_flag, p.status))) break;
-
-            for (int ps = 0; ok && ps < npass; ++ps, ++it) {
-                const int lo = ps * len, hi = lo + len;       // rows of this pass
-                const int blk0 = lo >> 4, blk1 = (hi + 15) >> 4;
-                const bool single = len == 1;
-
-                // ---- Q~ and K~ of this pass: rows inside the segment scaled, all others zero ------
-                {
-                    float base0 = 0.0f, base1 = 0.0f, tot0 = 0.0f, tot1 = 0.0f;
+            // per-row factors of the state (rows r0 and r0 + 8 are channels): 2^(b_N / 2) = 2^r = 2^(b_N - r)
+            float m_a, m_b;
+            {
+                float ta = 0.0f, tb = 0.0f;
 #pragma unroll
-                    for (int x = 0; x < 8; ++x) {
-                        if (x >= blk0 && x < blk1) {
-                            const float2 bsx = *reinterpret_cast<const float2*>(&sm.segsum[x][2 * lane]);
-                            tot0 += bsx.x; tot1 += bsx.y;
-                            if (x < warp) { base0 += bsx.x; base1 += bsx.y; }
-                        }
-                    }
-                    const bool warp_in = warp >= blk0 && warp < blk1;
-                    float run0 = base0, run1 = base1;
-#pragma unroll 4
-                    for (int rr = 0; rr < 16; ++rr) {
-                        const int r = row_base + rr;
-                        const int off = r * 128 + (((lane >> 2) ^ (r & 7)) << 4) + 4 * (lane & 3);
-                        uint32_t qo = 0u, ko = 0u;
-                        if (warp_in && r >= lo && r < hi && r < Lc) {
-                            const uint32_t g2 = *reinterpret_cast<const uint32_t*>(sm.g + off);
-                            const uint32_t q2 = *reinterpret_cast<const uint32_t*>(sm.q + off);
-                            const float g_lo = bf16_lo(g2), g_hi = bf16_hi(g2);
-                            float l0 = 0.0f, l1 = 0.0f;
-                            if ((dec16 >> rr) & 1u) { l0 = log2_decay(g_lo); l1 = log2_decay(g_hi); }
-                            float k_lo, k_hi;
-                            if (p.tied) {
-                                k_lo = 1.0f - g_lo; k_hi = 1.0f - g_hi;
-                            } else {
-                                const uint32_t k2 = *reinterpret_cast<const uint32_t*>(sm.k + off);
-                                k_lo = bf16_lo(k2); k_hi = bf16_hi(k2);
-                            }
-                            float e0, e1;        // b_i - r
-                            if (single) {
-                                e0 = 0.5f * l0; e1 = 0.5f * l1;
-                            } else {
-                                run0 += l0; run1 += l1;
-                                e0 = run0 - 0.5f * tot0; e1 = run1 - 0.5f * tot1;
-                            }
-                            qo = pack_bf16(bf16_lo(q2) * ex2(e0), bf16_hi(q2) * ex2(e1));
-                            ko = pack_bf16(k_lo * ex2(-e0), k_hi * ex2(-e1));
-                        }
-                        *reinterpret_cast<uint32_t*>(sm.qt + off) = qo;
-                        *reinterpret_cast<uint32_t*>(sm.kt + off) = ko;
-                    }
-                }
-                // ---- per-row factors of the state (rows r0 and r0 + 8 are channels) ---------------
-                float m_a, m_b;          // 2^(b_seg / 2) = 2^r = 2^(b_seg - r)
-                {
-                    float ta = 0.0f, tb = 0.0f;
-                    if (single) {
-                        if (decays(lo)) {
-                            const unsigned char* grow = sm.g + lo * 128;
-                            const int ca = r0, cb = r0 + 8;
-                            ta = log2_decay(__bfloat162float(
-                                *reinterpret_cast<const __nv_bfloat16*>(grow + (((ca >> 3) ^ (lo & 7)) << 4) + 2 * (ca & 7))));
-                            tb = log2_decay(__bfloat162float(
-                                *reinterpret_cast<const __nv_bfloat16*>(grow + (((cb >> 3) ^ (lo & 7)) << 4) + 2 * (cb & 7))));
-                        }
-                    } else {
-#pragma unroll
-                        for (int x = 0; x < 8; ++x) {
-                            if (x >= blk0 && x < blk1) { ta += sm.segsum[x][r0]; tb += sm.segsum[x][r0 + 8]; }
-                        }
-                    }
-                    m_a = ex2(0.5f * ta);
-                    m_b = ex2(0.5f * tb);
-                }
-                write_state_bf16(m_a, m_b);
-                if (ps == npass - 1) mbar_arrive(&sm.bar.gk_free);
-                fence_proxy_async();
-                tc_fence_before();
-                mbar_arrive(&sm.bar.x_ready);
-
-                // ---- E1: A = tril(S) -> bf16 over S's own columns (blocks 2 grp, 2 grp + 1 of this
-                //      thread's row, kept inside this warp's half of S's columns) ---------------------
-                if (!(ok = mbar_wait(&sm.bar.s_done, it & 1, limit, abort_flag, p.status))) break;
-                tc_fence_after();
-#pragma unroll
-                for (int pi = 0; pi < 2; ++pi) {
-                    const int pc = 2 * grp + pi;
-                    uint32_t pk[16];
-                    if (pc <= qd) {
-                        uint32_t sv[32];
-                        tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
-                        tmem_wait_ld();
-                        if (pc < qd) {
-#pragma unroll
-                            for (int c = 0; c < 16; ++c)
-                                pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < 16; ++c)
-                                pk[c] = pack_bf16(2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
-                                                  2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
-                        }
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) pk[c] = 0u;
-                    }
-                    tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
-                }
-                tmem_wait_st();
-                tc_fence_before();
-                mbar_arrive(&sm.bar.p_ready);
-
-                // ---- state carry across the segment, in fp32 registers -----------------------------
-                if (!(ok = mbar_wait(&sm.bar.ds_done, it & 1, limit, abort_flag, p.status))) break;
-                tc_fence_after();
-                update_state(m_a, m_b);
-
-                // ---- output rows of the segment -----------------------------------------------------
-                if (!(ok = mbar_wait(&sm.bar.o_done, it & 1, limit, abort_flag, p.status))) break;
-                tc_fence_after();
-                if (32 * qd < hi && 32 * qd + 32 > lo) stage_output(p.scale, i >= lo && i < hi);
+                for (int x = 0; x < 8; ++x) { ta += sm.segsum[x][r0]; tb += sm.segsum[x][r0 + 8]; }
+                m_a = ex2(0.5f * ta);
+                m_b = ex2(0.5f * tb);
             }
-            if (!ok) break;
+
+            // ---- second sweep: Q~ = Q o 2^(b - r), K~ = K o 2^(r - b) ------------------------------
+            if (n > 0 && !(ok = mbar_wait(&sm.bar.stage_free, (n - 1) & 1, limit, abort_flag, p.status))) break;
+#pragma unroll
+            for (int rr = 0; rr < 16; ++rr) {
+                const int off = scale_off + rr * 128 + ((lane_piece ^ (rr & 7)) << 4);
+                const float e0 = *reinterpret_cast<const float*>(sm.qt + off) + h0;
+                const float e1 = *reinterpret_cast<const float*>(sm.g + off) + h1;
+                const uint32_t q2 = *reinterpret_cast<const uint32_t*>(sm.q + off);
+                const uint32_t k2 = *reinterpret_cast<const uint32_t*>(sm.k + off);
+                float k_lo = bf16_lo(k2), k_hi = bf16_hi(k2);
+                if (p.tied) { k_lo = 1.0f - k_lo; k_hi = 1.0f - k_hi; }
+                const bool live = 16 * warp + rr < Lc;      // rows past the end of the sequence contribute nothing
+                const uint32_t qo = pack_bf16(bf16_lo(q2) * ex2(e0), bf16_hi(q2) * ex2(e1));
+                const uint32_t ko = pack_bf16(k_lo * ex2(-e0), k_hi * ex2(-e1));
+                *reinterpret_cast<uint32_t*>(sm.qt + off) = live ? qo : 0u;
+                *reinterpret_cast<uint32_t*>(sm.kt + off) = live ? ko : 0u;
+            }
+            write_state_bf16(m_a, m_b);
+            mbar_arrive(&sm.bar.in_free);
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(&sm.bar.x_ready);
+
+            // ---- E1: A = tril(S) -> bf16 over S's own columns (blocks 2 grp, 2 grp + 1 of this
+            //      thread's row, kept inside this warp's half of S's columns) -------------------------
+            if (!(ok = mbar_wait(&sm.bar.s_done, n & 1, limit, abort_flag, p.status))) break;
+            tc_fence_after();
+#pragma unroll
+            for (int pi = 0; pi < 2; ++pi) {
+                const int pc = 2 * grp + pi;
+                uint32_t pk[16];
+                if (pc <= qd) {
+                    uint32_t sv[32];
+                    tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
+                    tmem_wait_ld();
+                    if (pc < qd) {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c)
+                            pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; ++c)
+                            pk[c] = pack_bf16(2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
+                                              2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                }
+                tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&sm.bar.p_ready);
+
+            // ---- state carry across the chunk, in fp32 registers -----------------------------------
+            if (!(ok = mbar_wait(&sm.bar.ds_done, n & 1, limit, abort_flag, p.status))) break;
+            tc_fence_after();
+            update_state(m_a, m_b);
+
+            // ---- output tile -------------------------------------------------------------------------
+            if (!(ok = mbar_wait(&sm.bar.o_done, n & 1, limit, abort_flag, p.status))) break;
+            tc_fence_after();
+            stage_output(p.scale);
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(&sm.bar.st_ready);
         }
-        if (ok && p.state_out) {
+        if (tid == 0) p.redo[blockIdx.x] = given_up ? 1 : 0;
+        if (ok && !given_up && p.state_out) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 *reinterpret_cast<float2*>(p.state_out + unit + (size_t)r0 * kD + c0 + 8 * k) = make_float2(st[4 * k], st[4 * k + 1]);
@@ -592,7 +532,7 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 
 bool prefill_gated_tc_supported(int dk, int dv, bool bf16) { return bf16 && dk == kD && dv == kD; }
 
-cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, cudaStream_t st)
+cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, int* redo, cudaStream_t st)
 {
     CUtensorMap mq, mk, mv, mg, mo;
     // the gate shares the key's strides; without a key tensor its map stands in for the key's
@@ -605,6 +545,7 @@ cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, cudaS
     p.grid_w = a.grid_w; p.prefix_len = a.prefix_len; p.t0 = a.t0; p.scale = a.scale;
     p.tied = a.k ? 0 : 1;
     p.state_in = a.state_in; p.state_out = a.state_out;
+    p.redo = redo;
     p.status = a.status; p.wait_limit = a.wait_limit;
     const size_t smem = sizeof(Smem) + 1024;
     cudaError_t e = cudaFuncSetAttribute(prefill_gated_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

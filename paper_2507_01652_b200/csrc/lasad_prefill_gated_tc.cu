@@ -24,15 +24,17 @@
 //     S_new = diag(2^b_N) S_prev + diag(2^(b_N - r)) dS       fp32 registers
 //
 // Every exponent that is formed lies within +-|b_N|/2.  The kernel takes a chunk this way while
-// |b_N[c]| <= 200 for all channels (an average decay above 0.34 per step, log2 of a decay clamped
-// at -150); a chain with a chunk beyond that is given up at that chunk and marked in a per-chain
+// |b_N[c]| <= 200 for all channels (an average decay above 0.34 per step; gates at or below 0
+// count as decay 0); a chain with a chunk beyond that is given up at that chunk and marked in a per-chain
 // flag array, and the CUDA-core kernel, launched behind this one on every call, recomputes exactly
 // the marked chains (it forms only differences b_i - b_j <= 0 and is safe for every gate in
 // [0,1]).  A chain that is given up has not written its final state, so state_out may alias
 // state_in.
 //
-// The running sums b are formed once: the first sweep over the gate tile parks them in the
-// 4-byte slots the same thread overwrites in the second sweep, which turns Q and K into Q~, K~.
+// No exponential or logarithm is taken per element: within a warp's 16 rows the factor 2^(b_i - r)
+// is carried forward as a running product of the gates themselves and 2^(r - b_j) backward from
+// the warp's last row; log2 and exp2 only appear for the eight partial products per channel that
+// cross warps.
 //
 // Warp roles: warps 0-7 do the element-wise work.  For the scaling they split the chunk by rows
 // (warp w: rows 16 w ..), lanes across channel pairs, so the running sum b needs no exchange
@@ -59,7 +61,6 @@ constexpr uint32_t kColS = 0;      // S (fp32, 128 columns); A (bf16 pairs) alia
 constexpr uint32_t kColO = 128;    // O accumulator, 64 columns
 constexpr uint32_t kColDS = 192;   // dS accumulator (M = 64 layout), 64 columns
 constexpr unsigned kTeardownLimit = 1u << 26;
-constexpr float kMinLog2 = -150.0f;    // log2 of a decay is clamped here (2^-150 is 0 in fp32)
 constexpr float kSafeRange = 200.0f;   // largest |sum of log2 decays| one pass may span
 
 struct __align__(8) Barriers {
@@ -80,13 +81,13 @@ struct __align__(8) Barriers {
 struct Smem {
     // tiles first: each must sit on a 1024-byte boundary (128-byte swizzle atom = 8 rows)
     unsigned char q[kTileBytes];
-    unsigned char k[kTileBytes];    // keys; with the key tied to the gate, a copy of the gate
+    unsigned char k[kTileBytes];    // keys (unused when the key is tied to the gate)
     unsigned char v[kTileBytes];
-    unsigned char g[kTileBytes];    // gate lambda; after the first sweep the odd channels' running sums
-    unsigned char qt[kTileBytes];   // Q~ (before it is written: the even channels' running sums)
+    unsigned char g[kTileBytes];    // gate lambda
+    unsigned char qt[kTileBytes];   // Q~
     unsigned char kt[kTileBytes];   // K~; after the MMAs the staging buffer of the output tile
     unsigned char sb[kD * kD * 2];  // bf16 copy of diag(2^r) state, [dk][dv], 128 B rows, swizzled
-    float segsum[8][kD];            // sum of log2 Lambda over rows 16 x .. 16 x + 15, per channel
+    float segsum[8][kD];            // log2 of the product of Lambda over rows 16 x .. 16 x + 15, per channel
     Barriers bar;
     uint32_t tmem_base;
     int abort_flag;
@@ -117,14 +118,13 @@ __device__ __forceinline__ float lg2(float x)
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// log2 of a gate value under the clamp; 0 and negative values count as decay 0
-__device__ __forceinline__ float log2_decay(float g) { return fmaxf(lg2(fmaxf(g, 0.0f)), kMinLog2); }
 
-__device__ __forceinline__ float warp_max(float v)
+// packed bf16 multiply, round to nearest
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b)
 {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
+    uint32_t r;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
 }
 
 __global__ void __launch_bounds__(kThreads, 2)
@@ -285,6 +285,7 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         // swizzled by the row): scale_off + rr * 128 + (((lane >> 2) ^ (rr & 7)) << 4).
         const int scale_off = 16 * warp * 128 + 4 * (lane & 3);
         const int lane_piece = lane >> 2;
+        auto row_off = [&](int rr) { return scale_off + rr * 128 + ((lane_piece ^ (rr & 7)) << 4); };
 
         // SAD rule (Section 3.4) without a division per token: token tok of the chunk at call
         // offset cs is a boundary step iff it lies on the grid and phase + (tok mod w) is 0 or w,
@@ -385,32 +386,29 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                 const unsigned own_word = wx == 0 ? mk[0] : wx == 1 ? mk[1] : wx == 2 ? mk[2] : mk[3];
                 dec16 = (own_word >> (16 * (warp & 1))) & 0xffffu;
             }
+            // the gate pair of row rr of this warp, or (1, 1) where the step does not decay
+            auto gate_or_one = [&](uint32_t g2, int rr) { return ((dec16 >> rr) & 1u) ? g2 : 0x3f803f80u; };
 
-            // ---- first sweep: running sums of log2 Lambda down this warp's rows.  They are parked
-            //      in the slots this thread will overwrite in the second sweep (even channel: Q~'s,
-            //      odd channel: the gate's own), so nothing is computed twice.
+            // ---- first sweep: the product of the decays over this warp's 16 rows, per channel; only
+            //      its log2 crosses warps (a boundary step or a row past the end multiplies by 1)
             if (!(ok = mbar_wait(&sm.bar.full_in, n & 1, limit, abort_flag, p.status))) break;
             {
-                float run0 = 0.0f, run1 = 0.0f;
+                float p0 = 1.0f, p1 = 1.0f;
 #pragma unroll
                 for (int rr = 0; rr < 16; ++rr) {
-                    const int off = scale_off + rr * 128 + ((lane_piece ^ (rr & 7)) << 4);
-                    const uint32_t g2 = *reinterpret_cast<const uint32_t*>(sm.g + off);
-                    if ((dec16 >> rr) & 1u) {
-                        run0 += log2_decay(bf16_lo(g2));
-                        run1 += log2_decay(bf16_hi(g2));
-                    }
-                    *reinterpret_cast<float*>(sm.qt + off) = run0;
-                    *reinterpret_cast<float*>(sm.g + off) = run1;
-                    if (p.tied) *reinterpret_cast<uint32_t*>(sm.k + off) = g2;
+                    const uint32_t g2 = gate_or_one(*reinterpret_cast<const uint32_t*>(sm.g + row_off(rr)), rr);
+                    p0 *= bf16_lo(g2);
+                    p1 *= bf16_hi(g2);
                 }
-                *reinterpret_cast<float2*>(&sm.segsum[warp][2 * lane]) = make_float2(run0, run1);
+                // a product that has left the fp32 range reads as -inf and fails the range check
+                *reinterpret_cast<float2*>(&sm.segsum[warp][2 * lane]) = make_float2(lg2(p0), lg2(p1));
             }
             mbar_arrive(&sm.bar.scan);
             if (!(ok = mbar_wait(&sm.bar.scan, n & 1, limit, abort_flag, p.status))) break;
 
-            // ---- this warp's offset into the chunk, the chunk's total, the range check ------------
-            float h0, h1;       // (sum over the warps before this one) - r, so that b_i - r = running sum + h
+            // ---- this warp's place in the chunk, the chunk's total, the range check ----------------
+            float f0, f1;       // 2^(b - r) just before this warp's first row
+            float t0, t1;       // 2^(r - b) at this warp's last row
             {
                 float base0 = 0.0f, base1 = 0.0f, tot0 = 0.0f, tot1 = 0.0f;
 #pragma unroll
@@ -419,9 +417,12 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                     tot0 += bsx.x; tot1 += bsx.y;
                     if (x < warp) { base0 += bsx.x; base1 += bsx.y; }
                 }
-                h0 = base0 - 0.5f * tot0;
-                h1 = base1 - 0.5f * tot1;
-                if (warp_max(fmaxf(-tot0, -tot1)) > kSafeRange) {
+                const float2 own = *reinterpret_cast<const float2*>(&sm.segsum[warp][2 * lane]);
+                const float h0 = base0 - 0.5f * tot0, h1 = base1 - 0.5f * tot1;
+                f0 = ex2(h0); f1 = ex2(h1);
+                t0 = ex2(-(h0 + own.x)); t1 = ex2(-(h1 + own.y));
+                // (written so that a NaN fails too; a warp's lanes cover all 64 channels)
+                if (__any_sync(0xffffffffu, !(fabsf(tot0) <= kSafeRange) || !(fabsf(tot1) <= kSafeRange))) {
                     // decay too strong to scale a whole chunk around one reference: leave the chain
                     // to the CUDA-core kernel (every warp takes the same decision)
                     given_up = true;
@@ -439,22 +440,63 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                 m_b = ex2(0.5f * tb);
             }
 
-            // ---- second sweep: Q~ = Q o 2^(b - r), K~ = K o 2^(r - b) ------------------------------
+            // ---- second sweep: Q~ = Q o 2^(b - r) with the factor carried forward down the rows as a
+            //      running product of the gates, K~ = K o 2^(r - b) with its factor carried backward
+            //      from the warp's last row, so that no factor is ever inverted.  The fp32 factors are
+            //      rounded to bf16 and applied with packed bf16 multiplies.  (Rows in groups of eight:
+            //      a group's loads are issued before its stores, which the compiler must take to
+            //      alias later loads.)
             if (n > 0 && !(ok = mbar_wait(&sm.bar.stage_free, (n - 1) & 1, limit, abort_flag, p.status))) break;
 #pragma unroll
-            for (int rr = 0; rr < 16; ++rr) {
-                const int off = scale_off + rr * 128 + ((lane_piece ^ (rr & 7)) << 4);
-                const float e0 = *reinterpret_cast<const float*>(sm.qt + off) + h0;
-                const float e1 = *reinterpret_cast<const float*>(sm.g + off) + h1;
-                const uint32_t q2 = *reinterpret_cast<const uint32_t*>(sm.q + off);
-                const uint32_t k2 = *reinterpret_cast<const uint32_t*>(sm.k + off);
-                float k_lo = bf16_lo(k2), k_hi = bf16_hi(k2);
-                if (p.tied) { k_lo = 1.0f - k_lo; k_hi = 1.0f - k_hi; }
-                const bool live = 16 * warp + rr < Lc;      // rows past the end of the sequence contribute nothing
-                const uint32_t qo = pack_bf16(bf16_lo(q2) * ex2(e0), bf16_hi(q2) * ex2(e1));
-                const uint32_t ko = pack_bf16(k_lo * ex2(-e0), k_hi * ex2(-e1));
-                *reinterpret_cast<uint32_t*>(sm.qt + off) = live ? qo : 0u;
-                *reinterpret_cast<uint32_t*>(sm.kt + off) = live ? ko : 0u;
+            for (int r8 = 0; r8 < 16; r8 += 8) {
+                uint32_t g2[8], q2[8];
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    g2[x] = *reinterpret_cast<const uint32_t*>(sm.g + row_off(r8 + x));
+                    q2[x] = *reinterpret_cast<const uint32_t*>(sm.q + row_off(r8 + x));
+                }
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    const uint32_t gx = gate_or_one(g2[x], r8 + x);
+                    f0 *= bf16_lo(gx);
+                    f1 *= bf16_hi(gx);
+                    *reinterpret_cast<uint32_t*>(sm.qt + row_off(r8 + x)) = mul_bf16x2(q2[x], pack_bf16(f0, f1));
+                }
+            }
+            if (!p.tied) {
+#pragma unroll
+                for (int r8 = 8; r8 >= 0; r8 -= 8) {
+                    uint32_t g2[8], k2[8];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        g2[x] = *reinterpret_cast<const uint32_t*>(sm.g + row_off(r8 + x));
+                        k2[x] = *reinterpret_cast<const uint32_t*>(sm.k + row_off(r8 + x));
+                    }
+#pragma unroll
+                    for (int x = 7; x >= 0; --x) {
+                        *reinterpret_cast<uint32_t*>(sm.kt + row_off(r8 + x)) = mul_bf16x2(k2[x], pack_bf16(t0, t1));
+                        const uint32_t gx = gate_or_one(g2[x], r8 + x);
+                        t0 *= bf16_lo(gx);
+                        t1 *= bf16_hi(gx);
+                    }
+                }
+            } else {
+                // key tied to the gate: k = 1 - lambda in fp32 (0 on rows past the end of the sequence)
+#pragma unroll
+                for (int r8 = 8; r8 >= 0; r8 -= 8) {
+                    uint32_t g2[8];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) g2[x] = *reinterpret_cast<const uint32_t*>(sm.g + row_off(r8 + x));
+#pragma unroll
+                    for (int x = 7; x >= 0; --x) {
+                        const float one = 16 * warp + r8 + x < Lc ? 1.0f : 0.0f;
+                        *reinterpret_cast<uint32_t*>(sm.kt + row_off(r8 + x)) =
+                            pack_bf16((one - bf16_lo(g2[x])) * t0, (one - bf16_hi(g2[x])) * t1);
+                        const uint32_t gx = gate_or_one(g2[x], r8 + x);
+                        t0 *= bf16_lo(gx);
+                        t1 *= bf16_hi(gx);
+                    }
+                }
             }
             write_state_bf16(m_a, m_b);
             mbar_arrive(&sm.bar.in_free);

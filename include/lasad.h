@@ -92,7 +92,8 @@ int lasad_set_option(lasad_ctx* ctx, int option, int value);
  * lasad_create allocates 1024 slots.  A lasad_forward call with more (batch, head) pairs than
  * the context holds grows the storage first (cudaMalloc, which synchronises the device and must
  * not happen inside a stream capture); calling lasad_reserve up front keeps lasad_forward
- * allocation-free.
+ * allocation-free.  The same call sizes the 4-byte-per-pair flag array of lasad_forward_gated
+ * (lasad_create provides for 65536 pairs).
  */
 int lasad_reserve(lasad_ctx* ctx, int64_t units);
 
@@ -192,7 +193,17 @@ int lasad_decode_step_pos(lasad_ctx* ctx, const lasad_params* p,
  *   k      as in lasad_forward, or NULL: the key is tied to the gate, k_t = 1 - lambda_t (the
  *          paper's base decay, lambda_t = 1 - k_t; Algorithm 1).  k_stride always describes gate.
  *   The `decay` vector of lasad_forward has no counterpart here.  Other arguments, dtypes, sizes
- *   and error rules as for lasad_forward / lasad_decode_step.  Arithmetic is fp32 on CUDA cores.
+ *   and error rules as for lasad_forward / lasad_decode_step.
+ *
+ * lasad_forward_gated with BF16 and dk == dv == 64 runs on the tensor cores (two launches: the
+ * tensor-core kernel, which scales each 128-token chunk's queries and keys around a per-channel
+ * reference decay and gives up a (batch, head) whose decay over one chunk falls below 2^-200 in
+ * some channel, and a CUDA-core kernel that recomputes exactly the pairs given up, so every gate
+ * in [0,1] is handled); LASAD_OPT_PREFILL_IMPL = 1 forces the CUDA-core kernel for all pairs.
+ * Other shapes and the decode step use fp32 arithmetic on CUDA cores.  The calls of one ctx
+ * share a per-pair flag array: two lasad_forward_gated calls on one ctx must not overlap on the
+ * device, and a call with more (batch, head) pairs than lasad_create or lasad_reserve provided
+ * for (65536 by default) grows the array first, as described at lasad_reserve.
  */
 int lasad_forward_gated(lasad_ctx* ctx, const lasad_params* p,
                         const void* q, const void* k, const void* v, const void* gate,

@@ -200,6 +200,12 @@ def run_ours(args):
             print(json.dumps({"decode": dec}), flush=True)
         ctx.close()
         return
+    if args.only == "gated":
+        res = gated_sweep(ctx, peaks, dev, [wl], decode=False, reps=K)
+        if rank == 0:
+            print(json.dumps({"gated": res}), flush=True)
+        ctx.close()
+        return
 
     # ---- prefill: inputs resident in HBM -------------------------------------------------
     hq, hk, hv = [t.pin_memory() for t in workloads.make_qkv(wl)]
@@ -352,10 +358,11 @@ def prefill_sweep(ctx, peaks, dev, names, reps: int = 10):
     return out
 
 
-def gated_sweep(ctx, peaks, dev, reps: int = 10):
-    """The data-dependent (gated) form: kernel time of one prefill on the config 2 and config 3
-    shapes (L2 flushed between launches) and of one decode step on the config 4 shape (rotating
-    state sets), with a seeded logistic-normal gate and the key given explicitly."""
+def gated_sweep(ctx, peaks, dev, wls=None, decode: bool = True, reps: int = 10):
+    """The data-dependent (gated) form: time of one prefill call (tensor-core kernel plus the
+    CUDA-core kernel behind it that redoes flagged chains; L2 flushed between calls) on the
+    config 2, 3 and 5b shapes and of one decode step on the config 4 shape (rotating state
+    sets), with a seeded logistic-normal gate and the key given explicitly."""
     import torch
 
     from paper_2507_01652_b200 import workloads
@@ -363,8 +370,9 @@ def gated_sweep(ctx, peaks, dev, reps: int = 10):
     stream = torch.cuda.current_stream()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     out = {"prefill": [], "decode": None}
-    for name in ("config2", "config3"):
-        wl = workloads.WORKLOADS[name]
+    if wls is None:
+        wls = [workloads.WORKLOADS[name] for name in ("config2", "config3", "config5b")]
+    for wl in wls:
         q, k, v = [t.to(dev) for t in workloads.make_qkv(wl)]
         lam = workloads.make_gate(wl).to(dev)
         o = torch.empty_like(v)
@@ -386,6 +394,8 @@ def gated_sweep(ctx, peaks, dev, reps: int = 10):
                                "algorithmic_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
                                "frac_of_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)})
         del q, k, v, lam, o, s_out
+    if not decode:
+        return out
     dw = workloads.WORKLOADS["config4"]
     T = 16
     q, k, v = [t.to(dev) for t in workloads.make_qkv(dw, T)]
@@ -592,8 +602,9 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-configuration prefill sweep")
     ap.add_argument("--prefill-impl", type=int, default=0, choices=[0, 1, 2, 3],
                     help="prefill kernel: 0 library default, 1 CUDA cores, 2 tcgen05 CTA-per-chain, 3 tcgen05 task-streaming")
-    ap.add_argument("--only", choices=["all", "prefill", "decode"], default="all",
-                    help="time only one of the two kernels (small profiling runs)")
+    ap.add_argument("--only", choices=["all", "prefill", "decode", "gated"], default="all",
+                    help="time only one of the kernels (small profiling runs); gated = the gated prefill "
+                         "on --prefill-workload")
     ap.add_argument("--prefill-batch", type=int, default=0, help="override the prefill workload's batch")
     ap.add_argument("--decode-batch", type=int, default=0, help="override the decode workload's batch")
     args = ap.parse_args()

@@ -35,6 +35,7 @@
 // through the normal exit (copies in flight are waited for, TMEM is freed).
 #include "lasad_common.cuh"
 #include "lasad_tc_ptx.cuh"
+#include "lasad_tc_tma.cuh"
 
 namespace lasad {
 namespace {
@@ -589,39 +590,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     }
 }
 
-// cuTensorMapEncodeTiled, fetched through the runtime so that the library does not link libcuda.
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
-// [B,T,H,64] bf16 with element strides (b,t,h) -> 4-D map (d, h, t, b), box = one chunk of one head.
-bool encode_map(CUtensorMap* map, const void* base, int B, int T, int H, const long long* strides)
-{
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return false;
-    auto bytes = [](long long elems) { return (cuuint64_t)(elems > 0 ? elems * 2 : 128); };
-    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
-    const cuuint64_t gstr[3] = {bytes(strides[2]), bytes(strides[1]), bytes(strides[0])};
-    const cuuint32_t box[4] = {(cuuint32_t)kD, 1u, (cuuint32_t)kC, 1u};
-    const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, gstr, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 #ifdef LASAD_TC_TRACE
@@ -636,8 +604,8 @@ bool prefill_tc_supported(int dk, int dv, bool bf16) { return bf16 && dk == kD &
 cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st)
 {
     CUtensorMap mq, mk, mv, mo;
-    if (!encode_map(&mq, a.q, a.B, a.T, a.H, a.qs) || !encode_map(&mk, a.k, a.B, a.T, a.H, a.ks) ||
-        !encode_map(&mv, a.v, a.B, a.T, a.H, a.vs) || !encode_map(&mo, a.o, a.B, a.T, a.H, a.os))
+    if (!encode_chunk_map(&mq, a.q, a.B, a.T, a.H, a.qs) || !encode_chunk_map(&mk, a.k, a.B, a.T, a.H, a.ks) ||
+        !encode_chunk_map(&mv, a.v, a.B, a.T, a.H, a.vs) || !encode_chunk_map(&mo, a.o, a.B, a.T, a.H, a.os))
         return cudaErrorInvalidValue;
     TcParams p;
     p.B = a.B; p.T = a.T; p.H = a.H;

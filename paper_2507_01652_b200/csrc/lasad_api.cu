@@ -137,6 +137,7 @@ void fill_args(lasad::KernelArgs& a, const lasad_ctx* ctx, const lasad_params* p
         a.vs[d] = p->v_stride[d]; a.os[d] = p->o_stride[d];
     }
     a.status = ctx->d_status;
+    a.work = ctx->d_status + 16;     // same 256-byte block, zeroed at creation
     a.wait_limit = ctx->wait_limit;
 }
 

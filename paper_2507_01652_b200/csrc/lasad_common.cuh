@@ -24,6 +24,7 @@ struct KernelArgs {
     const int* pos;         // decode only: [B] absolute index of each sequence's token, or nullptr (t0 for all)
     const int* widths;      // decode only: [B] grid width of each sequence, or nullptr (grid_w for all)
     int* status;            // device status word (bounded waits report here)
+    int* work;              // two device ints, zero between launches: work counter of the persistent prefill
     unsigned wait_limit;
 };
 

@@ -1,8 +1,10 @@
 // LASAD chunked prefill on the 5th-generation tensor cores (sm_100a): TMA-fed tcgen05.mma with
 // TMEM accumulators, bf16 I/O, fp32 accumulation and an fp32 master state.
 //
-// One CTA owns one (batch, head) and walks its sequence in chunks of C = 128 tokens; two CTAs
-// fit on an SM (256 TMEM columns and ~106 KB of shared memory each).  With n_i = number of
+// One CTA owns one (batch, head) at a time and walks its sequence in chunks of C = 128 tokens; two
+// CTAs fit on an SM (256 TMEM columns and ~106 KB of shared memory each).  With more chains than
+// resident CTAs, a CTA that finishes a chain draws the next one from a device-side work counter;
+// its loads run two chunks ahead across the chain boundary.  With n_i = number of
 // decaying steps from the chunk start up to and including token i (SAD rule, Section 3.4, from
 // the token's grid position), N = n of the chunk's last token and gamma the head's decay, the
 // SAD recurrence (Section 3.4) unrolled over one chunk is
@@ -63,6 +65,7 @@ struct __align__(8) Barriers {
     unsigned long long p_ready;    // A/P in TMEM, state copy (and Q~) in smem (256 arrivals)
     unsigned long long o_done;     // O MMAs complete (and every MMA issued before them)
     unsigned long long st_ready;   // output tile staged in smem (256 arrivals)
+    unsigned long long tbl;        // exact path: the decay table may change / has changed (256 arrivals)
     unsigned long long drain;      // teardown: all MMAs retired
 };
 
@@ -72,8 +75,8 @@ struct Smem {
     unsigned char k[kStages][kTileBytes];
     unsigned char v[kStages][kTileBytes];
     unsigned char sb[kD * kD * 2];  // bf16 copy of the state, [dk][dv], 128 B rows, swizzled
-    float pw[kC + 4];               // gamma^m,  m = 0..128
-    float ipw[kC + 4];              // gamma^-m, m = 0..128 (normal path only)
+    float pw[kC + 4];               // exact path: gamma^m, m = 0..128, of the current chain's head
+    int ring[4];                    // chain index by ordinal % 4 (-1: no more work)
     Barriers bar;
     uint32_t tmem_base;
     int abort_flag;
@@ -98,6 +101,7 @@ struct TcParams {
     const float* decay;
     const float* state_in;
     float* state_out;
+    int* work;               // [2], zero between launches: chains drawn beyond the grid size, CTAs that have left
     int* status;
     unsigned wait_limit;
 };
@@ -190,12 +194,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const int b = blockIdx.x / p.H, h = blockIdx.x % p.H;
     const int n_chunks = (p.T + kC - 1) / kC;
+    const int n_chains = p.B * p.H;
     volatile int* abort_flag = &sm.abort_flag;
+    volatile int* ring = sm.ring;
     const unsigned limit = p.wait_limit;
-    const float gamma = p.decay[h];
-    const bool fast = gamma >= kFastPathMinDecay;
 
     // ---- set-up ---------------------------------------------------------------------------
     if (tid == 0) {
@@ -206,8 +209,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_init(&sm.bar.p_ready, kEThreads);
         mbar_init(&sm.bar.o_done, 1);
         mbar_init(&sm.bar.st_ready, kEThreads);
+        mbar_init(&sm.bar.tbl, kEThreads);
         mbar_init(&sm.bar.drain, 1);
         sm.abort_flag = 0;
+        sm.ring[0] = (int)blockIdx.x;     // the CTA's first chain; later ones come from the work counter
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 8) {
@@ -216,73 +221,94 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (tid <= kC) {
-        if (fast) {
-            // gamma^m and gamma^-m for m = 0..128 from exp2: |m log2 gamma| <= 95, so the relative
-            // error is ~1e-5, far below what bf16 I/O resolves, and a short sequence does not pay
-            // for double-precision arithmetic in every CTA's prologue
-            const float lg = log2f(gamma);
-            sm.pw[tid] = exp2f((float)tid * lg);
-            sm.ipw[tid] = exp2f(-(float)tid * lg);
-        } else {
-            // exact path: binary exponentiation in double precision (0^0 = 1)
-            double base = (double)gamma, acc = 1.0;
-            for (int e = tid; e > 0; e >>= 1) {
-                if (e & 1) acc *= base;
-                base *= base;
-            }
-            sm.pw[tid] = (float)acc;
-            sm.ipw[tid] = 0.0f;
-        }
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
 
+    // Every role walks the same sequence of chunks: all chunks of the CTA's first chain, then all
+    // chunks of the next chain the TMA warp drew from the work counter, and so on.  g counts the
+    // chunks of that sequence (stage g % 2, barrier phases from g); a chain's position in it is
+    // its ordinal, and ring[ordinal % 4] holds the chain's index, or -1 when the work has run out.
+    // The TMA warp publishes an ordinal's entry before it issues (or, for -1, completes by hand)
+    // the `full` barrier of that chain's first chunk, and the other roles read it after that wait.
+
     if (warp == 9) {
         // ===================== TMA warp: loads two chunks ahead, stores each output tile =======
         if (elect_one()) {
+            // load iterator: (chain, chunk, ordinal) of the next chunk to be loaded
+            int ld_chain = (int)blockIdx.x, ld_n = 0, ld_ord = 0;
+            int ld_b = ld_chain / p.H, ld_h = ld_chain - ld_b * p.H;
+            bool ended = false;            // the end marker has been delivered
+            int last_real = -1;            // sequence number of the last chunk whose loads were issued
+            auto draw = [&]() {
+                const int c = (int)gridDim.x + atomicAdd(p.work, 1);
+                return c < n_chains ? c : -1;
+            };
             // A stage is refilled in two steps: K and V as soon as every MMA of the chunk that used
             // them has retired, Q (whose buffer stages the output tile) once the store has read it.
-            auto issue_kv = [&](int n) {
-                const int s = n % kStages;
+            auto issue_kv = [&](int g) {
+                const int s = g % kStages;
+                if (ld_chain < 0) {
+                    if (!ended) {
+                        mbar_arrive(&sm.bar.full[s]);     // completes the phase: the waiters find -1 in the ring
+                        ended = true;
+                    }
+                    return;
+                }
                 mbar_arrive_expect_tx(&sm.bar.full[s], 3 * kTileBytes);
-                tma_load_4d(sm.k[s], &tm_k, &sm.bar.full[s], 0, h, n * kC, b);
-                tma_load_4d(sm.v[s], &tm_v, &sm.bar.full[s], 0, h, n * kC, b);
+                tma_load_4d(sm.k[s], &tm_k, &sm.bar.full[s], 0, ld_h, ld_n * kC, ld_b);
+                tma_load_4d(sm.v[s], &tm_v, &sm.bar.full[s], 0, ld_h, ld_n * kC, ld_b);
+                last_real = g;
             };
-            auto issue_q = [&](int n) {
-                const int s = n % kStages;
-                tma_load_4d(sm.q[s], &tm_q, &sm.bar.full[s], 0, h, n * kC, b);
+            auto issue_q = [&](int g) {
+                if (ld_chain < 0) return;
+                const int s = g % kStages;
+                tma_load_4d(sm.q[s], &tm_q, &sm.bar.full[s], 0, ld_h, ld_n * kC, ld_b);
+                if (++ld_n == n_chunks) {
+                    ld_n = 0;
+                    ++ld_ord;
+                    ld_chain = draw();
+                    ring[ld_ord & 3] = ld_chain;
+                    ld_b = ld_chain / p.H;
+                    ld_h = ld_chain - ld_b * p.H;
+                }
             };
-            int loads_issued = min(n_chunks, kStages);
-            for (int n = 0; n < loads_issued; ++n) {
-                issue_kv(n);
-                issue_q(n);
+            for (int g = 0; g < kStages; ++g) {
+                issue_kv(g);
+                issue_q(g);
             }
-            for (int n = 0; n < n_chunks; ++n) {
-                const int s = n % kStages;
-                const bool refill = n + kStages < n_chunks;
-                if (refill) {
-                    if (!mbar_wait(&sm.bar.o_done, n & 1, limit, abort_flag, p.status)) break;
-                    issue_kv(n + kStages);
-                    loads_issued = n + kStages + 1;
-                }
-                // the output tile of chunk n sits in the Q buffer of its stage
-                const bool staged = mbar_wait(&sm.bar.st_ready, n & 1, limit, abort_flag, p.status);
+            // store iterator: the chunk whose output tile leaves next
+            int st_chain = (int)blockIdx.x, st_n = 0, st_ord = 0;
+            int st_b = st_chain / p.H, st_h = st_chain - st_b * p.H;
+            for (int g = 0; st_chain >= 0; ++g) {
+                const int s = g % kStages;
+                if (!mbar_wait(&sm.bar.o_done, g & 1, limit, abort_flag, p.status)) break;
+                issue_kv(g + kStages);
+                // the output tile of chunk g sits in the Q buffer of its stage
+                const bool staged = mbar_wait(&sm.bar.st_ready, g & 1, limit, abort_flag, p.status);
                 if (staged) {
-                    tma_store_4d(&tm_o, sm.q[s], 0, h, n * kC, b);
+                    tma_store_4d(&tm_o, sm.q[s], 0, st_h, st_n * kC, st_b);
                     tma_store_commit();
-                    if (refill) tma_store_wait_read();        // the store has finished reading the buffer
+                    if (ld_chain >= 0) tma_store_wait_read();  // the store has finished reading the buffer
                 }
-                if (refill) issue_q(n + kStages);              // (also after a failed wait: the stage's barrier must complete)
+                issue_q(g + kStages);                          // (also after a failed wait: the stage's barrier must complete)
                 if (!staged) break;
+                if (++st_n == n_chunks) {
+                    st_n = 0;
+                    ++st_ord;
+                    st_chain = ring[st_ord & 3];               // published by this thread when the loads reached it
+                    st_b = st_chain / p.H;
+                    st_h = st_chain - st_b * p.H;
+                }
             }
             tma_store_wait_all();
             // leave only when every issued load has landed (they write this CTA's shared memory)
-            for (int n = max(0, loads_issued - kStages); n < loads_issued; ++n)
+            // (once the end marker is out, the chunk before the last loaded one has been processed,
+            // and its stage's barrier has moved on by the marker's phase: only the last one is waited for)
+            for (int g = max(0, ended ? last_real : last_real - kStages + 1); g <= last_real; ++g)
                 for (unsigned it = 0; it < kTeardownLimit; ++it)
-                    if (mbar_try_wait(&sm.bar.full[n % kStages], (n / kStages) & 1)) break;
+                    if (mbar_try_wait(&sm.bar.full[g % kStages], (g / kStages) & 1)) break;
         }
         __syncwarp();
     } else if (warp == 8) {
@@ -295,10 +321,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const uint64_t dq0 = make_desc(smem_u32(sm.q[0])), dq1 = make_desc(smem_u32(sm.q[1]));
         const uint64_t dk0 = make_desc(smem_u32(sm.k[0])), dk1 = make_desc(smem_u32(sm.k[1]));
         const uint64_t dv0 = make_desc(smem_u32(sm.v[0])), dv1 = make_desc(smem_u32(sm.v[1]));
-        auto issue_m1 = [&](int n) {
-            const int s = n % kStages;
+        int m_n = 0, m_ord = 0;           // chunk within its chain and chain ordinal of the chunk whose scores come next
+        bool fast_next = true;            // path of that chunk's chain
+        // waits for chunk g's tiles, finds out whose they are and issues its score MMAs;
+        // 0 = issued, 1 = the work has run out, -1 = a wait gave up
+        auto issue_m1 = [&](int g) {
+            const int s = g % kStages;
             const uint64_t dqs = s ? dq1 : dq0, dks = s ? dk1 : dk0;
-            if (!mbar_wait(&sm.bar.full[s], (n / kStages) & 1, limit, abort_flag, p.status)) return false;
+            if (!mbar_wait(&sm.bar.full[s], (g / kStages) & 1, limit, abort_flag, p.status)) return -1;
+            if (m_n == 0) {
+                const int chain = ring[m_ord & 3];
+                if (chain < 0) return 1;
+                fast_next = p.decay[chain % p.H] >= kFastPathMinDecay;
+            }
+            if (++m_n == n_chunks) {
+                m_n = 0;
+                ++m_ord;
+            }
             tc_fence_after();
             if (elect_one()) {
 #pragma unroll
@@ -307,14 +346,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 mma_commit(&sm.bar.s_done);
             }
             __syncwarp();
-            return true;
+            return 0;
         };
-        bool ok = n_chunks > 0 && issue_m1(0);
-        for (int n = 0; ok && n < n_chunks; ++n) {
-            const int s = n % kStages;
+        int more = issue_m1(0);
+        for (int g = 0; more == 0; ++g) {
+            const int s = g % kStages;
             const uint64_t dqs = s ? dq1 : dq0, dks = s ? dk1 : dk0, dvs = s ? dv1 : dv0;
-            TRACE_M(8 * n + 0);
-            if (!mbar_wait(&sm.bar.x_ready, n & 1, limit, abort_flag, p.status)) { ok = false; break; }
+            const bool fast = fast_next;
+            TRACE_M(8 * g + 0);
+            if (!mbar_wait(&sm.bar.x_ready, g & 1, limit, abort_flag, p.status)) break;
             tc_fence_after();
             if (elect_one()) {
 #pragma unroll
@@ -331,10 +371,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
             }
             __syncwarp();
-            TRACE_M(8 * n + 1);
-            if (!mbar_wait(&sm.bar.p_ready, n & 1, limit, abort_flag, p.status)) { ok = false; break; }
+            TRACE_M(8 * g + 1);
+            if (!mbar_wait(&sm.bar.p_ready, g & 1, limit, abort_flag, p.status)) break;
             tc_fence_after();
-            TRACE_M(8 * n + 2);
+            TRACE_M(8 * g + 2);
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kC / 16; ++kk)  // A/P: 8 TMEM columns per step (tokens 0..63 at columns
@@ -350,9 +390,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 mma_commit(&sm.bar.o_done);
             }
             __syncwarp();
-            TRACE_M(8 * n + 3);
-            if (n + 1 < n_chunks) ok = issue_m1(n + 1);
-            TRACE_M(8 * n + 4);
+            TRACE_M(8 * g + 3);
+            more = issue_m1(g + 1);
+            TRACE_M(8 * g + 4);
         }
         // make sure nothing is still running on the tensor pipe before TMEM is freed
         if (elect_one()) {
@@ -373,22 +413,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // st[4k], st[4k+1] = (row r0, columns c0 + 8k, + 1), st[4k+2], st[4k+3] = (row r0 + 8, same).
         const int r0 = qd * 16 + (lane >> 2);
         const int c0 = 32 * grp + 2 * (lane & 3);
-        const size_t unit = (size_t)blockIdx.x * kD * kD;
-
-        // position of the call's first token relative to the grid (SAD rule, Section 3.4)
-        GridPos gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0, lane);
 
         float st[16];                            // fp32 master state, this thread's 16 values
-#pragma unroll
-        for (int e = 0; e < 16; ++e) st[e] = 0.0f;
-        if (p.state_in) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float2 a = *reinterpret_cast<const float2*>(p.state_in + unit + (size_t)r0 * kD + c0 + 8 * k);
-                const float2 c = *reinterpret_cast<const float2*>(p.state_in + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k);
-                st[4 * k] = a.x; st[4 * k + 1] = a.y; st[4 * k + 2] = c.x; st[4 * k + 3] = c.y;
-            }
-        }
         // bf16 copy of mult * state for the Q x state MMA of the next chunk: [dk][dv] rows of 128 B,
         // 16-byte pieces swizzled by the row; this thread writes eight bf16 pairs
         auto write_state_bf16 = [&](float mult) {
@@ -432,150 +458,204 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         };
 
         bool ok = true;
-        if (fast) {
-            // ------------------------------- normal path ---------------------------------------
-            ChunkDecay cd = chunk_decay(gp, 0, min(kC, p.T), qd, lane);
-            write_state_bf16(sm.pw[cd.n_last]);
-            ok = mbar_wait(&sm.bar.full[0], 0, limit, abort_flag, p.status);
-            if (ok) {
-                scale_row_inplace<4>(sm.v[0] + i * 128, sm.pw[cd.n_last - cd.ni], 4 * grp, i & 7);
+        int g = 0;                      // chunks of this CTA's sequence done so far
+        unsigned tbl_phase = 0;         // completed phases of the table barrier
+        int chain = (int)blockIdx.x;
+        for (int ord = 0; ok; ++ord) {
+            // ---- next chain: its index is in the ring once the tiles of its first chunk are in ----
+            if (!(ok = mbar_wait(&sm.bar.full[g % kStages], (g / kStages) & 1, limit, abort_flag, p.status))) break;
+            if (ord > 0) chain = ring[ord & 3];
+            if (chain < 0) break;
+            const int h = chain % p.H;
+            const size_t unit = (size_t)chain * kD * kD;
+            const float gamma = p.decay[h];
+            const bool fast = gamma >= kFastPathMinDecay;
+            const float lg = fast ? log2f(gamma) : 0.0f;
+            // position of the call's first token relative to the grid (SAD rule, Section 3.4)
+            GridPos gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0, lane);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) st[e] = 0.0f;
+            if (p.state_in) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float2 a = *reinterpret_cast<const float2*>(p.state_in + unit + (size_t)r0 * kD + c0 + 8 * k);
+                    const float2 c = *reinterpret_cast<const float2*>(p.state_in + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k);
+                    st[4 * k] = a.x; st[4 * k + 1] = a.y; st[4 * k + 2] = c.x; st[4 * k + 3] = c.y;
+                }
+            }
+
+            if (fast) {
+                // ------------------------------- normal path ---------------------------------------
+                // gamma^m straight from ex2.approx: |m log2 gamma| <= 95, relative error ~1e-5, far
+                // below what bf16 I/O resolves
+                auto gpow = [&](int m) { return ex2_approx((float)m * lg); };
+                ChunkDecay cd = chunk_decay(gp, 0, min(kC, p.T), qd, lane);
+                write_state_bf16(gpow(cd.n_last));
+                scale_row_inplace<4>(sm.v[g % kStages] + i * 128, gpow(cd.n_last - cd.ni), 4 * grp, i & 7);
                 fence_proxy_async();
                 mbar_arrive(&sm.bar.x_ready);
-            }
-            for (int n = 0; ok && n < n_chunks; ++n) {
-                const int s = n % kStages;
-                TRACE_E(8 * n + 0);
-                if (!(ok = mbar_wait(&sm.bar.s_done, n & 1, limit, abort_flag, p.status))) break;
-                tc_fence_after();
-                TRACE_E(8 * n + 1);
-                // ---- E1: A = tril(S) -> bf16 over S's own columns.  This warp converts the
-                //      32-column blocks 2 grp and 2 grp + 1 of its rows and keeps the result inside
-                //      its own half of S's columns (block pc -> columns 64 grp + 16 (pc & 1), always
-                //      behind this warp's own reads); the A V~ MMAs walk the columns in that order.
+                for (int n = 0; ok && n < n_chunks; ++n, ++g) {
+                    const int s = g % kStages;
+                    TRACE_E(8 * g + 0);
+                    if (!(ok = mbar_wait(&sm.bar.s_done, g & 1, limit, abort_flag, p.status))) break;
+                    tc_fence_after();
+                    TRACE_E(8 * g + 1);
+                    // ---- E1: A = tril(S) -> bf16 over S's own columns.  This warp converts the
+                    //      32-column blocks 2 grp and 2 grp + 1 of its rows and keeps the result inside
+                    //      its own half of S's columns (block pc -> columns 64 grp + 16 (pc & 1), always
+                    //      behind this warp's own reads); the A V~ MMAs walk the columns in that order.
 #pragma unroll
-                for (int pi = 0; pi < 2; ++pi) {
-                    const int pc = 2 * grp + pi;
-                    uint32_t pk[16];
-                    if (pc <= qd) {
-                        uint32_t sv[32];
-                        tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
-                        tmem_wait_ld();
-                        if (pc < qd) {
+                    for (int pi = 0; pi < 2; ++pi) {
+                        const int pc = 2 * grp + pi;
+                        uint32_t pk[16];
+                        if (pc <= qd) {
+                            uint32_t sv[32];
+                            tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
+                            tmem_wait_ld();
+                            if (pc < qd) {
 #pragma unroll
-                            for (int c = 0; c < 16; ++c)
-                                pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
+                                for (int c = 0; c < 16; ++c)
+                                    pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 16; ++c)
+                                    pk[c] = pack_bf16(2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
+                                                      2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
+                            }
                         } else {
 #pragma unroll
-                            for (int c = 0; c < 16; ++c)
-                                pk[c] = pack_bf16(2 * c <= lane ? __uint_as_float(sv[2 * c]) : 0.0f,
-                                                  2 * c + 1 <= lane ? __uint_as_float(sv[2 * c + 1]) : 0.0f);
+                            for (int c = 0; c < 16; ++c) pk[c] = 0u;
                         }
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                        tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
                     }
-                    tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(&sm.bar.p_ready);
+                    TRACE_E(8 * g + 2);
+
+                    // ---- while the O MMAs run: the state recurrence in fp32 registers ----------------
+                    const float out_f = p.scale * gpow(-(cd.n_last - cd.ni));   // scale * gamma^-(N - n_i)
+                    if (!(ok = mbar_wait(&sm.bar.ds_done, g & 1, limit, abort_flag, p.status))) break;
+                    tc_fence_after();
+                    update_state(gpow(cd.n_last));
+                    TRACE_E(8 * g + 3);
+                    const bool more = n + 1 < n_chunks;
+                    if (more) {
+                        const int cs1 = (n + 1) * kC;
+                        cd = chunk_decay(gp, cs1, min(kC, p.T - cs1), qd, lane);
+                    } else if (p.state_out) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            *reinterpret_cast<float2*>(p.state_out + unit + (size_t)r0 * kD + c0 + 8 * k) =
+                                make_float2(st[4 * k], st[4 * k + 1]);
+                            *reinterpret_cast<float2*>(p.state_out + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k) =
+                                make_float2(st[4 * k + 2], st[4 * k + 3]);
+                        }
+                    }
+                    TRACE_E(8 * g + 4);
+
+                    // ---- E2: o_i = scale * gamma^-(N - n_i) * O'_i ------------------------------------
+                    if (!(ok = mbar_wait(&sm.bar.o_done, g & 1, limit, abort_flag, p.status))) break;
+                    tc_fence_after();
+                    TRACE_E(8 * g + 5);
+                    stage_output(s, out_f);
+                    if (more) write_state_bf16(gpow(cd.n_last));   // gamma^N(next) * S_new
+                    fence_proxy_async();
+                    tc_fence_before();
+                    mbar_arrive(&sm.bar.st_ready);
+                    TRACE_E(8 * g + 6);
+
+                    // ---- V~ of the chain's next chunk, once its loads have landed.  This stage is
+                    //      released (st_ready above) before the wait, so the wait never holds a buffer
+                    //      back.  (The first chunk of the next chain is prepared at the top.)
+                    if (more) {
+                        const int s1 = (g + 1) % kStages;
+                        if (!(ok = mbar_wait(&sm.bar.full[s1], ((g + 1) / kStages) & 1, limit, abort_flag, p.status))) break;
+                        scale_row_inplace<4>(sm.v[s1] + i * 128, gpow(cd.n_last - cd.ni), 4 * grp, i & 7);
+                        fence_proxy_async();
+                        mbar_arrive(&sm.bar.x_ready);
+                    }
                 }
-                tmem_wait_st();
-                fence_proxy_async();   // state copy written at the end of the previous iteration
-                tc_fence_before();
-                mbar_arrive(&sm.bar.p_ready);
-                TRACE_E(8 * n + 2);
-
-                // ---- while the O MMAs run: the state recurrence in fp32 registers ----------------
-                const float out_f = p.scale * sm.ipw[cd.n_last - cd.ni];   // scale * gamma^-(N - n_i)
-                if (!(ok = mbar_wait(&sm.bar.ds_done, n & 1, limit, abort_flag, p.status))) break;
-                tc_fence_after();
-                update_state(sm.pw[cd.n_last]);
-                TRACE_E(8 * n + 3);
-                const bool more = n + 1 < n_chunks;
-                if (more) {
-                    const int cs1 = (n + 1) * kC;
-                    cd = chunk_decay(gp, cs1, min(kC, p.T - cs1), qd, lane);
+            } else {
+                // ------------------------------- exact path ----------------------------------------
+                // table of gamma^m, m = 0..128, by binary exponentiation in double precision
+                // (0^0 = 1); every thread is done with the previous chain's table before it changes
+                mbar_arrive(&sm.bar.tbl);
+                if (!(ok = mbar_wait(&sm.bar.tbl, tbl_phase & 1, limit, abort_flag, p.status))) break;
+                ++tbl_phase;
+                if (tid <= kC) {
+                    double base = (double)gamma, acc = 1.0;
+                    for (int e = tid; e > 0; e >>= 1) {
+                        if (e & 1) acc *= base;
+                        base *= base;
+                    }
+                    sm.pw[tid] = (float)acc;
                 }
-                TRACE_E(8 * n + 4);
-
-                // ---- E2: o_i = scale * gamma^-(N - n_i) * O'_i ------------------------------------
-                if (!(ok = mbar_wait(&sm.bar.o_done, n & 1, limit, abort_flag, p.status))) break;
-                tc_fence_after();
-                TRACE_E(8 * n + 5);
-                stage_output(s, out_f);
-                if (more) write_state_bf16(sm.pw[cd.n_last]);   // gamma^N(next) * S_new
-                fence_proxy_async();
-                tc_fence_before();
-                mbar_arrive(&sm.bar.st_ready);
-                TRACE_E(8 * n + 6);
-
-                // ---- V~ of the next chunk, once its loads have landed.  This stage is released
-                //      (st_ready above) before the wait, so the wait never holds a buffer back.
-                if (more) {
-                    const int s1 = (n + 1) % kStages;
-                    if (!(ok = mbar_wait(&sm.bar.full[s1], ((n + 1) / kStages) & 1, limit, abort_flag, p.status))) break;
-                    scale_row_inplace<4>(sm.v[s1] + i * 128, sm.pw[cd.n_last - cd.ni], 4 * grp, i & 7);
+                mbar_arrive(&sm.bar.tbl);
+                if (!(ok = mbar_wait(&sm.bar.tbl, tbl_phase & 1, limit, abort_flag, p.status))) break;
+                ++tbl_phase;
+                write_state_bf16(1.0f);
+                for (int n = 0; ok && n < n_chunks; ++n, ++g) {
+                    const int s = g % kStages;
+                    const int cs = n * kC;
+                    const ChunkDecay cd = chunk_decay(gp, cs, min(kC, p.T - cs), qd, lane);
+                    if (n > 0 &&
+                        !(ok = mbar_wait(&sm.bar.full[s], (g / kStages) & 1, limit, abort_flag, p.status))) break;
+                    if (!(ok = mbar_wait(&sm.bar.s_done, g & 1, limit, abort_flag, p.status))) break;
+                    tc_fence_after();
+                    // K~ first (M1 has finished reading K): it unblocks the dS MMAs
+                    if (grp == 1) scale_row_inplace<8>(sm.k[s] + i * 128, sm.pw[cd.n_last - cd.ni], 0, i & 7);
                     fence_proxy_async();
                     mbar_arrive(&sm.bar.x_ready);
-                }
-            }
-        } else {
-            // ------------------------------- exact path ----------------------------------------
-            write_state_bf16(1.0f);
-            for (int n = 0; ok && n < n_chunks; ++n) {
-                const int s = n % kStages;
-                const int cs = n * kC;
-                const ChunkDecay cd = chunk_decay(gp, cs, min(kC, p.T - cs), qd, lane);
-                if (!(ok = mbar_wait(&sm.bar.s_done, n & 1, limit, abort_flag, p.status))) break;
-                tc_fence_after();
-                // K~ first (M1 has finished reading K): it unblocks the dS MMAs
-                if (grp == 1) scale_row_inplace<8>(sm.k[s] + i * 128, sm.pw[cd.n_last - cd.ni], 0, i & 7);
-                fence_proxy_async();
-                mbar_arrive(&sm.bar.x_ready);
-                // P = S o gamma^(n_i - n_j) o [j <= i], weights straight from the table
+                    // P = S o gamma^(n_i - n_j) o [j <= i], weights straight from the table
 #pragma unroll 1
-                for (int pi = 0; pi < 2; ++pi) {
-                    const int pc = 2 * grp + pi;
-                    uint32_t pk[16];
-                    if (pc <= qd) {
-                        uint32_t sv[32];
-                        tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
-                        tmem_wait_ld();
+                    for (int pi = 0; pi < 2; ++pi) {
+                        const int pc = 2 * grp + pi;
+                        uint32_t pk[16];
+                        if (pc <= qd) {
+                            uint32_t sv[32];
+                            tmem_ld32(tmem + lane_base + kColS + 32 * pc, sv);
+                            tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const int j0 = 32 * pc + 2 * c;
-                            const int d0 = cd.ni - cd.n_of(j0), d1 = cd.ni - cd.n_of(j0 + 1);
-                            const float v0 = j0 <= i ? __uint_as_float(sv[2 * c]) * sm.pw[d0 > 0 ? d0 : 0] : 0.0f;
-                            const float v1 = j0 + 1 <= i ? __uint_as_float(sv[2 * c + 1]) * sm.pw[d1 > 0 ? d1 : 0] : 0.0f;
-                            pk[c] = pack_bf16(v0, v1);
+                            for (int c = 0; c < 16; ++c) {
+                                const int j0 = 32 * pc + 2 * c;
+                                const int d0 = cd.ni - cd.n_of(j0), d1 = cd.ni - cd.n_of(j0 + 1);
+                                const float v0 = j0 <= i ? __uint_as_float(sv[2 * c]) * sm.pw[d0 > 0 ? d0 : 0] : 0.0f;
+                                const float v1 = j0 + 1 <= i ? __uint_as_float(sv[2 * c + 1]) * sm.pw[d1 > 0 ? d1 : 0] : 0.0f;
+                                pk[c] = pack_bf16(v0, v1);
+                            }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 16; ++c) pk[c] = 0u;
                         }
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) pk[c] = 0u;
+                        tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
                     }
-                    tmem_st16(tmem + lane_base + kColS + 64 * grp + 16 * pi, pk);
-                }
-                if (grp == 0) scale_row_inplace<8>(sm.q[s] + i * 128, sm.pw[cd.ni], 0, i & 7);
-                tmem_wait_st();
-                fence_proxy_async();
-                tc_fence_before();
-                mbar_arrive(&sm.bar.p_ready);
+                    if (grp == 0) scale_row_inplace<8>(sm.q[s] + i * 128, sm.pw[cd.ni], 0, i & 7);
+                    tmem_wait_st();
+                    fence_proxy_async();
+                    tc_fence_before();
+                    mbar_arrive(&sm.bar.p_ready);
 
-                if (!(ok = mbar_wait(&sm.bar.ds_done, n & 1, limit, abort_flag, p.status))) break;
-                tc_fence_after();
-                update_state(sm.pw[cd.n_last]);
-                if (!(ok = mbar_wait(&sm.bar.o_done, n & 1, limit, abort_flag, p.status))) break;
-                tc_fence_after();
-                stage_output(s, p.scale);
-                write_state_bf16(1.0f);
-                fence_proxy_async();
-                tc_fence_before();
-                mbar_arrive(&sm.bar.st_ready);
-            }
-        }
-        if (ok && p.state_out) {
+                    if (!(ok = mbar_wait(&sm.bar.ds_done, g & 1, limit, abort_flag, p.status))) break;
+                    tc_fence_after();
+                    update_state(sm.pw[cd.n_last]);
+                    if (n + 1 == n_chunks && p.state_out) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                *reinterpret_cast<float2*>(p.state_out + unit + (size_t)r0 * kD + c0 + 8 * k) = make_float2(st[4 * k], st[4 * k + 1]);
-                *reinterpret_cast<float2*>(p.state_out + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k) =
-                    make_float2(st[4 * k + 2], st[4 * k + 3]);
+                        for (int k = 0; k < 4; ++k) {
+                            *reinterpret_cast<float2*>(p.state_out + unit + (size_t)r0 * kD + c0 + 8 * k) =
+                                make_float2(st[4 * k], st[4 * k + 1]);
+                            *reinterpret_cast<float2*>(p.state_out + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k) =
+                                make_float2(st[4 * k + 2], st[4 * k + 3]);
+                        }
+                    }
+                    if (!(ok = mbar_wait(&sm.bar.o_done, g & 1, limit, abort_flag, p.status))) break;
+                    tc_fence_after();
+                    stage_output(s, p.scale);
+                    if (n + 1 < n_chunks) write_state_bf16(1.0f);
+                    fence_proxy_async();
+                    tc_fence_before();
+                    mbar_arrive(&sm.bar.st_ready);
+                }
             }
         }
     }
@@ -587,6 +667,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+    // the last CTA to leave puts the work counter back to zero for the next launch
+    if (tid == 0) {
+        __threadfence();
+        if (atomicAdd(p.work + 1, 1) == (int)gridDim.x - 1) {
+            p.work[0] = 0;
+            p.work[1] = 0;
+            __threadfence();
+        }
     }
 }
 
@@ -611,11 +700,20 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st)
     p.B = a.B; p.T = a.T; p.H = a.H;
     p.grid_w = a.grid_w; p.prefix_len = a.prefix_len; p.t0 = a.t0; p.scale = a.scale;
     p.decay = a.decay; p.state_in = a.state_in; p.state_out = a.state_out;
+    p.work = a.work;
     p.status = a.status; p.wait_limit = a.wait_limit;
     const size_t smem = sizeof(Smem) + 1024;
     cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    prefill_tc_kernel<<<(unsigned)(a.B * a.H), kThreads, smem, st>>>(mq, mk, mv, mo, p);
+    // Two CTAs fit on an SM; with more chains than that, the CTAs stay and draw further chains
+    // from the work counter, so a chain's first loads overlap the previous chain's last chunk.
+    int dev = 0, sms = 0;
+    e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const long long chains = (long long)a.B * a.H;
+    const unsigned grid = (unsigned)(chains < 2LL * sms ? chains : 2LL * sms);
+    prefill_tc_kernel<<<grid, kThreads, smem, st>>>(mq, mk, mv, mo, p);
     return cudaGetLastError();
 }
 

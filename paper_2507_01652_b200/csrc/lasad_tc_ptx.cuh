@@ -224,6 +224,14 @@ __device__ __forceinline__ void scale_row_inplace(unsigned char* row, float f, i
     }
 }
 
+// 2^x, hardware approximation (relative error about 2^-22; flushes denormals)
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 // One thread of a converged warp.  Issuing tcgen05.mma / TMA instructions under this predicate
 // instead of `lane == 0` lets the compiler keep their descriptors in uniform registers: a chain
 // of 16 small MMAs then issues in ~39 instead of ~75 cycles per instruction.

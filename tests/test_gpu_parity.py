@@ -253,6 +253,29 @@ def test_argument_errors_launch_nothing(ctx):
 # ------------------------------------------------------------------------------------------
 # task-streaming prefill (implementation 3): paths the shared cases above do not reach
 # ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("T", [100, 129, 300])
+def test_more_chains_than_resident_ctas(ctx, T):
+    """More (batch, head) pairs than CTAs that fit on the device: the CTA-per-chain kernel keeps its
+    CTAs and hands them further chains from its work counter.  Heads on the normal and on the exact
+    path alternate (a CTA changes path from one chain to the next), with an incoming state; the call
+    is repeated, so the counter must have returned to zero."""
+    B, H, d, w = 47, 13, 64, 7
+    gen = torch.Generator().manual_seed(300 + T)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+    g = torch.tensor([0.95, 0.0, 0.999, 0.3, 0.6, 0.59, 1.0, 0.9, 0.5, 0.97, 0.2, 0.99, 0.8])
+    s_in = torch.randn(B, H, d, d, generator=gen)
+    o_ref, s_ref = oracle(q, k, v, g, w, 0, 3, 0.5, s_in)
+    dq, dk, dv, dg, ds = _dev(q, k, v, g, s_in)
+    for rep in range(2):
+        o, s = _forward(ctx, 2, dq, dk, dv, dg, w, t0=3, scale=0.5, state_in=ds)
+        assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+        assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
+    # a smaller call afterwards (fewer chains than CTAs) starts from a clean counter as well
+    o, s = _forward(ctx, 2, dq[:2], dk[:2], dv[:2], dg, w, t0=3, scale=0.5, state_in=ds[:2])
+    assert rel_err(o, o_ref[:2]) <= TOL[torch.bfloat16]
+    assert rel_err(s, s_ref[:2]) <= TOL[torch.bfloat16]
+
+
 def test_streaming_prefill_many_heads_and_relay_growth(ctx):
     """More heads than the kernel's shared-memory decay cache holds (H > 256) and more (batch,
     head) pairs than the context's initial relay storage (B * H > 1024, so the call grows it)."""

@@ -365,45 +365,52 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             }
         };
 
-        bool ok = true, given_up = false;
-        for (int n = 0; ok && n < n_chunks; ++n) {
-            const int cs = n * kC;
+        // which of this warp's 16 rows of the next chunk in line are decaying steps (live and not a
+        // row boundary); every call moves on by one chunk
+        int mask_chunk = 0;
+        auto next_mask = [&]() {
+            const int cs = mask_chunk * kC;
             const int Lc = min(kC, p.T - cs);
-            // which of this warp's 16 rows are decaying steps (live and not a row boundary)
-            unsigned dec16;
-            {
-                unsigned mk[4];
+            unsigned mk[4];
 #pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    const int tok = 32 * x + lane;
-                    const int m = phase + rmod[x];
-                    const bool boundary = grid_w > 0 && cs + tok >= pre && (m == 0 || m == grid_w);
-                    mk[x] = __ballot_sync(0xffffffffu, tok < Lc && !boundary);
-                }
-                phase += phase_step;
-                if (phase >= grid_w) phase -= grid_w;
-                const int wx = warp >> 1;
-                const unsigned own_word = wx == 0 ? mk[0] : wx == 1 ? mk[1] : wx == 2 ? mk[2] : mk[3];
-                dec16 = (own_word >> (16 * (warp & 1))) & 0xffffu;
+            for (int x = 0; x < 4; ++x) {
+                const int tok = 32 * x + lane;
+                const int m = phase + rmod[x];
+                const bool boundary = grid_w > 0 && cs + tok >= pre && (m == 0 || m == grid_w);
+                mk[x] = __ballot_sync(0xffffffffu, tok < Lc && !boundary);
             }
+            phase += phase_step;
+            if (phase >= grid_w) phase -= grid_w;
+            ++mask_chunk;
+            const int wx = warp >> 1;
+            const unsigned own_word = wx == 0 ? mk[0] : wx == 1 ? mk[1] : wx == 2 ? mk[2] : mk[3];
+            return (own_word >> (16 * (warp & 1))) & 0xffffu;
+        };
+        // first sweep over a chunk's gate tile: the product of the decays over this warp's 16 rows,
+        // per channel; only its log2 crosses warps (a boundary step or a row past the end multiplies
+        // by 1).  It needs nothing but the gate tile, so it runs as early as that tile is in.
+        auto first_sweep = [&](unsigned dec) {
+            float p0 = 1.0f, p1 = 1.0f;
+#pragma unroll
+            for (int rr = 0; rr < 16; ++rr) {
+                uint32_t g2 = *reinterpret_cast<const uint32_t*>(sm.g + row_off(rr));
+                g2 = ((dec >> rr) & 1u) ? g2 : 0x3f803f80u;
+                p0 *= bf16_lo(g2);
+                p1 *= bf16_hi(g2);
+            }
+            // a product that has left the fp32 range reads as -inf and fails the range check
+            *reinterpret_cast<float2*>(&sm.segsum[warp][2 * lane]) = make_float2(lg2(p0), lg2(p1));
+            mbar_arrive(&sm.bar.scan);
+        };
+
+        bool ok = true, given_up = false;
+        unsigned dec16 = next_mask();
+        ok = mbar_wait(&sm.bar.full_in, 0, limit, abort_flag, p.status);
+        if (ok) first_sweep(dec16);
+        for (int n = 0; ok && n < n_chunks; ++n) {
+            const int Lc = min(kC, p.T - n * kC);
             // the gate pair of row rr of this warp, or (1, 1) where the step does not decay
             auto gate_or_one = [&](uint32_t g2, int rr) { return ((dec16 >> rr) & 1u) ? g2 : 0x3f803f80u; };
-
-            // ---- first sweep: the product of the decays over this warp's 16 rows, per channel; only
-            //      its log2 crosses warps (a boundary step or a row past the end multiplies by 1)
-            if (!(ok = mbar_wait(&sm.bar.full_in, n & 1, limit, abort_flag, p.status))) break;
-            {
-                float p0 = 1.0f, p1 = 1.0f;
-#pragma unroll
-                for (int rr = 0; rr < 16; ++rr) {
-                    const uint32_t g2 = gate_or_one(*reinterpret_cast<const uint32_t*>(sm.g + row_off(rr)), rr);
-                    p0 *= bf16_lo(g2);
-                    p1 *= bf16_hi(g2);
-                }
-                // a product that has left the fp32 range reads as -inf and fails the range check
-                *reinterpret_cast<float2*>(&sm.segsum[warp][2 * lane]) = make_float2(lg2(p0), lg2(p1));
-            }
-            mbar_arrive(&sm.bar.scan);
             if (!(ok = mbar_wait(&sm.bar.scan, n & 1, limit, abort_flag, p.status))) break;
 
             // ---- this warp's place in the chunk, the chunk's total, the range check ----------------
@@ -536,6 +543,17 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             tc_fence_before();
             mbar_arrive(&sm.bar.p_ready);
 
+            // ---- while the O MMAs run: the first sweep of the next chunk, if its gate tile is in
+            //      already (it was requested when this chunk's operands were written) --------------
+            const bool more = n + 1 < n_chunks;
+            unsigned dec_next = 0;
+            bool swept = false;
+            if (more) {
+                dec_next = next_mask();
+                swept = __all_sync(0xffffffffu, mbar_test_wait(&sm.bar.full_in, (n + 1) & 1));
+                if (swept) first_sweep(dec_next);
+            }
+
             // ---- state carry across the chunk, in fp32 registers -----------------------------------
             if (!(ok = mbar_wait(&sm.bar.ds_done, n & 1, limit, abort_flag, p.status))) break;
             tc_fence_after();
@@ -548,6 +566,11 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(&sm.bar.st_ready);
+            if (more && !swept) {
+                if (!(ok = mbar_wait(&sm.bar.full_in, (n + 1) & 1, limit, abort_flag, p.status))) break;
+                first_sweep(dec_next);
+            }
+            dec16 = dec_next;
         }
         if (tid == 0) p.redo[blockIdx.x] = given_up ? 1 : 0;
         if (ok && !given_up && p.state_out) {

@@ -97,6 +97,17 @@ int reserve_redo(lasad_ctx* ctx, int64_t units)
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// What LASAD_OPT_PREFILL_IMPL = 0 stands for on a problem of `batch` sequences.
+int auto_prefill_impl(const lasad_ctx* ctx, const lasad_params* p, int64_t batch, bool tc_ok)
+{
+    if (!tc_ok) return 1;
+    // Few chains and several chunks each: one CTA per chain would leave most SMs idle, so the
+    // chunks are streamed over all of them instead (measured: faster up to about SMs / 3 chains).
+    if (batch * p->H * 3 <= ctx->sm_count && lasad::prefill_stream_chunks(p->T) >= 2 && ctx->stream_max_ctas > 0)
+        return 3;
+    return 2;
+}
+
 int fail_cuda(lasad_ctx* ctx, cudaError_t e)
 {
     ctx->last_cuda_error = (int)e;
@@ -253,7 +264,7 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
 
     int impl = ctx->opt_prefill_impl;
     const bool tc_ok = lasad::prefill_tc_supported(p->dk, p->dv, bf16);
-    if (impl == 0) impl = tc_ok ? 2 : 1;
+    if (impl == 0) impl = auto_prefill_impl(ctx, p, p->B, tc_ok);
     if (impl == 3) {
         if (!tc_ok) return LASAD_ERR_UNSUPPORTED;
         const int64_t units = (int64_t)p->B * p->H;
@@ -508,8 +519,15 @@ int lasad_forward_host(lasad_ctx* ctx, const lasad_params* p, const void* q, con
         if (e == cudaSuccess && b >= 2) e = cudaStreamWaitEvent(st, ctx->ev_out[sl], 0);   // the slot's output has left
         if (e != cudaSuccess) break;
         float* sb = use_state ? ctx->d_host_state + (size_t)b * unit_floats : nullptr;
+        // one batch element per launch, but with the kernel the whole batch would get, so that the
+        // results equal lasad_forward's on the same data bit for bit
+        const int asked = ctx->opt_prefill_impl;
+        if (asked == 0)
+            ctx->opt_prefill_impl =
+                auto_prefill_impl(ctx, p, p->B, lasad::prefill_tc_supported(p->dk, p->dv, p->dtype == LASAD_BF16));
         rc = lasad_forward(ctx, &pb, base, base + off_k, base + off_v, ctx->d_host_decay, state_in ? sb : nullptr,
                            base + off_o, state_out ? sb : nullptr, st);
+        ctx->opt_prefill_impl = asked;
         if (rc != LASAD_OK) break;
         e = cudaEventRecord(ctx->ev_comp[sl], st);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_out, ctx->ev_comp[sl], 0);

@@ -276,6 +276,25 @@ def test_more_chains_than_resident_ctas(ctx, T):
     assert rel_err(s, s_ref[:2]) <= TOL[torch.bfloat16]
 
 
+def test_default_prefill_picks_a_kernel_by_the_number_of_chains(ctx):
+    """Option 0: few (batch, head) pairs with several chunks each go to the task-streaming kernel,
+    everything else in bf16 / d = 64 to the CTA-per-chain kernel; whichever runs, the result is that
+    kernel's bit for bit, and right."""
+    d, w, T = 64, 12, 700
+    gen = torch.Generator().manual_seed(4242)
+    g_all = 0.9 + 0.0999 * torch.rand(16, generator=gen)
+    for B, H, expect in ((1, 16, 3), (12, 16, 2)):
+        q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+        g = g_all[:H]
+        o_ref, s_ref = oracle(q, k, v, g, w)
+        dq, dk, dv, dg = _dev(q, k, v, g)
+        o0, s0 = _forward(ctx, 0, dq, dk, dv, dg, w)
+        o1, s1 = _forward(ctx, expect, dq, dk, dv, dg, w)
+        assert torch.equal(o0, o1) and torch.equal(s0, s1), (B, H)
+        assert rel_err(o0, o_ref) <= TOL[torch.bfloat16]
+        assert rel_err(s0, s_ref) <= TOL[torch.bfloat16]
+
+
 def test_streaming_prefill_many_heads_and_relay_growth(ctx):
     """More heads than the kernel's shared-memory decay cache holds (H > 256) and more (batch,
     head) pairs than the context's initial relay storage (B * H > 1024, so the call grows it)."""

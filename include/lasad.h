@@ -55,10 +55,13 @@ enum { LASAD_F32 = 0, LASAD_BF16 = 1 };
 
 /* Options for lasad_set_option. */
 enum {
-    LASAD_OPT_PREFILL_IMPL = 0, /* 0 auto (bf16, d = 64: 3 when B * H <= SMs / 3 and T > 128, else 2;
-                                   other shapes 1), 1 CUDA-core fp32 kernel, 2 tcgen05 kernel with
-                                   one CTA per (batch, head) at a time, 3 tcgen05 kernel streaming
-                                   (batch, head, chunk) tasks through persistent CTAs              */
+    LASAD_OPT_PREFILL_IMPL = 0, /* 0 auto (bf16, d = 64: 4 when B * H <= SMs / 2 and T > 1920, else 3
+                                   when B * H <= SMs / 3 and T > 128, else 2; other shapes 1),
+                                   1 CUDA-core fp32 kernel,
+                                   2 tcgen05 kernel with one CTA per (batch, head) at a time,
+                                   3 tcgen05 kernel streaming (batch, head, chunk) tasks through
+                                   persistent CTAs, 4 as 2 with few long sequences cut into segments
+                                   that run side by side (three launches; 2 where nothing is cut)   */
     LASAD_OPT_PREFILL_CHUNK = 1,/* CUDA-core prefill chunk length: 0 auto, else 16/32/64          */
     LASAD_OPT_DECODE_TPU = 2,   /* decode: threads per (b,h) state; 0 auto, else 32/64/128/256 */
     LASAD_OPT_WAIT_LIMIT = 3    /* iteration cap of device-side waits; 0 = library default   */

@@ -20,6 +20,8 @@ struct lasad_ctx {
     int64_t relay_cap;
     uint64_t epoch;               // launches of the task-streaming prefill so far
     int stream_max_ctas;
+    // states at the cuts when the CTA-per-chain prefill splits few, long chains into segments
+    float* d_segstate;            // [2 x SMs][dk * dv]
     // per-chain flags of the gated tensor-core prefill: chains it left to the CUDA-core kernel
     int* d_redo;                  // [redo_cap]
     int64_t redo_cap;
@@ -101,10 +103,12 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 int auto_prefill_impl(const lasad_ctx* ctx, const lasad_params* p, int64_t batch, bool tc_ok)
 {
     if (!tc_ok) return 1;
-    // Few chains and several chunks each: one CTA per chain would leave most SMs idle, so the
-    // chunks are streamed over all of them instead (measured: faster up to about SMs / 3 chains).
-    if (batch * p->H * 3 <= ctx->sm_count && lasad::prefill_stream_chunks(p->T) >= 2 && ctx->stream_max_ctas > 0)
-        return 3;
+    // Few chains: one CTA per chain would leave most SMs idle.  Long chains (up to SMs / 2 of them)
+    // are cut into segments that run side by side; shorter ones (up to SMs / 3) have their chunks
+    // streamed over all SMs.  The limits are where the measurements cross.
+    const int chunks = lasad::prefill_stream_chunks(p->T);
+    if (batch * p->H * 2 <= ctx->sm_count && chunks >= 16) return 4;
+    if (batch * p->H * 3 <= ctx->sm_count && chunks >= 2 && ctx->stream_max_ctas > 0) return 3;
     return 2;
 }
 
@@ -173,6 +177,7 @@ int lasad_create(lasad_ctx** out, int device)
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) ctx->stream_max_ctas = lasad::prefill_stream_max_ctas(device);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_segstate, (size_t)2 * ctx->sm_count * 64 * 64 * sizeof(float));
     cudaSetDevice(prev);
     if (e == cudaSuccess && reserve_units(ctx, kDefaultRelayUnits) != LASAD_OK) e = cudaErrorMemoryAllocation;
     if (e == cudaSuccess && reserve_redo(ctx, kDefaultRedoUnits) != LASAD_OK) e = cudaErrorMemoryAllocation;
@@ -180,6 +185,7 @@ int lasad_create(lasad_ctx** out, int device)
         if (ctx->d_status) cudaFree(ctx->d_status);
         if (ctx->d_relay) cudaFree(ctx->d_relay);
         if (ctx->d_redo) cudaFree(ctx->d_redo);
+        if (ctx->d_segstate) cudaFree(ctx->d_segstate);
         delete ctx;
         return LASAD_ERR_CUDA;
     }
@@ -193,6 +199,7 @@ int lasad_destroy(lasad_ctx* ctx)
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_relay) cudaFree(ctx->d_relay);
     if (ctx->d_redo) cudaFree(ctx->d_redo);
+    if (ctx->d_segstate) cudaFree(ctx->d_segstate);
     for (int i = 0; i < 2; ++i)
         if (ctx->d_stage[i]) cudaFree(ctx->d_stage[i]);
     if (ctx->d_host_decay) cudaFree(ctx->d_host_decay);
@@ -223,7 +230,7 @@ int lasad_set_option(lasad_ctx* ctx, int option, int value)
     if (!ctx) return LASAD_ERR_INVALID_ARG;
     switch (option) {
         case LASAD_OPT_PREFILL_IMPL:
-            if (value < 0 || value > 3) return LASAD_ERR_INVALID_ARG;
+            if (value < 0 || value > 4) return LASAD_ERR_INVALID_ARG;
             ctx->opt_prefill_impl = value;
             return LASAD_OK;
         case LASAD_OPT_PREFILL_CHUNK:
@@ -292,11 +299,17 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
         ctx->launches += 1;
         return LASAD_OK;
     }
-    if (impl == 2) {
+    if (impl == 2 || impl == 4) {
         if (!tc_ok) return LASAD_ERR_UNSUPPORTED;
+        int launches = 1;
+        if (impl == 4) {
+            a.seg_state = ctx->d_segstate;
+            if (lasad::prefill_tc_segments(lasad::prefill_stream_chunks(p->T), (long long)p->B * p->H, ctx->sm_count) > 1)
+                launches = 3;
+        }
         const cudaError_t e = lasad::launch_prefill_tc(a, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
-        ctx->launches += 1;
+        ctx->launches += launches;
         return LASAD_OK;
     }
     int chunk = ctx->opt_prefill_chunk;

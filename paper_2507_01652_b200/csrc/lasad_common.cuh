@@ -25,6 +25,7 @@ struct KernelArgs {
     const int* widths;      // decode only: [B] grid width of each sequence, or nullptr (grid_w for all)
     int* status;            // device status word (bounded waits report here)
     int* work;              // two device ints, zero between launches: work counter of the persistent prefill
+    float* seg_state;       // prefill, CTA-per-chain kernel: room for 2 x SMs states, or nullptr (chains are not cut)
     unsigned wait_limit;
 };
 
@@ -75,6 +76,8 @@ bool prefill_gated_tc_supported(int dk, int dv, bool bf16);
 cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, int* redo, cudaStream_t st);
 bool prefill_tc_supported(int dk, int dv, bool bf16);
 cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st);
+// segments per chain that launch_prefill_tc cuts the chains into when a.seg_state is given (1: not cut)
+int prefill_tc_segments(int n_chunks, long long chains, int sms);
 
 // What the task-streaming tensor-core prefill needs beyond the caller's buffers: the per-chain
 // relay slots through which the carried state passes from one chunk's CTA to the next chunk's.

@@ -63,8 +63,11 @@ struct __align__(8) Barriers {
     unsigned long long x_ready;    // V~ (normal path) or K~ (exact path) written: dS may start (256 arrivals)
     unsigned long long ds_done;    // dS MMAs complete
     unsigned long long p_ready;    // A/P in TMEM, state copy (and Q~) in smem (256 arrivals)
-    unsigned long long o_done;     // O MMAs complete (and every MMA issued before them)
-    unsigned long long st_ready;   // output tile staged in smem (256 arrivals)
+    // The two barriers the TMA warp waits on exist once per stage: a barrier's next phase then
+    // belongs to the chunk two further on, whose loads the TMA warp issues only after it has seen
+    // this phase, so a one-bit phase parity can never be taken for a later phase's.
+    unsigned long long o_done[kStages];    // O MMAs complete (and every MMA issued before them)
+    unsigned long long st_ready[kStages];  // output tile staged in smem (256 arrivals)
     unsigned long long tbl;        // exact path: the decay table may change / has changed (256 arrivals)
     unsigned long long drain;      // teardown: all MMAs retired
 };
@@ -102,6 +105,11 @@ struct TcParams {
     const float* state_in;
     float* state_out;
     int* work;               // [2], zero between launches: chains drawn beyond the grid size, CTAs that have left
+    // A chain may be cut into n_segs segments of seg_chunks chunks that are computed independently
+    // (work unit = one segment of one chain); a segment then starts from the state
+    // seg_state[segment * B * H + chain], which earlier launches have prepared.  n_segs = 1: whole chains.
+    int seg_chunks, n_segs;
+    const float* seg_state;
     int* status;
     unsigned wait_limit;
 };
@@ -185,6 +193,9 @@ __device__ __forceinline__ ChunkDecay chunk_decay(GridPos& g, int cs, int L, int
 #ifndef LASAD_MINBLOCKS
 #define LASAD_MINBLOCKS 2
 #endif
+// kSegments: work units are segments of chains (see TcParams); false: whole chains, and none of
+// the unit arithmetic below costs anything.
+template <bool kSegments>
 __global__ void __launch_bounds__(kThreads, LASAD_MINBLOCKS)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, TcParams p)
@@ -194,8 +205,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const int n_chunks = (p.T + kC - 1) / kC;
-    const int n_chains = p.B * p.H;
+    // work unit u = segment u / (B H) of chain u % (B H): chunks [first, first + count) of the chain
+    // (everything from the kernel's parameters each time: nothing of it is worth a register)
+    auto unit_chain = [&](int u) { return kSegments ? u % (p.B * p.H) : u; };
+    auto unit_seg = [&](int u) { return kSegments ? u / (p.B * p.H) : 0; };
+    auto unit_first = [&](int u) { return kSegments ? unit_seg(u) * p.seg_chunks : 0; };
+    auto unit_count = [&](int u) {
+        return kSegments ? min(p.seg_chunks, (p.T + kC - 1) / kC - unit_first(u)) : (p.T + kC - 1) / kC;
+    };
     volatile int* abort_flag = &sm.abort_flag;
     volatile int* ring = sm.ring;
     const unsigned limit = p.wait_limit;
@@ -207,8 +224,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_init(&sm.bar.x_ready, kEThreads);
         mbar_init(&sm.bar.ds_done, 1);
         mbar_init(&sm.bar.p_ready, kEThreads);
-        mbar_init(&sm.bar.o_done, 1);
-        mbar_init(&sm.bar.st_ready, kEThreads);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&sm.bar.o_done[s], 1);
+            mbar_init(&sm.bar.st_ready[s], kEThreads);
+        }
         mbar_init(&sm.bar.tbl, kEThreads);
         mbar_init(&sm.bar.drain, 1);
         sm.abort_flag = 0;
@@ -237,19 +256,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // ===================== TMA warp: loads two chunks ahead, stores each output tile =======
         if (elect_one()) {
             // load iterator: (chain, chunk, ordinal) of the next chunk to be loaded
-            int ld_chain = (int)blockIdx.x, ld_n = 0, ld_ord = 0;
-            int ld_b = ld_chain / p.H, ld_h = ld_chain - ld_b * p.H;
+            int ld_unit = (int)blockIdx.x, ld_n = 0, ld_ord = 0;
+            int ld_b = unit_chain(ld_unit) / p.H, ld_h = unit_chain(ld_unit) - ld_b * p.H;
+            int ld_first = unit_first(ld_unit), ld_count = unit_count(ld_unit);
             bool ended = false;            // the end marker has been delivered
             int last_real = -1;            // sequence number of the last chunk whose loads were issued
             auto draw = [&]() {
-                const int c = (int)gridDim.x + atomicAdd(p.work, 1);
-                return c < n_chains ? c : -1;
+                const int u = (int)gridDim.x + atomicAdd(p.work, 1);
+                return u < p.B * p.H * (kSegments ? p.n_segs : 1) ? u : -1;
             };
             // A stage is refilled in two steps: K and V as soon as every MMA of the chunk that used
             // them has retired, Q (whose buffer stages the output tile) once the store has read it.
             auto issue_kv = [&](int g) {
                 const int s = g % kStages;
-                if (ld_chain < 0) {
+                if (ld_unit < 0) {
                     if (!ended) {
                         mbar_arrive(&sm.bar.full[s]);     // completes the phase: the waiters find -1 in the ring
                         ended = true;
@@ -257,21 +277,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     return;
                 }
                 mbar_arrive_expect_tx(&sm.bar.full[s], 3 * kTileBytes);
-                tma_load_4d(sm.k[s], &tm_k, &sm.bar.full[s], 0, ld_h, ld_n * kC, ld_b);
-                tma_load_4d(sm.v[s], &tm_v, &sm.bar.full[s], 0, ld_h, ld_n * kC, ld_b);
+                tma_load_4d(sm.k[s], &tm_k, &sm.bar.full[s], 0, ld_h, (ld_first + ld_n) * kC, ld_b);
+                tma_load_4d(sm.v[s], &tm_v, &sm.bar.full[s], 0, ld_h, (ld_first + ld_n) * kC, ld_b);
                 last_real = g;
             };
             auto issue_q = [&](int g) {
-                if (ld_chain < 0) return;
+                if (ld_unit < 0) return;
                 const int s = g % kStages;
-                tma_load_4d(sm.q[s], &tm_q, &sm.bar.full[s], 0, ld_h, ld_n * kC, ld_b);
-                if (++ld_n == n_chunks) {
+                tma_load_4d(sm.q[s], &tm_q, &sm.bar.full[s], 0, ld_h, (ld_first + ld_n) * kC, ld_b);
+                if (++ld_n == ld_count) {
                     ld_n = 0;
                     ++ld_ord;
-                    ld_chain = draw();
-                    ring[ld_ord & 3] = ld_chain;
-                    ld_b = ld_chain / p.H;
-                    ld_h = ld_chain - ld_b * p.H;
+                    ld_unit = draw();
+                    ring[ld_ord & 3] = ld_unit;
+                    if (ld_unit >= 0) {
+                        ld_b = unit_chain(ld_unit) / p.H;
+                        ld_h = unit_chain(ld_unit) - ld_b * p.H;
+                        ld_first = unit_first(ld_unit);
+                        ld_count = unit_count(ld_unit);
+                    }
                 }
             };
             for (int g = 0; g < kStages; ++g) {
@@ -279,27 +303,32 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 issue_q(g);
             }
             // store iterator: the chunk whose output tile leaves next
-            int st_chain = (int)blockIdx.x, st_n = 0, st_ord = 0;
-            int st_b = st_chain / p.H, st_h = st_chain - st_b * p.H;
-            for (int g = 0; st_chain >= 0; ++g) {
+            int st_unit = (int)blockIdx.x, st_n = 0, st_ord = 0;
+            int st_b = unit_chain(st_unit) / p.H, st_h = unit_chain(st_unit) - st_b * p.H;
+            int st_first = unit_first(st_unit), st_count = unit_count(st_unit);
+            for (int g = 0; st_unit >= 0; ++g) {
                 const int s = g % kStages;
-                if (!mbar_wait(&sm.bar.o_done, g & 1, limit, abort_flag, p.status)) break;
+                if (!mbar_wait(&sm.bar.o_done[s], (g / kStages) & 1, limit, abort_flag, p.status)) break;
                 issue_kv(g + kStages);
                 // the output tile of chunk g sits in the Q buffer of its stage
-                const bool staged = mbar_wait(&sm.bar.st_ready, g & 1, limit, abort_flag, p.status);
+                const bool staged = mbar_wait(&sm.bar.st_ready[s], (g / kStages) & 1, limit, abort_flag, p.status);
                 if (staged) {
-                    tma_store_4d(&tm_o, sm.q[s], 0, st_h, st_n * kC, st_b);
+                    tma_store_4d(&tm_o, sm.q[s], 0, st_h, (st_first + st_n) * kC, st_b);
                     tma_store_commit();
-                    if (ld_chain >= 0) tma_store_wait_read();  // the store has finished reading the buffer
+                    if (ld_unit >= 0) tma_store_wait_read();   // the store has finished reading the buffer
                 }
                 issue_q(g + kStages);                          // (also after a failed wait: the stage's barrier must complete)
                 if (!staged) break;
-                if (++st_n == n_chunks) {
+                if (++st_n == st_count) {
                     st_n = 0;
                     ++st_ord;
-                    st_chain = ring[st_ord & 3];               // published by this thread when the loads reached it
-                    st_b = st_chain / p.H;
-                    st_h = st_chain - st_b * p.H;
+                    st_unit = ring[st_ord & 3];                // published by this thread when the loads reached it
+                    if (st_unit >= 0) {
+                        st_b = unit_chain(st_unit) / p.H;
+                        st_h = unit_chain(st_unit) - st_b * p.H;
+                        st_first = unit_first(st_unit);
+                        st_count = unit_count(st_unit);
+                    }
                 }
             }
             tma_store_wait_all();
@@ -321,7 +350,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const uint64_t dq0 = make_desc(smem_u32(sm.q[0])), dq1 = make_desc(smem_u32(sm.q[1]));
         const uint64_t dk0 = make_desc(smem_u32(sm.k[0])), dk1 = make_desc(smem_u32(sm.k[1]));
         const uint64_t dv0 = make_desc(smem_u32(sm.v[0])), dv1 = make_desc(smem_u32(sm.v[1]));
-        int m_n = 0, m_ord = 0;           // chunk within its chain and chain ordinal of the chunk whose scores come next
+        int m_n = 0, m_ord = 0;           // chunk within its unit and unit ordinal of the chunk whose scores come next
+        int m_count = 1;                  // chunks of that unit
         bool fast_next = true;            // path of that chunk's chain
         // waits for chunk g's tiles, finds out whose they are and issues its score MMAs;
         // 0 = issued, 1 = the work has run out, -1 = a wait gave up
@@ -330,11 +360,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const uint64_t dqs = s ? dq1 : dq0, dks = s ? dk1 : dk0;
             if (!mbar_wait(&sm.bar.full[s], (g / kStages) & 1, limit, abort_flag, p.status)) return -1;
             if (m_n == 0) {
-                const int chain = ring[m_ord & 3];
-                if (chain < 0) return 1;
-                fast_next = p.decay[chain % p.H] >= kFastPathMinDecay;
+                const int u = ring[m_ord & 3];
+                if (u < 0) return 1;
+                fast_next = p.decay[unit_chain(u) % p.H] >= kFastPathMinDecay;
+                m_count = unit_count(u);
             }
-            if (++m_n == n_chunks) {
+            if (++m_n == m_count) {
                 m_n = 0;
                 ++m_ord;
             }
@@ -387,7 +418,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int kk = 0; kk < kD / 16; ++kk)
                         mma_ss(tmem + kColO, dqs + 2 * kk, d_sb + 128 * kk, idesc_qs, 1);
                 }
-                mma_commit(&sm.bar.o_done);
+                mma_commit(&sm.bar.o_done[s]);
             }
             __syncwarp();
             TRACE_M(8 * g + 3);
@@ -460,41 +491,64 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         bool ok = true;
         int g = 0;                      // chunks of this CTA's sequence done so far
         unsigned tbl_phase = 0;         // completed phases of the table barrier
-        int chain = (int)blockIdx.x;
+        int cur_unit = (int)blockIdx.x;
         for (int ord = 0; ok; ++ord) {
-            // ---- next chain: its index is in the ring once the tiles of its first chunk are in ----
+            // ---- next unit: its index is in the ring once the tiles of its first chunk are in -----
             if (!(ok = mbar_wait(&sm.bar.full[g % kStages], (g / kStages) & 1, limit, abort_flag, p.status))) break;
-            if (ord > 0) chain = ring[ord & 3];
-            if (chain < 0) break;
+            if (ord > 0) cur_unit = ring[ord & 3];
+            if (cur_unit < 0) break;
+            const int chain = unit_chain(cur_unit);
+            const int first = unit_first(cur_unit);
+            const int T_here = kSegments ? min(unit_count(cur_unit) * kC, p.T - first * kC) : p.T;   // tokens of this unit
+            const int n_here = (T_here + kC - 1) / kC;
             const int h = chain % p.H;
-            const size_t unit = (size_t)chain * kD * kD;
             const float gamma = p.decay[h];
             const bool fast = gamma >= kFastPathMinDecay;
             const float lg = fast ? log2f(gamma) : 0.0f;
-            // position of the call's first token relative to the grid (SAD rule, Section 3.4)
-            GridPos gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0, lane);
+            // position of the unit's first token relative to the grid (SAD rule, Section 3.4)
+            GridPos gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0 + (long long)first * kC, lane);
+            {
+                // the state the unit starts from: the caller's (or zero) for a whole chain, the prepared
+                // one for a segment (also for a chain's first: state_out may alias state_in, and the
+                // chain's last segment may be done before its first has started)
+                const float* sin = nullptr;
+                if (kSegments)
+                    sin = p.seg_state + ((size_t)unit_seg(cur_unit) * (p.B * p.H) + chain) * kD * kD;
+                else if (p.state_in)
+                    sin = p.state_in + (size_t)chain * kD * kD;
 #pragma unroll
-            for (int e = 0; e < 16; ++e) st[e] = 0.0f;
-            if (p.state_in) {
+                for (int e = 0; e < 16; ++e) st[e] = 0.0f;
+                if (sin) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float2 a = *reinterpret_cast<const float2*>(p.state_in + unit + (size_t)r0 * kD + c0 + 8 * k);
-                    const float2 c = *reinterpret_cast<const float2*>(p.state_in + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k);
-                    st[4 * k] = a.x; st[4 * k + 1] = a.y; st[4 * k + 2] = c.x; st[4 * k + 3] = c.y;
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 a = *reinterpret_cast<const float2*>(sin + (size_t)r0 * kD + c0 + 8 * k);
+                        const float2 c = *reinterpret_cast<const float2*>(sin + (size_t)(r0 + 8) * kD + c0 + 8 * k);
+                        st[4 * k] = a.x; st[4 * k + 1] = a.y; st[4 * k + 2] = c.x; st[4 * k + 3] = c.y;
+                    }
                 }
             }
+            // the final state leaves with a chain's last segment only
+            auto state_leaves = [&]() {
+                if (!p.state_out || unit_first(cur_unit) + unit_count(cur_unit) != (p.T + kC - 1) / kC) return;
+                float* dst = p.state_out + (size_t)unit_chain(cur_unit) * kD * kD;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    *reinterpret_cast<float2*>(dst + (size_t)r0 * kD + c0 + 8 * k) = make_float2(st[4 * k], st[4 * k + 1]);
+                    *reinterpret_cast<float2*>(dst + (size_t)(r0 + 8) * kD + c0 + 8 * k) = make_float2(st[4 * k + 2], st[4 * k + 3]);
+                }
+            };
 
             if (fast) {
                 // ------------------------------- normal path ---------------------------------------
                 // gamma^m straight from ex2.approx: |m log2 gamma| <= 95, relative error ~1e-5, far
                 // below what bf16 I/O resolves
                 auto gpow = [&](int m) { return ex2_approx((float)m * lg); };
-                ChunkDecay cd = chunk_decay(gp, 0, min(kC, p.T), qd, lane);
+                ChunkDecay cd = chunk_decay(gp, 0, min(kC, T_here), qd, lane);
                 write_state_bf16(gpow(cd.n_last));
                 scale_row_inplace<4>(sm.v[g % kStages] + i * 128, gpow(cd.n_last - cd.ni), 4 * grp, i & 7);
                 fence_proxy_async();
                 mbar_arrive(&sm.bar.x_ready);
-                for (int n = 0; ok && n < n_chunks; ++n, ++g) {
+                for (int n = 0; ok && n < n_here; ++n, ++g) {
                     const int s = g % kStages;
                     TRACE_E(8 * g + 0);
                     if (!(ok = mbar_wait(&sm.bar.s_done, g & 1, limit, abort_flag, p.status))) break;
@@ -539,30 +593,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     tc_fence_after();
                     update_state(gpow(cd.n_last));
                     TRACE_E(8 * g + 3);
-                    const bool more = n + 1 < n_chunks;
+                    const bool more = n + 1 < n_here;
                     if (more) {
                         const int cs1 = (n + 1) * kC;
-                        cd = chunk_decay(gp, cs1, min(kC, p.T - cs1), qd, lane);
-                    } else if (p.state_out) {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            *reinterpret_cast<float2*>(p.state_out + unit + (size_t)r0 * kD + c0 + 8 * k) =
-                                make_float2(st[4 * k], st[4 * k + 1]);
-                            *reinterpret_cast<float2*>(p.state_out + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k) =
-                                make_float2(st[4 * k + 2], st[4 * k + 3]);
-                        }
+                        cd = chunk_decay(gp, cs1, min(kC, T_here - cs1), qd, lane);
+                    } else {
+                        state_leaves();
                     }
                     TRACE_E(8 * g + 4);
 
                     // ---- E2: o_i = scale * gamma^-(N - n_i) * O'_i ------------------------------------
-                    if (!(ok = mbar_wait(&sm.bar.o_done, g & 1, limit, abort_flag, p.status))) break;
+                    if (!(ok = mbar_wait(&sm.bar.o_done[s], (g / kStages) & 1, limit, abort_flag, p.status))) break;
                     tc_fence_after();
                     TRACE_E(8 * g + 5);
                     stage_output(s, out_f);
                     if (more) write_state_bf16(gpow(cd.n_last));   // gamma^N(next) * S_new
                     fence_proxy_async();
                     tc_fence_before();
-                    mbar_arrive(&sm.bar.st_ready);
+                    mbar_arrive(&sm.bar.st_ready[s]);
                     TRACE_E(8 * g + 6);
 
                     // ---- V~ of the chain's next chunk, once its loads have landed.  This stage is
@@ -595,10 +643,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (!(ok = mbar_wait(&sm.bar.tbl, tbl_phase & 1, limit, abort_flag, p.status))) break;
                 ++tbl_phase;
                 write_state_bf16(1.0f);
-                for (int n = 0; ok && n < n_chunks; ++n, ++g) {
+                for (int n = 0; ok && n < n_here; ++n, ++g) {
                     const int s = g % kStages;
                     const int cs = n * kC;
-                    const ChunkDecay cd = chunk_decay(gp, cs, min(kC, p.T - cs), qd, lane);
+                    const ChunkDecay cd = chunk_decay(gp, cs, min(kC, T_here - cs), qd, lane);
                     if (n > 0 &&
                         !(ok = mbar_wait(&sm.bar.full[s], (g / kStages) & 1, limit, abort_flag, p.status))) break;
                     if (!(ok = mbar_wait(&sm.bar.s_done, g & 1, limit, abort_flag, p.status))) break;
@@ -639,22 +687,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     if (!(ok = mbar_wait(&sm.bar.ds_done, g & 1, limit, abort_flag, p.status))) break;
                     tc_fence_after();
                     update_state(sm.pw[cd.n_last]);
-                    if (n + 1 == n_chunks && p.state_out) {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            *reinterpret_cast<float2*>(p.state_out + unit + (size_t)r0 * kD + c0 + 8 * k) =
-                                make_float2(st[4 * k], st[4 * k + 1]);
-                            *reinterpret_cast<float2*>(p.state_out + unit + (size_t)(r0 + 8) * kD + c0 + 8 * k) =
-                                make_float2(st[4 * k + 2], st[4 * k + 3]);
-                        }
-                    }
-                    if (!(ok = mbar_wait(&sm.bar.o_done, g & 1, limit, abort_flag, p.status))) break;
+                    if (n + 1 >= n_here) state_leaves();
+                    if (!(ok = mbar_wait(&sm.bar.o_done[s], (g / kStages) & 1, limit, abort_flag, p.status))) break;
                     tc_fence_after();
                     stage_output(s, p.scale);
-                    if (n + 1 < n_chunks) write_state_bf16(1.0f);
+                    if (n + 1 < n_here) write_state_bf16(1.0f);
                     fence_proxy_async();
                     tc_fence_before();
-                    mbar_arrive(&sm.bar.st_ready);
+                    mbar_arrive(&sm.bar.st_ready[s]);
                 }
             }
         }
@@ -679,6 +719,212 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Few chains, long sequences: the chains are cut into segments that run side by side.
+//
+// The SAD recurrence (Section 3.4) is linear in the state, so over a segment [a, b) of a chain
+//     S_b = gamma^(decaying steps in [a, b)) S_a + L,     L = the state the segment reaches from zero.
+// First launch (below): L for every segment but a chain's last, from K and V alone (the dS MMAs
+// of the main kernel and nothing else).  Second launch: S_a for every segment, an element-wise
+// scan over a chain's segments.  Third launch: the main kernel with one work unit per segment.
+// ---------------------------------------------------------------------------------------------
+struct StateSmem {
+    unsigned char k[kStages][kTileBytes];
+    unsigned char v[kStages][kTileBytes];
+    float pw[kC + 4];               // exact path: gamma^m, m = 0..128
+    unsigned long long full[kStages];
+    unsigned long long x_ready;     // V~ (normal path) or K~ (exact path) written (256 arrivals)
+    unsigned long long ds_done[kStages];   // dS MMAs of the stage's chunk complete (per stage: see Barriers)
+    unsigned long long drain;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+constexpr int kStateTmemCols = 64;
+
+__global__ void __launch_bounds__(kThreads, 2)
+prefill_seg_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, TcParams p,
+                         float* seg_state)
+{
+    extern __shared__ unsigned char smem_raw[];
+    StateSmem& sm = *reinterpret_cast<StateSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int n_chains = p.B * p.H;
+    const int seg = blockIdx.x / n_chains, chain = blockIdx.x - seg * n_chains;   // seg < n_segs - 1
+    const int b = chain / p.H, h = chain - b * p.H;
+    const int first = seg * p.seg_chunks, n_here = p.seg_chunks;                  // only a last segment is shorter
+    volatile int* abort_flag = &sm.abort_flag;
+    const unsigned limit = p.wait_limit;
+    const float gamma = p.decay[h];
+    const bool fast = gamma >= kFastPathMinDecay;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(&sm.full[s], 1);
+        mbar_init(&sm.x_ready, kEThreads);
+        for (int s = 0; s < kStages; ++s) mbar_init(&sm.ds_done[s], 1);
+        mbar_init(&sm.drain, 1);
+        sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 8) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
+                     "r"(kStateTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (!fast && tid <= kC) {
+        double base = (double)gamma, acc = 1.0;
+        for (int e = tid; e > 0; e >>= 1) {
+            if (e & 1) acc *= base;
+            base *= base;
+        }
+        sm.pw[tid] = (float)acc;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    if (warp == 9) {
+        if (elect_one()) {
+            auto issue = [&](int n) {
+                const int s = n % kStages;
+                mbar_arrive_expect_tx(&sm.full[s], 2 * kTileBytes);
+                tma_load_4d(sm.k[s], &tm_k, &sm.full[s], 0, h, (first + n) * kC, b);
+                tma_load_4d(sm.v[s], &tm_v, &sm.full[s], 0, h, (first + n) * kC, b);
+            };
+            int issued = min(n_here, kStages);
+            for (int n = 0; n < issued; ++n) issue(n);
+            for (int n = 0; n + kStages < n_here; ++n) {
+                if (!mbar_wait(&sm.ds_done[n % kStages], (n / kStages) & 1, limit, abort_flag, p.status)) break;
+                issue(n + kStages);
+                issued = n + kStages + 1;
+            }
+            // leave only when every issued load has landed (they write this CTA's shared memory)
+            for (int n = max(0, issued - kStages); n < issued; ++n)
+                for (unsigned it = 0; it < kTeardownLimit; ++it)
+                    if (mbar_try_wait(&sm.full[n % kStages], (n / kStages) & 1)) break;
+        }
+        __syncwarp();
+    } else if (warp == 8) {
+        constexpr uint32_t idesc_kv = make_idesc(64, 64, 1, 1);    // K^T (MN-major) x V (MN-major)
+        const uint64_t dk0 = make_desc(smem_u32(sm.k[0])), dk1 = make_desc(smem_u32(sm.k[1]));
+        const uint64_t dv0 = make_desc(smem_u32(sm.v[0])), dv1 = make_desc(smem_u32(sm.v[1]));
+        for (int n = 0; n < n_here; ++n) {
+            const int s = n % kStages;
+            const uint64_t dks = s ? dk1 : dk0, dvs = s ? dv1 : dv0;
+            if (!mbar_wait(&sm.full[s], (n / kStages) & 1, limit, abort_flag, p.status)) break;
+            if (!mbar_wait(&sm.x_ready, n & 1, limit, abort_flag, p.status)) break;
+            tc_fence_after();
+            if (elect_one()) {
+#pragma unroll
+                for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K and of V per step
+                    mma_ss(tmem, dks + 128 * kk, dvs + 128 * kk, idesc_kv, kk > 0);
+                mma_commit(&sm.ds_done[s]);
+            }
+            __syncwarp();
+        }
+        if (elect_one()) {
+            mma_commit(&sm.drain);
+            for (unsigned it = 0; it < kTeardownLimit; ++it)
+                if (mbar_try_wait(&sm.drain, 0)) break;
+        }
+        __syncwarp();
+    } else {
+        const int qd = warp & 3, grp = warp >> 2;
+        const int i = qd * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+        const int r0 = qd * 16 + (lane >> 2);
+        const int c0 = 32 * grp + 2 * (lane & 3);
+        GridPos gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0 + (long long)first * kC, lane);
+        const float lg = fast ? log2f(gamma) : 0.0f;
+        float st[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) st[e] = 0.0f;
+        bool ok = true;
+        for (int n = 0; ok && n < n_here; ++n) {
+            const int s = n % kStages;
+            const ChunkDecay cd = chunk_decay(gp, n * kC, kC, qd, lane);     // (full chunks: not a chain's last segment)
+            if (!(ok = mbar_wait(&sm.full[s], (n / kStages) & 1, limit, abort_flag, p.status))) break;
+            float g_chunk;
+            if (fast) {
+                g_chunk = ex2_approx((float)cd.n_last * lg);
+                scale_row_inplace<4>(sm.v[s] + i * 128, ex2_approx((float)(cd.n_last - cd.ni) * lg), 4 * grp, i & 7);
+            } else {
+                g_chunk = sm.pw[cd.n_last];
+                if (grp == 1) scale_row_inplace<8>(sm.k[s] + i * 128, sm.pw[cd.n_last - cd.ni], 0, i & 7);
+            }
+            fence_proxy_async();
+            mbar_arrive(&sm.x_ready);
+            if (!(ok = mbar_wait(&sm.ds_done[s], (n / kStages) & 1, limit, abort_flag, p.status))) break;
+            tc_fence_after();
+            uint32_t dsv[16];
+            tmem_ld_16x256b_x4(tmem + lane_base + 32 * grp, dsv);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; e += 2)
+                fma2(st[e], st[e + 1], g_chunk, __uint_as_float(dsv[e]), __uint_as_float(dsv[e + 1]), st[e], st[e + 1]);
+            tc_fence_before();
+        }
+        if (ok) {
+            float* dst = seg_state + ((size_t)(seg + 1) * n_chains + chain) * kD * kD;    // scanned in place later
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                *reinterpret_cast<float2*>(dst + (size_t)r0 * kD + c0 + 8 * k) = make_float2(st[4 * k], st[4 * k + 1]);
+                *reinterpret_cast<float2*>(dst + (size_t)(r0 + 8) * kD + c0 + 8 * k) = make_float2(st[4 * k + 2], st[4 * k + 3]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kStateTmemCols) : "memory");
+    }
+}
+
+// seg_state[s + 1] holds L of segment s on entry; on exit seg_state[s] is the state at the start of
+// segment s (seg_state[0]: the caller's incoming state or zero).  One thread per state element, a
+// chain's segments in order; the loads of a batch of segments are issued together, only the
+// multiply-adds are serial.  steps[s] = decaying steps among segment s's tokens (SAD rule, Section
+// 3.4), the same for every chain, counted on the host.
+constexpr int kMaxSegs = 320;
+struct SegSteps {
+    int n[kMaxSegs];
+};
+
+__global__ void __launch_bounds__(256)
+prefill_seg_scan_kernel(TcParams p, SegSteps steps, float* seg_state)
+{
+    constexpr int kBatch = 8;
+    const int per_chain = kD * kD / 256;
+    const int chain = blockIdx.x / per_chain;
+    const int e = (blockIdx.x - chain * per_chain) * 256 + threadIdx.x;
+    const size_t stride = (size_t)p.B * p.H * kD * kD;        // from one segment's slot to the next
+    float* slot = seg_state + (size_t)chain * kD * kD + e;
+    const float gamma = p.decay[chain % p.H];
+    const float lg = gamma > 0.0f ? log2f(gamma) : 0.0f;
+    float carry = p.state_in ? p.state_in[(size_t)chain * kD * kD + e] : 0.0f;
+    slot[0] = carry;
+    for (int s0 = 0; s0 + 1 < p.n_segs; s0 += kBatch) {
+        float loc[kBatch];
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j)
+            loc[j] = s0 + j + 1 < p.n_segs ? slot[(size_t)(s0 + j + 1) * stride] : 0.0f;
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            if (s0 + j + 1 < p.n_segs) {
+                const int n = steps.n[s0 + j];
+                const float g = n == 0 ? 1.0f : gamma > 0.0f ? exp2f((float)n * lg) : 0.0f;
+                carry = fmaf(g, carry, loc[j]);
+                slot[(size_t)(s0 + j + 1) * stride] = carry;
+            }
+        }
+    }
+}
+
 }  // namespace
 
 #ifdef LASAD_TC_TRACE
@@ -689,6 +935,17 @@ extern "C" int lasad_debug_read_trace(long long* host, int n)
 #endif
 
 bool prefill_tc_supported(int dk, int dv, bool bf16) { return bf16 && dk == kD && dv == kD; }
+
+int prefill_tc_segments(int n_chunks, long long chains, int sms)
+{
+    // as many segments as there are CTA slots per chain, each of at least two chunks
+    long long segs = chains > 0 ? 2LL * sms / chains : 1;
+    if (segs > n_chunks / 2) segs = n_chunks / 2;
+    if (segs > kMaxSegs) segs = kMaxSegs;
+    if (segs < 2) return 1;
+    const int len = (int)((n_chunks + segs - 1) / segs);
+    return (n_chunks + len - 1) / len;
+}
 
 cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st)
 {
@@ -701,9 +958,12 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st)
     p.grid_w = a.grid_w; p.prefix_len = a.prefix_len; p.t0 = a.t0; p.scale = a.scale;
     p.decay = a.decay; p.state_in = a.state_in; p.state_out = a.state_out;
     p.work = a.work;
+    p.n_segs = 1; p.seg_chunks = (a.T + kC - 1) / kC; p.seg_state = nullptr;
     p.status = a.status; p.wait_limit = a.wait_limit;
     const size_t smem = sizeof(Smem) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // Two CTAs fit on an SM; with more chains than that, the CTAs stay and draw further chains
     // from the work counter, so a chain's first loads overlap the previous chain's last chunk.
@@ -712,8 +972,37 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st)
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
     const long long chains = (long long)a.B * a.H;
-    const unsigned grid = (unsigned)(chains < 2LL * sms ? chains : 2LL * sms);
-    prefill_tc_kernel<<<grid, kThreads, smem, st>>>(mq, mk, mv, mo, p);
+    if (a.seg_state) {
+        // few chains: cut them into segments that run side by side (three launches, see above)
+        const int n_chunks = (a.T + kC - 1) / kC;
+        const int segs = prefill_tc_segments(n_chunks, chains, sms);
+        if (segs > 1) {
+            p.seg_chunks = (n_chunks + segs - 1) / segs;
+            p.n_segs = segs;
+            p.seg_state = a.seg_state;
+            const size_t ssmem = sizeof(StateSmem) + 1024;
+            e = cudaFuncSetAttribute(prefill_seg_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssmem);
+            if (e != cudaSuccess) return e;
+            prefill_seg_state_kernel<<<(unsigned)(chains * (segs - 1)), kThreads, ssmem, st>>>(mk, mv, p, a.seg_state);
+            e = cudaGetLastError();
+            if (e != cudaSuccess) return e;
+            SegSteps steps;
+            for (int sg = 0; sg + 1 < segs; ++sg) {
+                const long long lo = a.t0 + (long long)sg * p.seg_chunks * kC, hi = lo + (long long)p.seg_chunks * kC;
+                steps.n[sg] = (int)(decay_steps_upto(hi - 1, a.grid_w, a.prefix_len) -
+                                    decay_steps_upto(lo - 1, a.grid_w, a.prefix_len));
+            }
+            prefill_seg_scan_kernel<<<(unsigned)(chains * (kD * kD / 256)), 256, 0, st>>>(p, steps, a.seg_state);
+            e = cudaGetLastError();
+            if (e != cudaSuccess) return e;
+        }
+    }
+    const long long units = chains * p.n_segs;
+    const unsigned grid = (unsigned)(units < 2LL * sms ? units : 2LL * sms);
+    if (p.n_segs > 1)
+        prefill_tc_kernel<true><<<grid, kThreads, smem, st>>>(mq, mk, mv, mo, p);
+    else
+        prefill_tc_kernel<false><<<grid, kThreads, smem, st>>>(mq, mk, mv, mo, p);
     return cudaGetLastError();
 }
 

@@ -14,7 +14,8 @@ from tests._util import TOL, oracle, rel_err, to64
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = [1, 2, 3]  # 1 = CUDA-core fp32 kernel, 2 = tcgen05 kernel (CTA per chain), 3 = tcgen05 task-streaming kernel
+IMPLS = [1, 2, 3, 4]  # 1 = CUDA-core fp32 kernel, 2 = tcgen05 kernel (CTA per chain), 3 = tcgen05 task-streaming kernel,
+                      # 4 = as 2, few long chains cut into segments
 
 
 @pytest.fixture(scope="module")
@@ -274,6 +275,29 @@ def test_more_chains_than_resident_ctas(ctx, T):
     o, s = _forward(ctx, 2, dq[:2], dk[:2], dv[:2], dg, w, t0=3, scale=0.5, state_in=ds[:2])
     assert rel_err(o, o_ref[:2]) <= TOL[torch.bfloat16]
     assert rel_err(s, s_ref[:2]) <= TOL[torch.bfloat16]
+
+
+@pytest.mark.parametrize("B,H,T", [(1, 5, 2000), (2, 12, 1500), (1, 1, 9216), (3, 16, 1153)])
+def test_few_long_chains_cut_into_segments(ctx, B, H, T):
+    """Implementation 4: a first launch gets every segment's own contribution to the state from K and
+    V, a scan hands every segment its starting state, and the segments then run side by side.
+    Ragged last chunk, heads on both decay paths, an incoming state, a prefix token, a start in
+    mid-row, state_out aliasing state_in; twice in a row."""
+    d, w = 64, 13
+    gen = torch.Generator().manual_seed(900 + T)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+    g = 0.9 + 0.0999 * torch.rand(H, generator=gen)
+    g[0] = 0.45
+    if H > 3:
+        g[1], g[2], g[3] = 0.0, 1.0, 0.59
+    s_in = torch.randn(B, H, d, d, generator=gen)
+    o_ref, s_ref = oracle(q, k, v, g, w, 1, 5, 0.5, s_in)
+    dq, dk, dv, dg = _dev(q, k, v, g)
+    for rep in range(2):
+        ds = s_in.cuda()
+        o, s = _forward(ctx, 4, dq, dk, dv, dg, w, prefix_len=1, t0=5, scale=0.5, state_in=ds, state_out=ds)
+        assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+        assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
 
 
 def test_default_prefill_picks_a_kernel_by_the_number_of_chains(ctx):

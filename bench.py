@@ -272,7 +272,7 @@ def run_ours(args):
     # ---- the other prefill configurations (context for the headline; rank 0 reports) ----------
     sweep = None
     if args.only == "all" and not args.no_sweep:
-        sweep = prefill_sweep(ctx, peaks, dev, ("config1", "config2", "config3", "config5a"))
+        sweep = prefill_sweep(ctx, peaks, dev, ("config1", "config2", "config3", "config5a", "config5b@1"))
     gated = None
     if args.only == "all" and not args.no_sweep:
         gated = gated_sweep(ctx, peaks, dev)
@@ -333,7 +333,10 @@ def prefill_sweep(ctx, peaks, dev, names, reps: int = 10):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     out = []
     for name in names:
-        wl = workloads.WORKLOADS[name]
+        # "name@B": the named workload at another batch size (e.g. one image at a time)
+        wl = workloads.WORKLOADS[name.split("@")[0]]
+        if "@" in name:
+            wl = wl.scaled(B=int(name.split("@")[1]))
         q, k, v = [t.to(dev) for t in workloads.make_qkv(wl)]
         g = workloads.make_decay(wl).to(dev)
         o = torch.empty_like(v)

@@ -90,7 +90,9 @@ struct __align__(8) Barriers {
     unsigned long long p_ready;    // A/P in TMEM (and Q~ in smem) (256 arrivals)
     unsigned long long sb_ready;   // bf16 copy of the incoming state in smem (256 arrivals)
     unsigned long long o_done;     // O MMAs complete (and every MMA issued before them)
-    unsigned long long st_ready;   // output tile staged in smem (256 arrivals)
+    // one per stage: its next phase is the task two further on, whose loads the TMA warp issues only
+    // after it has seen this phase, so the one-bit phase parity is never taken for a later phase's
+    unsigned long long st_ready[kStages];   // output tile staged in smem (256 arrivals)
     unsigned long long tbl_free;   // exact path: every thread is done with the current table (256)
     unsigned long long tbl_ready;  // exact path: the table of this task's head is written (256)
     unsigned long long drain;      // teardown: all MMAs retired
@@ -249,7 +251,7 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         mbar_init(&sm.bar.p_ready, kEThreads);
         mbar_init(&sm.bar.sb_ready, kEThreads);
         mbar_init(&sm.bar.o_done, 1);
-        mbar_init(&sm.bar.st_ready, kEThreads);
+        for (int s = 0; s < kStages; ++s) mbar_init(&sm.bar.st_ready[s], kEThreads);
         mbar_init(&sm.bar.tbl_free, kEThreads);
         mbar_init(&sm.bar.tbl_ready, kEThreads);
         mbar_init(&sm.bar.drain, 1);
@@ -291,7 +293,7 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 const int s = g % kStages;
                 // the output tile of task g sits in the Q buffer of its stage; by now every MMA
                 // that read this stage has retired (the element-wise warps waited for o_done)
-                if (!mbar_wait(&sm.bar.st_ready, g & 1, limit, abort_flag, p.status)) break;
+                if (!mbar_wait(&sm.bar.st_ready[s], (g / kStages) & 1, limit, abort_flag, p.status)) break;
                 const Task t = decode_task(first + g * G, p.X, p.H);
                 tma_store_4d(&tm_o, sm.q[s], 0, t.h, t.n * kC, t.b);
                 tma_store_commit();
@@ -682,7 +684,7 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             stage_output(s, out_f);
             fence_proxy_async();
             tc_fence_before();
-            mbar_arrive(&sm.bar.st_ready);
+            mbar_arrive(&sm.bar.st_ready[s]);
             TRACE_E(7);
 
             // ---- next task of this CTA -----------------------------------------------------------

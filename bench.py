@@ -32,8 +32,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) from the ncu captures
 # summarised under profiles/; None until a capture of that kernel exists.
 NCU_TRAFFIC_BYTES = {
-    # prefill_tc_kernel: 578.8 MB measured on the 608.7 MB capture case, scaled by tokens to config 5b
-    "prefill": 864_400_000,
+    # prefill_tc_kernel: 577.3 MB measured on the 608.7 MB capture case, scaled by tokens to config 5b
+    "prefill": 862_200_000,
     # decode_kernel, config 4, inside the kernel (the rest of the written state drains from L2 later)
     "decode": 111_900_000,
 }

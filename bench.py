@@ -35,7 +35,7 @@ NCU_TRAFFIC_BYTES = {
     # prefill_tc_kernel: 577.3 MB measured on the 608.7 MB capture case, scaled by tokens to config 5b
     "prefill": 862_200_000,
     # decode_kernel, config 4, inside the kernel (the rest of the written state drains from L2 later)
-    "decode": 111_900_000,
+    "decode": 112_200_000,
 }
 
 

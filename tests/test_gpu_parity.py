@@ -382,9 +382,12 @@ def test_streaming_prefill_launch_counter_wraps(ctx):
 # ------------------------------------------------------------------------------------------
 # host-buffer entry point: the pipelined copies must not change the result
 # ------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("dtype,d,B", [(torch.bfloat16, 64, 5), (torch.float32, 32, 3), (torch.bfloat16, 64, 1)])
-def test_forward_host_equals_device_path(ctx, dtype, d, B):
-    T, H, w, P = 333, 3, 12, 1
+@pytest.mark.parametrize("dtype,d,B,T", [(torch.bfloat16, 64, 5, 333), (torch.float32, 32, 3, 333),
+                                         (torch.bfloat16, 64, 1, 333), (torch.bfloat16, 64, 3, 2100)])
+def test_forward_host_equals_device_path(ctx, dtype, d, B, T):
+    """(T = 333 with few chains runs the task-streaming kernel under the default option, T = 2100 the
+    segment-parallel mode: the host entry point must take the same one as the device entry point.)"""
+    H, w, P = 3, 12, 1
     gen = torch.Generator().manual_seed(41 + B)
     q, k, v = [(torch.randn(B, T, H, d, generator=gen) / d ** 0.5).to(dtype).pin_memory() for _ in range(3)]
     g = torch.tensor([0.9, 0.97, 0.999]).pin_memory()

@@ -433,7 +433,7 @@ def test_decode_per_sequence_positions_and_widths(ctx):
 # ------------------------------------------------------------------------------------------
 # bounded waits: a wait that runs out is reported, nothing hangs, the context stays usable
 # ------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("impl", [2, 3])
+@pytest.mark.parametrize("impl", [2, 3, 4])
 def test_expired_device_wait_is_reported_and_context_survives(ctx, impl):
     """With the poll limit of the device-side waits set to 1, some wait runs out before its
     barrier completes: the kernel must leave through its normal exit, the status word must say

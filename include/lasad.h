@@ -55,8 +55,9 @@ enum { LASAD_F32 = 0, LASAD_BF16 = 1 };
 
 /* Options for lasad_set_option. */
 enum {
-    LASAD_OPT_PREFILL_IMPL = 0, /* 0 auto (bf16, d = 64: 4 when B * H <= SMs / 2 and T > 1920, else 3
-                                   when B * H <= SMs / 3 and T > 128, else 2; other shapes 1),
+    LASAD_OPT_PREFILL_IMPL = 0, /* 0 auto (bf16, d = 64: 4 when B * H <= SMs / 3 and T > 1920 or
+                                   B * H <= SMs / 2 and T > 3968, else 3 when B * H <= SMs / 3 and
+                                   T > 128, else 2; other shapes 1),
                                    1 CUDA-core fp32 kernel,
                                    2 tcgen05 kernel with one CTA per (batch, head) at a time,
                                    3 tcgen05 kernel streaming (batch, head, chunk) tasks through

@@ -103,12 +103,14 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 int auto_prefill_impl(const lasad_ctx* ctx, const lasad_params* p, int64_t batch, bool tc_ok)
 {
     if (!tc_ok) return 1;
-    // Few chains: one CTA per chain would leave most SMs idle.  Long chains (up to SMs / 2 of them)
-    // are cut into segments that run side by side; shorter ones (up to SMs / 3) have their chunks
-    // streamed over all SMs.  The limits are where the measurements cross.
+    // Few chains: one CTA per chain would leave most SMs idle.  Long chains (16 chunks and up to
+    // SMs / 3 chains, or 32 chunks and up to SMs / 2) are cut into segments that run side by side;
+    // shorter ones (up to SMs / 3) have their chunks streamed over all SMs.  The limits are where
+    // the measurements cross.
     const int chunks = lasad::prefill_stream_chunks(p->T);
-    if (batch * p->H * 2 <= ctx->sm_count && chunks >= 16) return 4;
-    if (batch * p->H * 3 <= ctx->sm_count && chunks >= 2 && ctx->stream_max_ctas > 0) return 3;
+    const int64_t chains = batch * p->H;
+    if ((chains * 3 <= ctx->sm_count && chunks >= 16) || (chains * 2 <= ctx->sm_count && chunks >= 32)) return 4;
+    if (chains * 3 <= ctx->sm_count && chunks >= 2 && ctx->stream_max_ctas > 0) return 3;
     return 2;
 }
 

@@ -455,8 +455,11 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const int piece = ((4 * grp + k) ^ (r0 & 7)) * 16;    // r0 + 8 has the same low bits
-                *reinterpret_cast<uint32_t*>(row0 + piece) = pack_bf16(mult * st[4 * k], mult * st[4 * k + 1]);
-                *reinterpret_cast<uint32_t*>(row0 + 8 * 128 + piece) = pack_bf16(mult * st[4 * k + 2], mult * st[4 * k + 3]);
+                float a0, a1, b0, b1;
+                mul2(st[4 * k], st[4 * k + 1], mult, a0, a1);
+                mul2(st[4 * k + 2], st[4 * k + 3], mult, b0, b1);
+                *reinterpret_cast<uint32_t*>(row0 + piece) = pack_bf16(a0, a1);
+                *reinterpret_cast<uint32_t*>(row0 + 8 * 128 + piece) = pack_bf16(b0, b1);
             }
         };
         // E3: S_new = g * S_prev + dS
@@ -465,7 +468,8 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             tmem_ld_16x256b_x4(tmem + lane_base + kColDS + 32 * grp, dsv);
             tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 16; ++e) st[e] = fmaf(g, st[e], __uint_as_float(dsv[e]));
+            for (int e = 0; e < 16; e += 2)
+                fma2(st[e], st[e + 1], g, __uint_as_float(dsv[e]), __uint_as_float(dsv[e + 1]), st[e], st[e + 1]);
         };
         // E2: this thread's 32 columns of output row i -> bf16 -> the stage's Q buffer
         auto stage_output = [&](int s, float f) {
@@ -477,12 +481,14 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 tmem_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
-                    uint4 x;
-                    x.x = pack_bf16(f * __uint_as_float(ov[8 * c]), f * __uint_as_float(ov[8 * c + 1]));
-                    x.y = pack_bf16(f * __uint_as_float(ov[8 * c + 2]), f * __uint_as_float(ov[8 * c + 3]));
-                    x.z = pack_bf16(f * __uint_as_float(ov[8 * c + 4]), f * __uint_as_float(ov[8 * c + 5]));
-                    x.w = pack_bf16(f * __uint_as_float(ov[8 * c + 6]), f * __uint_as_float(ov[8 * c + 7]));
-                    reinterpret_cast<uint4*>(orow)[(4 * grp + 2 * hh + c) ^ (i & 7)] = x;
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        float r0, r1;
+                        mul2(__uint_as_float(ov[8 * c + 2 * e]), __uint_as_float(ov[8 * c + 2 * e + 1]), f, r0, r1);
+                        w[e] = pack_bf16(r0, r1);
+                    }
+                    reinterpret_cast<uint4*>(orow)[(4 * grp + 2 * hh + c) ^ (i & 7)] = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
         };
@@ -521,9 +527,9 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             const uint32_t tag_in = (p.epoch16 << 16) | ((uint32_t)t.n & 0xffffu);
             const uint32_t tag_out = (p.epoch16 << 16) | ((uint32_t)(t.n + 1) & 0xffffu);
 
-            // gamma^m: normal path straight from exp2 (|m log2 gamma| <= 95, relative error ~1e-5);
+            // gamma^m: normal path straight from ex2.approx (|m log2 gamma| <= 95, relative error ~1e-5);
             // exact path from a table in double precision (0^0 = 1), rebuilt for this task's head
-            auto gpow = [&](int m) { return exp2f((float)m * lg); };
+            auto gpow = [&](int m) { return ex2_approx((float)m * lg); };
             if (!fast) {
                 // every thread is done with the previous exact task's table before it is rewritten
                 if (exact_tasks > 0 &&

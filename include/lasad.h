@@ -111,6 +111,11 @@ int lasad_reserve(lasad_ctx* ctx, int64_t units);
  *   q, k    [B,T,H,dk]  (strided)      decay      [H] fp32, gamma_h in [0,1]
  *   v       [B,T,H,dv]                 state_in   [B,H,dk,dv] fp32 or NULL (zero state)
  *   o       [B,T,H,dv]  written        state_out  [B,H,dk,dv] fp32 or NULL; may alias state_in
+ *
+ * The call may be recorded into a CUDA graph (stream capture) and replayed, with one exception:
+ * prefill implementation 3 numbers its launches on the host, so while `cuda_stream` is being
+ * captured the default never picks it and LASAD_OPT_PREFILL_IMPL = 3 makes the call return
+ * LASAD_ERR_UNSUPPORTED.
  */
 int lasad_forward(lasad_ctx* ctx, const lasad_params* p,
                   const void* q, const void* k, const void* v,

@@ -273,7 +273,19 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
 
     int impl = ctx->opt_prefill_impl;
     const bool tc_ok = lasad::prefill_tc_supported(p->dk, p->dv, bf16);
-    if (impl == 0) impl = auto_prefill_impl(ctx, p, p->B, tc_ok);
+    const bool chosen = impl == 0;
+    if (chosen) impl = auto_prefill_impl(ctx, p, p->B, tc_ok);
+    if (impl == 3) {
+        // The relay packets of this kernel carry the launch's number, which the host counts: a
+        // launch recorded into a CUDA graph would replay with the number it was recorded with and
+        // could take an earlier replay's packets for its own.  During a stream capture the default
+        // therefore falls back to the CTA-per-chain kernel, and an explicit request is refused.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap != cudaStreamCaptureStatusNone) {
+            if (!chosen) return LASAD_ERR_UNSUPPORTED;
+            impl = 2;
+        }
+    }
     if (impl == 3) {
         if (!tc_ok) return LASAD_ERR_UNSUPPORTED;
         const int64_t units = (int64_t)p->B * p->H;

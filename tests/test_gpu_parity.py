@@ -319,6 +319,43 @@ def test_default_prefill_picks_a_kernel_by_the_number_of_chains(ctx):
         assert rel_err(s0, s_ref) <= TOL[torch.bfloat16]
 
 
+@pytest.mark.parametrize("T", [700, 2300])
+def test_prefill_recorded_into_a_cuda_graph_and_replayed(ctx, T):
+    """A prefill call captured into a CUDA graph and replayed on new inputs.  With few chains the
+    default would take the task-streaming kernel (T = 700), whose packets carry a host-side launch
+    number; under capture it must fall back, and asking for that kernel by option must be refused.
+    T = 2300 records the three launches of the segment-parallel mode."""
+    B, H, d, w = 1, 4, 64, 9
+    gen = torch.Generator().manual_seed(77 + T)
+    g = torch.tensor([0.93, 0.5, 0.999, 0.97])
+    dg = g.cuda()
+    dq, dk, dv = [torch.empty(B, T, H, d, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+    o = torch.empty_like(dv)
+    s = torch.empty(B, H, d, d, device="cuda")
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        ctx.lasad_forward(dq, dk, dv, dg, w, o=o, state_out=s)          # warm-up outside the capture
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=stream):
+            ctx.lasad_forward(dq, dk, dv, dg, w, o=o, state_out=s)
+            ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 3)
+            try:
+                with pytest.raises(binding.LasadError):
+                    ctx.lasad_forward(dq, dk, dv, dg, w, o=o, state_out=s)
+            finally:
+                ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
+    for rep in range(3):
+        q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+        dq.copy_(q); dk.copy_(k); dv.copy_(v)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        o_ref, s_ref = oracle(q, k, v, g, w)
+        assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+        assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
+
+
 def test_streaming_prefill_many_heads_and_relay_growth(ctx):
     """More heads than the kernel's shared-memory decay cache holds (H > 256) and more (batch,
     head) pairs than the context's initial relay storage (B * H > 1024, so the call grows it)."""

@@ -165,3 +165,35 @@ def test_gated_state_handoff(ctx):
         torch.cuda.synchronize()
         assert rel_err(torch.cat([o1, o2], 1), o_ref) <= TOL[torch.bfloat16]
         assert rel_err(s2, s_ref) <= TOL[torch.bfloat16]
+
+
+def test_gated_prefill_recorded_into_a_cuda_graph_and_replayed(ctx):
+    """Both launches of the gated prefill (tensor-core kernel, CUDA-core kernel for flagged chains)
+    captured into a CUDA graph and replayed on new inputs; the second replay has a strong-decay
+    stretch, so the replayed CUDA-core launch has chains to redo."""
+    B, T, H, d, w = 2, 300, 3, 64, 10
+    dq, dk, dv, dl = [torch.empty(B, T, H, d, dtype=torch.bfloat16, device="cuda") for _ in range(4)]
+    o = torch.empty_like(dv)
+    s = torch.empty(B, H, d, d, device="cuda")
+    q, k, v, lam = _inputs(31, B, T, H, d, torch.bfloat16)
+    for dst, src in ((dq, q), (dk, k), (dv, v), (dl, lam)):
+        dst.copy_(src)
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        ctx.lasad_forward_gated(dq, dk, dv, dl, w, o=o, state_out=s)     # warm-up outside the capture
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=stream):
+            ctx.lasad_forward_gated(dq, dk, dv, dl, w, o=o, state_out=s)
+    for rep in range(3):
+        q, k, v, lam = _inputs(32 + rep, B, T, H, d, torch.bfloat16)
+        if rep == 1:
+            lam[:, 130:250] = 0.004
+        for dst, src in ((dq, q), (dk, k), (dv, v), (dl, lam)):
+            dst.copy_(src)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        o_ref, s_ref = oracle(q, k, v, lam, w)
+        assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+        assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep

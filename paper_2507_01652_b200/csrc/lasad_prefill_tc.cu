@@ -843,11 +843,12 @@ prefill_seg_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
 #pragma unroll
         for (int e = 0; e < 16; ++e) st[e] = 0.0f;
         bool ok = true;
-        for (int n = 0; ok && n < n_here; ++n) {
+        // scales chunk n's operand (V~ on the normal path, K~ on the exact one) once its tiles are in;
+        // returns gamma^N of the chunk.  (Full chunks: this is never a chain's last segment.)
+        auto prepare = [&](int n, float& g_chunk) {
             const int s = n % kStages;
-            const ChunkDecay cd = chunk_decay(gp, n * kC, kC, qd, lane);     // (full chunks: not a chain's last segment)
-            if (!(ok = mbar_wait(&sm.full[s], (n / kStages) & 1, limit, abort_flag, p.status))) break;
-            float g_chunk;
+            const ChunkDecay cd = chunk_decay(gp, n * kC, kC, qd, lane);
+            if (!mbar_wait(&sm.full[s], (n / kStages) & 1, limit, abort_flag, p.status)) return false;
             if (fast) {
                 g_chunk = ex2_approx((float)cd.n_last * lg);
                 scale_row_inplace<4>(sm.v[s] + i * 128, ex2_approx((float)(cd.n_last - cd.ni) * lg), 4 * grp, i & 7);
@@ -856,7 +857,16 @@ prefill_seg_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 if (grp == 1) scale_row_inplace<8>(sm.k[s] + i * 128, sm.pw[cd.n_last - cd.ni], 0, i & 7);
             }
             fence_proxy_async();
-            mbar_arrive(&sm.x_ready);
+            return true;
+        };
+        float g_chunk = 1.0f;
+        ok = prepare(0, g_chunk);
+        if (ok) mbar_arrive(&sm.x_ready);
+        for (int n = 0; ok && n < n_here; ++n) {
+            const int s = n % kStages;
+            // the next chunk's operand is scaled while this chunk's MMAs run (other stage)
+            float g_next = 1.0f;
+            if (n + 1 < n_here && !(ok = prepare(n + 1, g_next))) break;
             if (!(ok = mbar_wait(&sm.ds_done[s], (n / kStages) & 1, limit, abort_flag, p.status))) break;
             tc_fence_after();
             uint32_t dsv[16];
@@ -866,6 +876,8 @@ prefill_seg_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             for (int e = 0; e < 16; e += 2)
                 fma2(st[e], st[e + 1], g_chunk, __uint_as_float(dsv[e]), __uint_as_float(dsv[e + 1]), st[e], st[e + 1]);
             tc_fence_before();
+            if (n + 1 < n_here) mbar_arrive(&sm.x_ready);     // the accumulator has been read: the next dS may start
+            g_chunk = g_next;
         }
         if (ok) {
             float* dst = seg_state + ((size_t)(seg + 1) * n_chains + chain) * kD * kD;    // scanned in place later

@@ -62,7 +62,7 @@ enum {
                                    2 tcgen05 kernel with one CTA per (batch, head) at a time,
                                    3 tcgen05 kernel streaming (batch, head, chunk) tasks through
                                    persistent CTAs, 4 as 2 with few long sequences cut into segments
-                                   that run side by side (three launches; 2 where nothing is cut)   */
+                                   that run side by side (two launches; 2 where nothing is cut)     */
     LASAD_OPT_PREFILL_CHUNK = 1,/* CUDA-core prefill chunk length: 0 auto, else 16/32/64          */
     LASAD_OPT_DECODE_TPU = 2,   /* decode: threads per (b,h) state; 0 auto, else 32/64/128/256 */
     LASAD_OPT_WAIT_LIMIT = 3    /* iteration cap of device-side waits; 0 = library default   */

@@ -21,7 +21,7 @@ struct lasad_ctx {
     uint64_t epoch;               // launches of the task-streaming prefill so far
     int stream_max_ctas;
     // states at the cuts when the CTA-per-chain prefill splits few, long chains into segments
-    float* d_segstate;            // [2 x SMs][dk * dv]
+    float* d_segstate;            // [2 x SMs][dk * dv], then [2 x SMs] counters
     // per-chain flags of the gated tensor-core prefill: chains it left to the CUDA-core kernel
     int* d_redo;                  // [redo_cap]
     int64_t redo_cap;
@@ -179,7 +179,12 @@ int lasad_create(lasad_ctx** out, int device)
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) ctx->stream_max_ctas = lasad::prefill_stream_max_ctas(device);
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_segstate, (size_t)2 * ctx->sm_count * 64 * 64 * sizeof(float));
+    if (e == cudaSuccess) {
+        // 2 x SMs states, then as many counters (zero between launches)
+        const size_t bytes = (size_t)2 * ctx->sm_count * (64 * 64 * sizeof(float) + sizeof(int));
+        e = cudaMalloc(&ctx->d_segstate, bytes);
+        if (e == cudaSuccess) e = cudaMemset(ctx->d_segstate, 0, bytes);
+    }
     cudaSetDevice(prev);
     if (e == cudaSuccess && reserve_units(ctx, kDefaultRelayUnits) != LASAD_OK) e = cudaErrorMemoryAllocation;
     if (e == cudaSuccess && reserve_redo(ctx, kDefaultRedoUnits) != LASAD_OK) e = cudaErrorMemoryAllocation;
@@ -319,7 +324,7 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
         if (impl == 4) {
             a.seg_state = ctx->d_segstate;
             if (lasad::prefill_tc_segments(lasad::prefill_stream_chunks(p->T), (long long)p->B * p->H, ctx->sm_count) > 1)
-                launches = 3;
+                launches = 2;
         }
         const cudaError_t e = lasad::launch_prefill_tc(a, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);

@@ -726,9 +726,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 // The SAD recurrence (Section 3.4) is linear in the state, so over a segment [a, b) of a chain
 //     S_b = gamma^(decaying steps in [a, b)) S_a + L,     L = the state the segment reaches from zero.
 // First launch (below): L for every segment but a chain's last, from K and V alone (the dS MMAs
-// of the main kernel and nothing else).  Second launch: S_a for every segment, an element-wise
-// scan over a chain's segments.  Third launch: the main kernel with one work unit per segment.
+// of the main kernel and nothing else); the CTA that finishes a chain's last L then turns them into
+// S_a for every segment, an element-wise scan over the chain's segments.  Second launch: the main
+// kernel with one work unit per segment.
 // ---------------------------------------------------------------------------------------------
+// steps[s] = decaying steps among segment s's tokens (SAD rule, Section 3.4), the same for every
+// chain, counted on the host.
+constexpr int kMaxSegs = 320;
+struct SegSteps {
+    int n[kMaxSegs];
+};
+
 struct StateSmem {
     unsigned char k[kStages][kTileBytes];
     unsigned char v[kStages][kTileBytes];
@@ -739,12 +747,13 @@ struct StateSmem {
     unsigned long long drain;
     uint32_t tmem_base;
     int abort_flag;
+    int last_of_chain;              // this CTA wrote the chain's last missing segment state: it runs the scan
 };
 constexpr int kStateTmemCols = 64;
 
 __global__ void __launch_bounds__(kThreads, 2)
 prefill_seg_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, TcParams p,
-                         float* seg_state)
+                         SegSteps steps, float* seg_state, int* seg_count)
 {
     extern __shared__ unsigned char smem_raw[];
     StateSmem& sm = *reinterpret_cast<StateSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -895,43 +904,56 @@ prefill_seg_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kStateTmemCols) : "memory");
     }
-}
 
-// seg_state[s + 1] holds L of segment s on entry; on exit seg_state[s] is the state at the start of
-// segment s (seg_state[0]: the caller's incoming state or zero).  One thread per state element, a
-// chain's segments in order; the loads of a batch of segments are issued together, only the
-// multiply-adds are serial.  steps[s] = decaying steps among segment s's tokens (SAD rule, Section
-// 3.4), the same for every chain, counted on the host.
-constexpr int kMaxSegs = 320;
-struct SegSteps {
-    int n[kMaxSegs];
-};
-
-__global__ void __launch_bounds__(256)
-prefill_seg_scan_kernel(TcParams p, SegSteps steps, float* seg_state)
-{
-    constexpr int kBatch = 8;
-    const int per_chain = kD * kD / 256;
-    const int chain = blockIdx.x / per_chain;
-    const int e = (blockIdx.x - chain * per_chain) * 256 + threadIdx.x;
-    const size_t stride = (size_t)p.B * p.H * kD * kD;        // from one segment's slot to the next
-    float* slot = seg_state + (size_t)chain * kD * kD + e;
-    const float gamma = p.decay[chain % p.H];
-    const float lg = gamma > 0.0f ? log2f(gamma) : 0.0f;
-    float carry = p.state_in ? p.state_in[(size_t)chain * kD * kD + e] : 0.0f;
-    slot[0] = carry;
-    for (int s0 = 0; s0 + 1 < p.n_segs; s0 += kBatch) {
-        float loc[kBatch];
+    // ---- the scan over the chain's segments, by whichever of its CTAs finishes last -------------
+    // seg_state[s + 1] holds L of segment s now; afterwards seg_state[s] is the state at the start
+    // of segment s (seg_state[0]: the caller's incoming state or zero).  seg_count[chain] counts the
+    // CTAs of the chain that are done and goes back to zero with the last one.
+    if (tid == 0) {
+        __threadfence();           // after the barrier above: covers every thread's stores of L
+        const int done = atomicAdd(seg_count + chain, 1);
+        sm.last_of_chain = done == p.n_segs - 2;
+        if (sm.last_of_chain) seg_count[chain] = 0;
+    }
+    __syncthreads();
+    if (sm.last_of_chain && tid < kEThreads) {
+        __threadfence();
+        constexpr int kBatch = 4;
+        const size_t stride = (size_t)n_chains * kD * kD;          // from one segment's slot to the next
+        float4* slot = reinterpret_cast<float4*>(seg_state + (size_t)chain * kD * kD) + tid;   // + j * 256: 16 elements per thread
+        const float lg = gamma > 0.0f ? log2f(gamma) : 0.0f;
+        float4 carry[4];
 #pragma unroll
-        for (int j = 0; j < kBatch; ++j)
-            loc[j] = s0 + j + 1 < p.n_segs ? slot[(size_t)(s0 + j + 1) * stride] : 0.0f;
+        for (int j = 0; j < 4; ++j) {
+            carry[j] = p.state_in ? reinterpret_cast<const float4*>(p.state_in + (size_t)chain * kD * kD)[tid + j * kEThreads]
+                                  : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            slot[j * kEThreads] = carry[j];
+        }
+        for (int s0 = 0; s0 + 1 < p.n_segs; s0 += kBatch) {
+            float4 loc[kBatch][4];
 #pragma unroll
-        for (int j = 0; j < kBatch; ++j) {
-            if (s0 + j + 1 < p.n_segs) {
-                const int n = steps.n[s0 + j];
-                const float g = n == 0 ? 1.0f : gamma > 0.0f ? exp2f((float)n * lg) : 0.0f;
-                carry = fmaf(g, carry, loc[j]);
-                slot[(size_t)(s0 + j + 1) * stride] = carry;
+            for (int b2 = 0; b2 < kBatch; ++b2)
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    loc[b2][j] = s0 + b2 + 1 < p.n_segs
+                                     ? __ldcg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(slot) +
+                                                                              (size_t)(s0 + b2 + 1) * stride) + j * kEThreads)
+                                     : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+            for (int b2 = 0; b2 < kBatch; ++b2) {
+                if (s0 + b2 + 1 < p.n_segs) {
+                    const int nst = steps.n[s0 + b2];
+                    const float g = nst == 0 ? 1.0f : gamma > 0.0f ? exp2f((float)nst * lg) : 0.0f;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        carry[j].x = fmaf(g, carry[j].x, loc[b2][j].x);
+                        carry[j].y = fmaf(g, carry[j].y, loc[b2][j].y);
+                        carry[j].z = fmaf(g, carry[j].z, loc[b2][j].z);
+                        carry[j].w = fmaf(g, carry[j].w, loc[b2][j].w);
+                        *(reinterpret_cast<float4*>(reinterpret_cast<float*>(slot) + (size_t)(s0 + b2 + 1) * stride) +
+                          j * kEThreads) = carry[j];
+                    }
+                }
             }
         }
     }
@@ -985,7 +1007,7 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st)
     if (e != cudaSuccess) return e;
     const long long chains = (long long)a.B * a.H;
     if (a.seg_state) {
-        // few chains: cut them into segments that run side by side (three launches, see above)
+        // few chains: cut them into segments that run side by side (two launches, see above)
         const int n_chunks = (a.T + kC - 1) / kC;
         const int segs = prefill_tc_segments(n_chunks, chains, sms);
         if (segs > 1) {
@@ -995,16 +1017,16 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st)
             const size_t ssmem = sizeof(StateSmem) + 1024;
             e = cudaFuncSetAttribute(prefill_seg_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssmem);
             if (e != cudaSuccess) return e;
-            prefill_seg_state_kernel<<<(unsigned)(chains * (segs - 1)), kThreads, ssmem, st>>>(mk, mv, p, a.seg_state);
-            e = cudaGetLastError();
-            if (e != cudaSuccess) return e;
             SegSteps steps;
             for (int sg = 0; sg + 1 < segs; ++sg) {
                 const long long lo = a.t0 + (long long)sg * p.seg_chunks * kC, hi = lo + (long long)p.seg_chunks * kC;
                 steps.n[sg] = (int)(decay_steps_upto(hi - 1, a.grid_w, a.prefix_len) -
                                     decay_steps_upto(lo - 1, a.grid_w, a.prefix_len));
             }
-            prefill_seg_scan_kernel<<<(unsigned)(chains * (kD * kD / 256)), 256, 0, st>>>(p, steps, a.seg_state);
+            // the per-chain counters sit behind the 2 x SMs state slots
+            int* seg_count = reinterpret_cast<int*>(a.seg_state + (size_t)2 * sms * kD * kD);
+            prefill_seg_state_kernel<<<(unsigned)(chains * (segs - 1)), kThreads, ssmem, st>>>(mk, mv, p, steps, a.seg_state,
+                                                                                              seg_count);
             e = cudaGetLastError();
             if (e != cudaSuccess) return e;
         }

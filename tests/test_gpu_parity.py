@@ -280,7 +280,7 @@ def test_more_chains_than_resident_ctas(ctx, T):
 @pytest.mark.parametrize("B,H,T", [(1, 5, 2000), (2, 12, 1500), (1, 1, 9216), (3, 16, 1153)])
 def test_few_long_chains_cut_into_segments(ctx, B, H, T):
     """Implementation 4: a first launch gets every segment's own contribution to the state from K and
-    V, a scan hands every segment its starting state, and the segments then run side by side.
+    V and a scan hands every segment its starting state; a second launch runs the segments side by side.
     Ragged last chunk, heads on both decay paths, an incoming state, a prefix token, a start in
     mid-row, state_out aliasing state_in; twice in a row."""
     d, w = 64, 13
@@ -324,7 +324,7 @@ def test_prefill_recorded_into_a_cuda_graph_and_replayed(ctx, T):
     """A prefill call captured into a CUDA graph and replayed on new inputs.  With few chains the
     default would take the task-streaming kernel (T = 700), whose packets carry a host-side launch
     number; under capture it must fall back, and asking for that kernel by option must be refused.
-    T = 2300 records the three launches of the segment-parallel mode."""
+    T = 2300 records the two launches of the segment-parallel mode."""
     B, H, d, w = 1, 4, 64, 9
     gen = torch.Generator().manual_seed(77 + T)
     g = torch.tensor([0.93, 0.5, 0.999, 0.97])

@@ -32,8 +32,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) from the ncu captures
 # summarised under profiles/; None until a capture of that kernel exists.
 NCU_TRAFFIC_BYTES = {
-    # prefill_tc_kernel: 577.3 MB measured on the 608.7 MB capture case, scaled by tokens to config 5b
-    "prefill": 862_200_000,
+    # prefill_pair_kernel (the default on config 5b): not captured since the kernel was written
+    "prefill": None,
     # decode_kernel, config 4, inside the kernel (the rest of the written state drains from L2 later)
     "decode": 112_200_000,
 }
@@ -305,7 +305,7 @@ def run_ours(args):
             "clocks": sampler.summary(),
             "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4),
-                         "traffic": NCU_TRAFFIC_BYTES["prefill"] if (wl.name == "config5b" and args.prefill_impl in (0, 2)) else None,
+                         "traffic": NCU_TRAFFIC_BYTES["prefill"] if (wl.name == "config5b" and args.prefill_impl in (0, 5)) else None,
                          "peak_source": peaks["source"],
                          "kernel_ms": round(kern_ms, 5), "bytes_per_launch": pf_bytes},
             "tensor": {"executed_tflops": round(tc_tflops, 1), "chunk": chunk,
@@ -603,8 +603,9 @@ def main():
                     help="chunk length used to count executed tensor flops")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-configuration prefill sweep")
-    ap.add_argument("--prefill-impl", type=int, default=0, choices=[0, 1, 2, 3],
-                    help="prefill kernel: 0 library default, 1 CUDA cores, 2 tcgen05 CTA-per-chain, 3 tcgen05 task-streaming")
+    ap.add_argument("--prefill-impl", type=int, default=0, choices=[0, 1, 2, 3, 4, 5],
+                    help="prefill kernel: 0 library default, 1 CUDA cores, 2 tcgen05 CTA-per-chain, 3 tcgen05 task-streaming, "
+                         "4 as 2 with few long chains cut into segments, 5 tcgen05 balanced (one CTA per SM, two pipelines)")
     ap.add_argument("--only", choices=["all", "prefill", "decode", "gated"], default="all",
                     help="time only one of the kernels (small profiling runs); gated = the gated prefill "
                          "on --prefill-workload")

@@ -57,12 +57,15 @@ enum { LASAD_F32 = 0, LASAD_BF16 = 1 };
 enum {
     LASAD_OPT_PREFILL_IMPL = 0, /* 0 auto (bf16, d = 64: 4 when B * H <= SMs / 3 and T > 1920 or
                                    B * H <= SMs / 2 and T > 3968, else 3 when B * H <= SMs / 3 and
-                                   T > 128, else 2; other shapes 1),
+                                   T > 128, else 5 when T > 3968 unless B * H fills whole rounds of
+                                   2 * SMs to 93 % or more, else 2; other shapes 1),
                                    1 CUDA-core fp32 kernel,
                                    2 tcgen05 kernel with one CTA per (batch, head) at a time,
                                    3 tcgen05 kernel streaming (batch, head, chunk) tasks through
                                    persistent CTAs, 4 as 2 with few long sequences cut into segments
-                                   that run side by side (two launches; 2 where nothing is cut)     */
+                                   that run side by side (two launches; 2 where nothing is cut),
+                                   5 tcgen05 kernel with one CTA per SM whose two chunk pipelines
+                                   work on one sequence at a time, the work cut evenly over the SMs */
     LASAD_OPT_PREFILL_CHUNK = 1,/* CUDA-core prefill chunk length: 0 auto, else 16/32/64          */
     LASAD_OPT_DECODE_TPU = 2,   /* decode: threads per (b,h) state; 0 auto, else 32/64/128/256 */
     LASAD_OPT_WAIT_LIMIT = 3    /* iteration cap of device-side waits; 0 = library default   */

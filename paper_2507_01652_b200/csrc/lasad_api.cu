@@ -10,7 +10,7 @@ struct lasad_ctx {
     int* d_status;        // device status word
     int last_cuda_error;
     uint64_t launches;
-    int opt_prefill_impl; // 0 auto, 1 simt, 2 tensor
+    int opt_prefill_impl; // LASAD_OPT_PREFILL_IMPL: 0 auto, 1..5 as listed in lasad.h
     int opt_prefill_chunk;
     int opt_decode_tpu;
     unsigned wait_limit;
@@ -25,6 +25,8 @@ struct lasad_ctx {
     // per-chain flags of the gated tensor-core prefill: chains it left to the CUDA-core kernel
     int* d_redo;                  // [redo_cap]
     int64_t redo_cap;
+    // state slots and flags at the cuts of the balanced tensor-core prefill (one per SM)
+    void* d_pair;
     // host-buffer pipeline of lasad_forward_host: two staging slots (q | k | v | o of one batch
     // element each), a decay and a state buffer, copy streams and the events that order them
     void* d_stage[2];
@@ -111,6 +113,13 @@ int auto_prefill_impl(const lasad_ctx* ctx, const lasad_params* p, int64_t batch
     const int64_t chains = batch * p->H;
     if ((chains * 3 <= ctx->sm_count && chunks >= 16) || (chains * 2 <= ctx->sm_count && chunks >= 32)) return 4;
     if (chains * 3 <= ctx->sm_count && chunks >= 2 && ctx->stream_max_ctas > 0) return 3;
+    // Long chains: the balanced kernel (one chain at a time per SM, left-over chains cut into equal
+    // pieces), unless the chains fill the two-per-SM slots of the CTA-per-chain kernel almost exactly.
+    if (chunks >= 32) {
+        const int64_t slots = 2LL * ctx->sm_count;
+        const int64_t waves = (chains + slots - 1) / slots;
+        if (chains * 100 < waves * slots * 93) return 5;
+    }
     return 2;
 }
 
@@ -185,6 +194,11 @@ int lasad_create(lasad_ctx** out, int device)
         e = cudaMalloc(&ctx->d_segstate, bytes);
         if (e == cudaSuccess) e = cudaMemset(ctx->d_segstate, 0, bytes);
     }
+    if (e == cudaSuccess) {
+        const size_t bytes = lasad::prefill_pair_scratch_bytes(ctx->sm_count);
+        e = cudaMalloc(&ctx->d_pair, bytes);
+        if (e == cudaSuccess) e = cudaMemset(ctx->d_pair, 0, bytes);
+    }
     cudaSetDevice(prev);
     if (e == cudaSuccess && reserve_units(ctx, kDefaultRelayUnits) != LASAD_OK) e = cudaErrorMemoryAllocation;
     if (e == cudaSuccess && reserve_redo(ctx, kDefaultRedoUnits) != LASAD_OK) e = cudaErrorMemoryAllocation;
@@ -193,6 +207,7 @@ int lasad_create(lasad_ctx** out, int device)
         if (ctx->d_relay) cudaFree(ctx->d_relay);
         if (ctx->d_redo) cudaFree(ctx->d_redo);
         if (ctx->d_segstate) cudaFree(ctx->d_segstate);
+        if (ctx->d_pair) cudaFree(ctx->d_pair);
         delete ctx;
         return LASAD_ERR_CUDA;
     }
@@ -207,6 +222,7 @@ int lasad_destroy(lasad_ctx* ctx)
     if (ctx->d_relay) cudaFree(ctx->d_relay);
     if (ctx->d_redo) cudaFree(ctx->d_redo);
     if (ctx->d_segstate) cudaFree(ctx->d_segstate);
+    if (ctx->d_pair) cudaFree(ctx->d_pair);
     for (int i = 0; i < 2; ++i)
         if (ctx->d_stage[i]) cudaFree(ctx->d_stage[i]);
     if (ctx->d_host_decay) cudaFree(ctx->d_host_decay);
@@ -237,7 +253,7 @@ int lasad_set_option(lasad_ctx* ctx, int option, int value)
     if (!ctx) return LASAD_ERR_INVALID_ARG;
     switch (option) {
         case LASAD_OPT_PREFILL_IMPL:
-            if (value < 0 || value > 4) return LASAD_ERR_INVALID_ARG;
+            if (value < 0 || value > 5) return LASAD_ERR_INVALID_ARG;
             ctx->opt_prefill_impl = value;
             return LASAD_OK;
         case LASAD_OPT_PREFILL_CHUNK:
@@ -314,6 +330,13 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
         }
         r.max_ctas = ctx->stream_max_ctas;
         const cudaError_t e = lasad::launch_prefill_stream(a, r, st);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        ctx->launches += 1;
+        return LASAD_OK;
+    }
+    if (impl == 5) {
+        if (!tc_ok || (int64_t)p->B * p->H * lasad::prefill_stream_chunks(p->T) > 0x7fffffffLL) return LASAD_ERR_UNSUPPORTED;
+        const cudaError_t e = lasad::launch_prefill_pair(a, ctx->d_pair, ctx->sm_count, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         ctx->launches += 1;
         return LASAD_OK;

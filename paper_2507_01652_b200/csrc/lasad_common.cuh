@@ -24,7 +24,8 @@ struct KernelArgs {
     const int* pos;         // decode only: [B] absolute index of each sequence's token, or nullptr (t0 for all)
     const int* widths;      // decode only: [B] grid width of each sequence, or nullptr (grid_w for all)
     int* status;            // device status word (bounded waits report here)
-    int* work;              // two device ints, zero between launches: work counter of the persistent prefill
+    int* work;              // device ints: [0], [1] zero between launches (work counters of the persistent
+                            // prefill kernels), [2] launches of the balanced prefill so far
     float* seg_state;       // prefill, CTA-per-chain kernel: room for 2 x SMs states, or nullptr (chains are not cut)
     unsigned wait_limit;
 };
@@ -76,6 +77,11 @@ bool prefill_gated_tc_supported(int dk, int dv, bool bf16);
 cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, int* redo, cudaStream_t st);
 bool prefill_tc_supported(int dk, int dv, bool bf16);
 cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st);
+// Balanced tensor-core prefill: one CTA per SM, two chunk pipelines per CTA on one chain, the flat
+// chunk sequence cut into equal runs.  `scratch`: prefill_pair_scratch_bytes(sms) bytes of device
+// memory, zero before the first launch (the kernel leaves it zero).
+size_t prefill_pair_scratch_bytes(int sms);
+cudaError_t launch_prefill_pair(const KernelArgs& a, void* scratch, int sms, cudaStream_t st);
 // segments per chain that launch_prefill_tc cuts the chains into when a.seg_state is given (1: not cut)
 int prefill_tc_segments(int n_chunks, long long chains, int sms);
 

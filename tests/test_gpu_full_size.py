@@ -28,7 +28,7 @@ def _sampled_chains(wl, n):
     return sorted(picks)
 
 
-@pytest.mark.parametrize("name", ["config3", "config5a", "config5b"])
+@pytest.mark.parametrize("name", ["config2", "config3", "config5a", "config5b"])
 def test_prefill_full_size_sampled_chains(ctx, name):
     wl = workloads.WORKLOADS[name]
     q, k, v = workloads.make_qkv(wl)

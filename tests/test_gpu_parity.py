@@ -14,7 +14,7 @@ from tests._util import TOL, oracle, rel_err, to64
 
 pytestmark = pytest.mark.gpu
 
-IMPLS = [1, 2, 3, 4]  # 1 = CUDA-core fp32 kernel, 2 = tcgen05 kernel (CTA per chain), 3 = tcgen05 task-streaming kernel,
+IMPLS = [1, 2, 3, 4, 5]  # 1 = CUDA-core fp32 kernel, 2 = tcgen05 kernel (CTA per chain), 3 = tcgen05 task-streaming kernel,
                       # 4 = as 2, few long chains cut into segments
 
 
@@ -302,12 +302,13 @@ def test_few_long_chains_cut_into_segments(ctx, B, H, T):
 
 def test_default_prefill_picks_a_kernel_by_the_number_of_chains(ctx):
     """Option 0: few (batch, head) pairs with several chunks each go to the task-streaming kernel,
-    everything else in bf16 / d = 64 to the CTA-per-chain kernel; whichever runs, the result is that
-    kernel's bit for bit, and right."""
-    d, w, T = 64, 12, 700
+    long sequences that do not fill whole rounds of CTA slots to the balanced kernel, everything else
+    in bf16 / d = 64 to the CTA-per-chain kernel; whichever runs, the result is that kernel's bit for
+    bit, and right."""
+    d, w = 64, 12
     gen = torch.Generator().manual_seed(4242)
-    g_all = 0.9 + 0.0999 * torch.rand(16, generator=gen)
-    for B, H, expect in ((1, 16, 3), (12, 16, 2)):
+    g_all = 0.9 + 0.0999 * torch.rand(100, generator=gen)
+    for B, H, T, expect in ((1, 16, 700, 3), (12, 16, 700, 2), (1, 100, 4000, 5)):
         q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
         g = g_all[:H]
         o_ref, s_ref = oracle(q, k, v, g, w)
@@ -317,6 +318,65 @@ def test_default_prefill_picks_a_kernel_by_the_number_of_chains(ctx):
         assert torch.equal(o0, o1) and torch.equal(s0, s1), (B, H)
         assert rel_err(o0, o_ref) <= TOL[torch.bfloat16]
         assert rel_err(s0, s_ref) <= TOL[torch.bfloat16]
+
+
+@pytest.mark.parametrize("B,H,T", [(1, 160, 1100), (2, 163, 1100), (1, 151, 260), (40, 5, 130), (1, 149, 2500),
+                                   (3, 7, 900)])
+def test_balanced_prefill_left_over_chains_cut_into_pieces(ctx, B, H, T):
+    """Implementation 5 with more chains than SMs: every CTA takes whole chains in rounds and one
+    piece of a left-over chain, whose state travels from CTA to CTA (pieces of 4 chunks, two or three
+    to a chain, some shares straddling two chains: 160 x 9 chunks; two rounds: 326 chains; chains too
+    short to be cut: 2 and 3 chunks; one long left-over chain over many CTAs: 149 x 20 chunks), and
+    with fewer chains than SMs (one chain per CTA).  Heads on both decay paths, an incoming state, a
+    prefix token, a start in mid-row, state_out aliasing state_in; twice in a row (the packet tags
+    must tell the launches apart)."""
+    d, w = 64, 13
+    gen = torch.Generator().manual_seed(1200 + H + T)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+    g = 0.9 + 0.0999 * torch.rand(H, generator=gen)
+    g[0], g[1], g[2], g[3] = 0.45, 0.0, 1.0, 0.59
+    g[H - 1] = 0.3
+    s_in = torch.randn(B, H, d, d, generator=gen)
+    o_ref, s_ref = oracle(q, k, v, g, w, 1, 5, 0.5, s_in)
+    dq, dk, dv, dg = _dev(q, k, v, g)
+    for rep in range(2):
+        ds = s_in.cuda()
+        o, s = _forward(ctx, 5, dq, dk, dv, dg, w, prefix_len=1, t0=5, scale=0.5, state_in=ds, state_out=ds)
+        assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+        assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
+
+
+def test_balanced_prefill_recorded_into_a_cuda_graph_and_replayed(ctx):
+    """Implementation 5 numbers its launches on the device, so a recorded launch may be replayed: the
+    hand-off packets of one replay must not pass for the next one's (160 chains of 9 chunks: the
+    left-over chains' states cross CTAs)."""
+    B, H, T, d, w = 1, 160, 1100, 64, 9
+    gen = torch.Generator().manual_seed(78)
+    g = 0.9 + 0.0999 * torch.rand(H, generator=gen)
+    dg = g.cuda()
+    dq, dk, dv = [torch.empty(B, T, H, d, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+    o = torch.empty_like(dv)
+    s = torch.empty(B, H, d, d, device="cuda")
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 5)
+    try:
+        with torch.cuda.stream(stream):
+            ctx.lasad_forward(dq, dk, dv, dg, w, o=o, state_out=s)          # warm-up outside the capture
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph, stream=stream):
+                ctx.lasad_forward(dq, dk, dv, dg, w, o=o, state_out=s)
+    finally:
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
+    for rep in range(3):
+        q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+        dq.copy_(q); dk.copy_(k); dv.copy_(v)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        o_ref, s_ref = oracle(q, k, v, g, w)
+        assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+        assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
 
 
 @pytest.mark.parametrize("T", [700, 2300])
@@ -470,7 +530,7 @@ def test_decode_per_sequence_positions_and_widths(ctx):
 # ------------------------------------------------------------------------------------------
 # bounded waits: a wait that runs out is reported, nothing hangs, the context stays usable
 # ------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("impl", [2, 3, 4])
+@pytest.mark.parametrize("impl", [2, 3, 4, 5])
 def test_expired_device_wait_is_reported_and_context_survives(ctx, impl):
     """With the poll limit of the device-side waits set to 1, some wait runs out before its
     barrier completes: the kernel must leave through its normal exit, the status word must say

@@ -30,9 +30,14 @@
  *     fp32 [B, H, dk, dv], 16-byte aligned.
  *   - Supported: dk == dv in {32, 64}; dtype F32 or BF16 (q, k, v, o share it; state, decay
  *     and all accumulation are fp32); any B, H, T >= 1.  Otherwise LASAD_ERR_UNSUPPORTED.
- *   - One ctx is bound to one device and may be used from one host thread at a time; its
- *     prefill calls share per-chain relay storage, so two lasad_forward calls on one ctx must
- *     not overlap on the device (issue them on one stream, or order the streams).
+ *   - One ctx is bound to one device, which must be the current device at every call that
+ *     takes the ctx (otherwise LASAD_ERR_INVALID_ARG), and may be used from one host thread at a
+ *     time; its prefill calls share scratch storage (state slots, work counters), so two
+ *     lasad_forward calls on one ctx must not overlap on the device (issue them on one stream,
+ *     or order the streams).
+ *   - A stride of 0 is accepted only for a dimension of one element.
+ *   - decay (and gate) values must lie in [0, 1] and be finite: they are device data, which the
+ *     library does not inspect; values outside that range give undefined results (no fault).
  */
 #ifndef LASAD_H_
 #define LASAD_H_
@@ -86,8 +91,10 @@ typedef struct lasad_params {
 
 typedef struct lasad_ctx lasad_ctx;
 
-/* Creates a context on CUDA device `device` (it owns one device status word).  The only
- * entry point that allocates. */
+/* Creates a context on CUDA device `device`: a status word, work counters and the scratch storage
+ * of the prefill kernels (state slots at the cuts of sequences, relay slots, per-pair flags; about
+ * 50 MiB in all).  Which later calls may allocate as well is said at lasad_reserve,
+ * lasad_forward_host and lasad_forward_gated; no other call allocates. */
 int lasad_create(lasad_ctx** out, int device);
 int lasad_destroy(lasad_ctx* ctx);
 int lasad_set_option(lasad_ctx* ctx, int option, int value);
@@ -161,7 +168,9 @@ int lasad_forward_host(lasad_ctx* ctx, const lasad_params* p,
  *                   status block takes the write and cannot be read back).
  *
  * The first call on a device looks up the array's device address and the device's limits; make
- * that first call before starting any stream capture.  All calls on a device share the one
+ * that first call before starting any stream capture.  A call whose `cuda_stream` is being
+ * captured returns LASAD_ERR_UNSUPPORTED and enqueues nothing: the kernel tells its calls apart by
+ * a number counted on the host, which a replayed recording would repeat.  All calls on a device share the one
  * array, which keeps the previous call's contents (the library invalidates them by a call
  * counter and clears the array before the counter repeats): two calls that overlap on the GPU
  * race on it, so issue them on one stream or order the streams.  Arguments q .. state_out and

@@ -146,11 +146,16 @@ int check_common(const lasad_ctx* ctx, const lasad_params* p, bool decode)
             const int64_t st = strides[s][d];
             if (st < 0 || (st * esz) % 16 != 0) return LASAD_ERR_INVALID_ARG;
         }
+        // a zero stride would alias the elements of a dimension: allowed only where it has one element
+        if ((strides[s][0] == 0 && p->B > 1) || (!decode && strides[s][1] == 0 && p->T > 1)) return LASAD_ERR_INVALID_ARG;
         const int width = (s < 2) ? p->dk : p->dv;
         if (strides[s][2] < width && p->H > 1) return LASAD_ERR_INVALID_ARG;
     }
     if (p->dk != p->dv || (p->dk != 32 && p->dk != 64)) return LASAD_ERR_UNSUPPORTED;
     if ((int64_t)p->B * p->H > 0x7fffffffLL) return LASAD_ERR_UNSUPPORTED;
+    // the context's buffers, SM count and kernel attributes belong to its device
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess || current != ctx->device) return LASAD_ERR_INVALID_ARG;
     return LASAD_OK;
 }
 
@@ -349,7 +354,7 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
             if (lasad::prefill_tc_segments(lasad::prefill_stream_chunks(p->T), (long long)p->B * p->H, ctx->sm_count) > 1)
                 launches = 2;
         }
-        const cudaError_t e = lasad::launch_prefill_tc(a, st);
+        const cudaError_t e = lasad::launch_prefill_tc(a, ctx->sm_count, st);
         if (e != cudaSuccess) return fail_cuda(ctx, e);
         ctx->launches += launches;
         return LASAD_OK;

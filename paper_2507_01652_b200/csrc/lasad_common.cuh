@@ -76,7 +76,7 @@ cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, 
 bool prefill_gated_tc_supported(int dk, int dv, bool bf16);
 cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, int* redo, cudaStream_t st);
 bool prefill_tc_supported(int dk, int dv, bool bf16);
-cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st);
+cudaError_t launch_prefill_tc(const KernelArgs& a, int sms, cudaStream_t st);
 // Balanced tensor-core prefill: one CTA per SM, two chunk pipelines per CTA on one chain, the flat
 // chunk sequence cut into equal runs.  `scratch`: prefill_pair_scratch_bytes(sms) bytes of device
 // memory, zero before the first launch (the kernel leaves it zero).

@@ -981,7 +981,7 @@ int prefill_tc_segments(int n_chunks, long long chains, int sms)
     return (n_chunks + len - 1) / len;
 }
 
-cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st)
+cudaError_t launch_prefill_tc(const KernelArgs& a, int sms, cudaStream_t st)
 {
     CUtensorMap mq, mk, mv, mo;
     if (!encode_chunk_map(&mq, a.q, a.B, a.T, a.H, a.qs) || !encode_chunk_map(&mk, a.k, a.B, a.T, a.H, a.ks) ||
@@ -1001,10 +1001,7 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, cudaStream_t st)
     if (e != cudaSuccess) return e;
     // Two CTAs fit on an SM; with more chains than that, the CTAs stay and draw further chains
     // from the work counter, so a chain's first loads overlap the previous chain's last chunk.
-    int dev = 0, sms = 0;
-    e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
+    if (sms <= 0) return cudaErrorInvalidValue;
     const long long chains = (long long)a.B * a.H;
     if (a.seg_state) {
         // few chains: cut them into segments that run side by side (two launches, see above)

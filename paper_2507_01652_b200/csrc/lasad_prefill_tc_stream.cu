@@ -830,6 +830,7 @@ extern "C" int lasad_forward_static(const lasad_params* p, const void* q, const 
         for (int d = 0; d < 3; ++d)
             if (strides[s][d] < 0 || (strides[s][d] * 2) % 16 != 0) return LASAD_ERR_INVALID_ARG;
         if (strides[s][2] < 64 && p->H > 1) return LASAD_ERR_INVALID_ARG;
+        if ((strides[s][0] == 0 && p->B > 1) || (strides[s][1] == 0 && p->T > 1)) return LASAD_ERR_INVALID_ARG;
     }
     if (p->dtype != LASAD_BF16 || p->dk != 64 || p->dv != 64) return LASAD_ERR_UNSUPPORTED;
     const int64_t units = (int64_t)p->B * p->H;
@@ -851,6 +852,12 @@ extern "C" int lasad_forward_static(const lasad_params* p, const void* q, const 
         st.max_ctas = n;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // The relay packets are tagged with a call number that this function counts on the host: a
+    // call recorded into a CUDA graph would replay with the number it was recorded with and could
+    // take the previous replay's packets for its own.  So a stream that is being captured is refused.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) return LASAD_ERR_CUDA;
+    if (cap != cudaStreamCaptureStatusNone) return LASAD_ERR_UNSUPPORTED;
     unsigned char* base = static_cast<unsigned char*>(st.scratch);
     const size_t relay_bytes = (size_t)kStaticUnits * lasad::kTcRelaySlotBytes;
 

@@ -248,6 +248,12 @@ def test_argument_errors_launch_nothing(ctx):
     assert e.value.code == binding.LASAD_ERR_INVALID_ARG
     with pytest.raises(ValueError):
         ctx.lasad_forward(q.cpu(), q, q, g, 4)
+    # a zero stride over a dimension with more than one element (a broadcast view) is refused
+    qb = torch.zeros(1, T, H, d, dtype=torch.bfloat16, device="cuda").expand(3, T, H, d)
+    q3 = torch.zeros(3, T, H, d, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.LasadError) as e:
+        ctx.lasad_forward(qb, q3, q3, g, 4)
+    assert e.value.code == binding.LASAD_ERR_INVALID_ARG
     assert ctx.launch_count == n0
 
 

@@ -1,4 +1,5 @@
-"""The allocation-free prefill entry point, `lasad_forward_static`, against `lasad_forward`.
+"""The allocation-free prefill entry point, `lasad_forward_static`, against `lasad_forward` and
+against the CPU oracle.
 
 Some hosts of this library must not let it allocate device memory: a serving process that fixes
 its device-memory plan at start-up, or a plug-in whose host framework owns every allocation.
@@ -12,7 +13,7 @@ import pytest
 import torch
 
 from paper_2507_01652_b200 import binding
-from tests._util import TOL, rel_err, to64
+from tests._util import TOL, oracle, rel_err, to64
 
 pytestmark = pytest.mark.gpu
 
@@ -42,8 +43,57 @@ def test_static_entry_point_matches_lasad_forward_twice_in_a_row():
             assert int(status.item()) == 0, "a device-side wait timed out"
             assert rel_err(o, to64(o_ref)) <= TOL[torch.bfloat16]
             assert rel_err(s, to64(s_ref)) <= TOL[torch.bfloat16]
+            # and against the oracle: the two entry points may share a kernel, so agreement
+            # between them alone would not show a fault common to both
+            o_orc, s_orc = oracle(q, k, v, g, w, P, 3, 0.5, s_in)
+            assert rel_err(o, o_orc) <= TOL[torch.bfloat16]
+            assert rel_err(s, s_orc) <= TOL[torch.bfloat16]
     finally:
         ctx.close()
+
+
+def test_static_entry_point_allocates_nothing_at_its_limit():
+    """B * H = 256, the most the built-in storage holds, without a status word of the caller's: the
+    driver's count of free device memory must not move over further calls, and the result must
+    match the oracle on sampled chains."""
+    B, T, H, w = 16, 300, 16, 10
+    q, k, v, g, s_in, w, P = _case(23, B, T, H, w, 0)
+    o = torch.empty_like(v)
+    s = torch.empty(B, H, 64, 64, device="cuda")
+    binding.lasad_forward_static(q, k, v, g, w, o, state_out=s, state_in=s_in)     # the device's first-call set-up, if still due
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        binding.lasad_forward_static(q, k, v, g, w, o, state_out=s, state_in=s_in)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, "device memory was allocated or freed by lasad_forward_static"
+    for b, h in ((0, 0), (7, 9), (15, 15)):
+        sl = (slice(b, b + 1), slice(None), slice(h, h + 1))
+        o_orc, s_orc = oracle(q[sl], k[sl], v[sl], g[h:h + 1], w, 0, 0, 1.0, s_in[b:b + 1, h:h + 1])
+        assert rel_err(o[sl], o_orc) <= TOL[torch.bfloat16], (b, h)
+        assert rel_err(s[b:b + 1, h:h + 1], s_orc) <= TOL[torch.bfloat16], (b, h)
+
+
+def test_static_entry_point_refuses_a_stream_that_is_being_captured():
+    """The kernel tells its calls apart by a number counted on the host, which a replayed recording
+    would repeat; so the entry point must refuse to be recorded rather than replay wrongly."""
+    q, k, v, g, s_in, w, P = _case(24, 1, 300, 2, 10, 0)
+    o = torch.empty_like(v)
+    binding.lasad_forward_static(q, k, v, g, w, o)          # set-up outside the capture
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            with pytest.raises(binding.LasadError) as e:
+                binding.lasad_forward_static(q, k, v, g, w, o, stream=stream.cuda_stream)
+    assert e.value.code == binding.LASAD_ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    o_orc, _ = oracle(q, k, v, g, w)
+    binding.lasad_forward_static(q, k, v, g, w, o)          # and it still works afterwards
+    torch.cuda.synchronize()
+    assert rel_err(o, o_orc) <= TOL[torch.bfloat16]
 
 
 def test_static_entry_point_rejects_what_it_cannot_hold():

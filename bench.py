@@ -57,7 +57,7 @@ class ClockSampler:
                0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
                0x2: "applications_clocks_setting", 0x10: "sync_boost"}
 
-    def __init__(self, device_index: int, period_s: float = 0.004):
+    def __init__(self, device_index: int, period_s: float = 0.001):
         self.period = period_s
         self.samples, self.reason_bits = [], 0
         self.max_mhz = None
@@ -278,8 +278,17 @@ def run_ours(args):
         gated = gated_sweep(ctx, peaks, dev)
 
     decode = None
+    decode_others = None
     if args.only != "prefill":
         decode = run_decode(args, ctx, peaks, dev, rank, barrier, max_ranks, K)
+        if args.only == "all" and not args.no_sweep:
+            decode_others = [run_decode(args, ctx, peaks, dev, rank, barrier, max_ranks, K, workload=name, hot=False)
+                             for name in ("config2", "config3")]
+    host_cost = None
+    scaling = None
+    if args.only == "all" and not args.no_sweep and rank == 0:
+        host_cost = host_cost_per_call(ctx, dev)
+        scaling = scaling_sweep(ctx, dev, cpu=(world == 1 and not args.no_cpu_baseline))
 
     # ---- CPU baseline: the oracle as it stands on this machine's host cores (rank 0, N = 1) ----
     cpu = None
@@ -311,6 +320,9 @@ def run_ours(args):
             "tensor": {"executed_tflops": round(tc_tflops, 1), "chunk": chunk,
                        "frac_of_bf16_peak": round(tc_tflops / peaks["bf16_tflops"], 4)},
             "decode": decode,
+            "decode_other_configs": decode_others,
+            "host_us_per_call": host_cost,
+            "scaling": scaling,
             "prefill_sweep": sweep,
             "gated": gated,
             "cpu_baseline": cpu,
@@ -321,16 +333,38 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+L2_BYTES = 126 << 20
+
+
+class L2Flush:
+    """Keeps a launch from finding its inputs in L2.  Workloads whose tensors exceed twice the L2
+    need nothing (back-to-back launches: what one launch leaves in L2 is the end of its data, the
+    next one starts at the beginning).  For smaller ones a 256 MiB buffer is READ between launches
+    (a reduction kernel): that fills L2 with clean lines, so the timed kernel neither hits its
+    inputs nor has to wait for dirty lines of the flush to drain to DRAM."""
+
+    def __init__(self, dev):
+        import torch
+        self.words = torch.zeros(32 << 20, dtype=torch.int64, device=dev)
+
+    def policy(self, nbytes: int) -> str:
+        return "back-to-back launches (tensors larger than 2x L2)" if nbytes > 2 * L2_BYTES else \
+            "256 MiB read between launches"
+
+    def __call__(self, nbytes: int):
+        if nbytes <= 2 * L2_BYTES:
+            self.words.sum()
+
+
 def prefill_sweep(ctx, peaks, dev, names, reps: int = 10):
     """Kernel time of one prefill per named workload (CUDA events around each launch, median of
-    `reps`); a buffer larger than L2 is written between launches so that no launch finds its
-    inputs in L2."""
+    `reps`), with the L2 policy of `L2Flush`."""
     import torch
 
     from paper_2507_01652_b200 import workloads
 
     stream = torch.cuda.current_stream()
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    flush = L2Flush(dev)
     out = []
     for name in names:
         # "name@B": the named workload at another batch size (e.g. one image at a time)
@@ -341,24 +375,33 @@ def prefill_sweep(ctx, peaks, dev, names, reps: int = 10):
         g = workloads.make_decay(wl).to(dev)
         o = torch.empty_like(v)
         s_out = torch.empty(wl.B, wl.H, wl.d, wl.d, dtype=torch.float32, device=dev)
-        times = []
-        for it in range(reps + 3):
-            flush.fill_(it & 1)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            ctx.lasad_forward(q, k, v, g, wl.grid_w, prefix_len=wl.prefix_len, o=o, state_out=s_out)
-            b.record(stream)
-            torch.cuda.synchronize()
-            if it >= 3:
-                times.append(a.elapsed_time(b))
-        ms = statistics.median(times)
         nbytes = prefill_bytes(wl)
+        ms = _time_launches(stream, flush, nbytes, reps,
+                            lambda: ctx.lasad_forward(q, k, v, g, wl.grid_w, prefix_len=wl.prefix_len, o=o, state_out=s_out))
         out.append({"workload": f"{wl.name}: B={wl.B} H={wl.H} T={wl.T} d={wl.d} {wl.dtype}",
                     "kernel_us": round(ms * 1e3, 2), "tokens_per_s": round(wl.B * wl.T / (ms * 1e-3), 1),
                     "algorithmic_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
-                    "frac_of_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)})
+                    "frac_of_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                    "l2_policy": flush.policy(nbytes)})
         del q, k, v, o, s_out
     return out
+
+
+def _time_launches(stream, flush, nbytes, reps, launch):
+    """Median CUDA-event time (ms) of `launch()` over `reps` launches after 3 warm-up ones."""
+    import torch
+
+    evs = []
+    for it in range(reps + 3):
+        flush(nbytes)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        launch()
+        b.record(stream)
+        if it >= 3:
+            evs.append((a, b))
+    torch.cuda.synchronize()
+    return statistics.median(a.elapsed_time(b) for a, b in evs)
 
 
 def gated_sweep(ctx, peaks, dev, wls=None, decode: bool = True, reps: int = 10):
@@ -371,7 +414,7 @@ def gated_sweep(ctx, peaks, dev, wls=None, decode: bool = True, reps: int = 10):
     from paper_2507_01652_b200 import workloads
 
     stream = torch.cuda.current_stream()
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    flush = L2Flush(dev)
     out = {"prefill": [], "decode": None}
     if wls is None:
         wls = [workloads.WORKLOADS[name] for name in ("config2", "config3", "config5b")]
@@ -380,22 +423,15 @@ def gated_sweep(ctx, peaks, dev, wls=None, decode: bool = True, reps: int = 10):
         lam = workloads.make_gate(wl).to(dev)
         o = torch.empty_like(v)
         s_out = torch.empty(wl.B, wl.H, wl.d, wl.d, dtype=torch.float32, device=dev)
-        times = []
-        for it in range(reps + 3):
-            flush.fill_(it & 1)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            ctx.lasad_forward_gated(q, k, v, lam, wl.grid_w, prefix_len=wl.prefix_len, o=o, state_out=s_out)
-            b.record(stream)
-            torch.cuda.synchronize()
-            if it >= 3:
-                times.append(a.elapsed_time(b))
-        ms = statistics.median(times)
         nbytes = wl.B * wl.T * wl.H * 5 * wl.d * wl.elem_bytes + wl.B * wl.H * wl.d * wl.d * 4   # q,k,v,gate in, o out
+        ms = _time_launches(stream, flush, nbytes, reps,
+                            lambda: ctx.lasad_forward_gated(q, k, v, lam, wl.grid_w, prefix_len=wl.prefix_len, o=o,
+                                                            state_out=s_out))
         out["prefill"].append({"workload": f"{wl.name}: B={wl.B} H={wl.H} T={wl.T} d={wl.d} {wl.dtype}",
                                "kernel_us": round(ms * 1e3, 2), "tokens_per_s": round(wl.B * wl.T / (ms * 1e-3), 1),
                                "algorithmic_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
-                               "frac_of_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)})
+                               "frac_of_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                               "l2_policy": flush.policy(nbytes)})
         del q, k, v, lam, o, s_out
     if not decode:
         return out
@@ -425,22 +461,103 @@ def gated_sweep(ctx, peaks, dev, wls=None, decode: bool = True, reps: int = 10):
     return out
 
 
-def run_decode(args, ctx, peaks, dev, rank, barrier, max_ranks, K):
-    """Decode sweep (config 4 shape): persistent fp32 state, one `lasad_decode_step` per grid position."""
+def host_cost_per_call(ctx, dev, calls: int = 1000):
+    """Host time of one library call: wall clock of `calls` enqueue-only calls (no synchronisation
+    inside the loop) on shapes whose kernels are shorter than the call, through the Python binding
+    (its ctypes marshalling is part of the figure)."""
+    import torch
+
+    out = {}
+    B, T, H, d = 1, 128, 2, 64
+    q = torch.zeros(B, T, H, d, dtype=torch.bfloat16, device=dev)
+    g = torch.full((H,), 0.95, device=dev)
+    o = torch.empty_like(q)
+    s = torch.zeros(B, H, d, d, device=dev)
+    for name, fn in (
+        ("lasad_forward", lambda: ctx.lasad_forward(q, q, q, g, 16, o=o, state_out=s)),
+        ("lasad_decode_step", lambda: ctx.lasad_decode_step(q[:, 0], q[:, 0], q[:, 0], g, s, 16, 0, 5, o=o[:, 0])),
+    ):
+        for _ in range(20):
+            fn()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(calls):
+            fn()
+        t1 = time.perf_counter()
+        torch.cuda.synchronize()
+        out[name] = round((t1 - t0) / calls * 1e6, 2)
+    out["note"] = f"{calls} enqueue-only calls each, B={B} H={H} T={T} (prefill) / one token (decode), Python binding included"
+    return out
+
+
+def scaling_sweep(ctx, dev, cpu: bool, grids=(16, 24, 32, 64, 96), reps: int = 10):
+    """Prefill throughput against sequence length N on the config 5 shape (B=8, H=24, d=64, bf16):
+    the GPU kernel (library default), and on the host cores the oracle's recurrent form (linear in N)
+    and its quadratic form (the explicit masked-decay sum, N^2).  The oracle runs on a subset of the
+    (batch, head) chains -- every chain costs the same -- and its time is scaled to all of them."""
+    import torch
+
+    from paper_2507_01652_b200 import workloads
+
+    stream = torch.cuda.current_stream()
+    flush = L2Flush(dev)
+    base = workloads.WORKLOADS["config5b"]
+    points = []
+    for gsz in grids:
+        wl = dataclasses.replace(base, grid_h=gsz, grid_w=gsz, name=f"config5 shape, {gsz}x{gsz} grid")
+        q, k, v = workloads.make_qkv(wl)
+        g = workloads.make_decay(wl)
+        dq, dk, dv, dg = q.to(dev), k.to(dev), v.to(dev), g.to(dev)
+        o = torch.empty_like(dv)
+        s_out = torch.empty(wl.B, wl.H, wl.d, wl.d, dtype=torch.float32, device=dev)
+        nbytes = prefill_bytes(wl)
+        ms = _time_launches(stream, flush, nbytes, reps,
+                            lambda: ctx.lasad_forward(dq, dk, dv, dg, wl.grid_w, o=o, state_out=s_out))
+        pt = {"N": wl.T, "grid": f"{gsz}x{gsz}", "gpu_kernel_us": round(ms * 1e3, 2),
+              "gpu_tokens_per_s": round(wl.B * wl.T / (ms * 1e-3), 1), "l2_policy": flush.policy(nbytes)}
+        del dq, dk, dv, o
+        if cpu:
+            from oracle import lasad_oracle as orc
+
+            # batch 0, as many heads as there are host threads (at most all 24)
+            nh = max(1, min(wl.H, orc.threads()))
+            sl = (slice(0, 1), slice(None), slice(0, nh))
+            q64, k64, v64 = [t[sl].to(torch.float64).numpy() for t in (q, k, v)]
+            g64 = g[:nh].to(torch.float64).numpy()
+            scale_up = wl.B * wl.H / nh
+            for form, fn in (("recurrent", orc.recurrent), ("quadratic", orc.quadratic)):
+                best = None
+                for _ in range(2 if wl.T <= 1024 else 1):
+                    t0 = time.perf_counter()
+                    fn(q64, k64, v64, g64, wl.grid_w)
+                    dt = time.perf_counter() - t0
+                    best = dt if best is None else min(best, dt)
+                pt[f"oracle_{form}_tokens_per_s"] = round(wl.B * wl.T / (best * scale_up), 1)
+                pt[f"oracle_{form}_sample_s"] = round(best, 3)
+            pt["oracle_sample"] = f"batch 0, heads 0..{nh - 1} ({nh} of {wl.B * wl.H} chains, {orc.threads()} threads), time scaled by {scale_up:g}"
+        points.append(pt)
+    return {"shape": "B=8 H=24 d=64 bf16 (config 5), prefill, library default kernel", "points": points}
+
+
+def run_decode(args, ctx, peaks, dev, rank, barrier, max_ranks, K, workload=None, hot: bool = True):
+    """Decode sweep: persistent fp32 state, one `lasad_decode_step` per grid position (`workload`:
+    a configuration's name; default: --decode-workload, the config 4 shape)."""
     import torch
 
     from paper_2507_01652_b200 import workloads
 
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(dev.index)
-    dw = workloads.WORKLOADS[args.decode_workload]
-    if args.decode_batch:
+    dw = workloads.WORKLOADS[workload or args.decode_workload]
+    if args.decode_batch and workload is None:
         dw = dw.scaled(B=args.decode_batch)
     dw = dataclasses.replace(dw, seed=rank_seed(dw.seed, rank))
     P = dw.prefix_len
     dq, dk_, dv_ = [t.to(dev) for t in workloads.make_qkv(dw)]
     dg = workloads.make_decay(dw).to(dev)
-    n_sets = 3  # rotating state sets: together > 2x L2, so no step finds its state in L2
+    # rotating state sets: together > 2x L2, so no step finds its state in L2
+    state_bytes = dw.B * dw.H * dw.d * dw.d * 4
+    n_sets = max(3, -(-2 * L2_BYTES // state_bytes) + 1)
     states = [torch.zeros(dw.B, dw.H, dw.d, dw.d, dtype=torch.float32, device=dev) for _ in range(n_sets)]
     do = torch.empty(dw.B, dw.H, dw.d, dtype=dq.dtype, device=dev)
     positions = list(range(P, dw.T))
@@ -460,7 +577,7 @@ def run_decode(args, ctx, peaks, dev, rank, barrier, max_ranks, K):
                                   dw.grid_w, P, t, o=do)
 
     dec = {}
-    for mode, cold in (("cold", True), ("hot", False)):
+    for mode, cold in (("cold", True), ("hot", False)) if hot else (("cold", True),):
         reset_states()
         sweep(cold)  # warm-up sweep
         barrier()
@@ -507,14 +624,15 @@ def run_decode(args, ctx, peaks, dev, rank, barrier, max_ranks, K):
         "workload": f"{dw.name}: B={dw.B} H={dw.H} d={dw.d} grid={dw.grid_h}x{dw.grid_w} prefix={P}, "
                     f"{len(positions)} positions, bf16 q/k/v/o, fp32 state",
         "us_per_step_cold_stream": round(dec["cold"], 3),
-        "us_per_step_hot_stream": round(dec["hot"], 3),
+        "us_per_step_hot_stream": round(dec["hot"], 3) if "hot" in dec else None,
         "us_per_step_cold_graph": None if graph_us is None else round(graph_us, 3),
         "bytes_per_step": dbytes,
         "states_rotated": n_sets,
         "roofline": {"bound": "hbm", "achieved": round(dbytes / (best_us * 1e-6) / 1e9, 1),
                      "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": round(dbytes / (best_us * 1e-6) / 1e9 / peaks["hbm_gbs"], 4),
-                     "traffic": NCU_TRAFFIC_BYTES["decode"] if dw.name == "config4" else None, "peak_source": peaks["source"],
+                     "traffic": NCU_TRAFFIC_BYTES["decode"] if (dw.name == "config4" and dw.B == 256) else None,
+                     "peak_source": peaks["source"],
                      "timed": "cold sweep, CUDA graph" if graph_us is not None else "cold sweep, stream"},
     }
     if "graph_error" in dec:

@@ -35,8 +35,16 @@
  * Layout: q,k [B,T,H,dk], v [B,T,H,dv], o [B,T,H,dv], state [B,H,dk,dv], all
  * contiguous doubles.  state_in may be NULL (s_0 = 0); state_out may be NULL.
  *
- * Parity pins for both functions live in tests/test_oracle_pins.py.
+ * A third function, lasad_oracle_layer_core, is Algorithm 1's loop body with the
+ * operator's neighbours inside: q_t = SiLU(q~_t), lambda_t = Sigmoid(g~_t),
+ * k_t = 1 - lambda_t (or a supplied key), the decay select, the state update and the
+ * readout as above, and then Norm(o_t).  The paper does not say which norm; the
+ * reading taken is a weight-free RMS norm over the d_v channels of a head,
+ * o / sqrt(mean(o^2) + eps).
+ *
+ * Parity pins for all three functions live in tests/test_oracle_pins.py.
  */
+#include <math.h>
 #include <stddef.h>
 #include <stdint.h>
 #include <stdlib.h>
@@ -172,6 +180,64 @@ int lasad_oracle_quadratic(const lasad_oracle_dims* d,
                         for (int e = 0; e < dv; ++e) so[c * dv + e] += w[c] * sin[c * dv + e];
             }
             free(w);
+        }
+    }
+    return fail ? -1 : 0;
+}
+
+/*
+ * Algorithm 1's loop body including the operator's neighbours: per token
+ *     q_t = SiLU(q~_t),  lambda_t = Sigmoid(g~_t),  k_t = 1 - lambda_t (k == NULL) or the given key,
+ *     lambda_t^spatial = 1 at a row-boundary step, lambda_t otherwise,
+ *     s_t = diag(lambda_t^spatial) s_{t-1} + k_t v_t^T,   o_t^T = scale * q_t^T s_t,
+ *     out_t = o_t / sqrt(mean_e(o_t[e]^2) + eps)          (the norm reading stated at the top).
+ * q_pre, gate_pre [B,T,H,dk] are pre-activations; k may be NULL; layouts as above.
+ */
+int lasad_oracle_layer_core(const lasad_oracle_dims* d,
+                            const double* q_pre, const double* k, const double* v,
+                            const double* gate_pre, const double* state_in, double eps,
+                            double* o, double* state_out)
+{
+    const int B = d->B, T = d->T, H = d->H, dk = d->dk, dv = d->dv;
+    int fail = 0;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int b = 0; b < B; ++b) {
+        for (int h = 0; h < H; ++h) {
+            double* s = (double*)malloc(sizeof(double) * (dk * dv + 2 * dk));
+            if (!s) { fail = 1; continue; }
+            double* qt = s + dk * dv;   /* SiLU(q~_t) */
+            double* kt = qt + dk;       /* key of this token */
+            if (state_in)
+                memcpy(s, state_in + ((size_t)b * H + h) * dk * dv, sizeof(double) * dk * dv);
+            else
+                memset(s, 0, sizeof(double) * dk * dv);
+            for (int t = 0; t < T; ++t) {
+                const size_t row = ((size_t)b * T + t) * H + h;
+                const double* vt = v + row * dv;
+                double* ot = o + row * dv;
+                const int boundary = is_boundary(d, d->t0 + t);
+                for (int c = 0; c < dk; ++c) {
+                    const double x = q_pre[row * dk + c];
+                    qt[c] = x / (1.0 + exp(-x));                               /* SiLU */
+                    const double lam = 1.0 / (1.0 + exp(-gate_pre[row * dk + c])); /* Sigmoid */
+                    kt[c] = k ? k[row * dk + c] : 1.0 - lam;
+                    const double lam_spatial = boundary ? 1.0 : lam;
+                    for (int e = 0; e < dv; ++e)
+                        s[c * dv + e] = lam_spatial * s[c * dv + e] + kt[c] * vt[e];
+                }
+                double ss = 0.0;
+                for (int e = 0; e < dv; ++e) {
+                    double acc = 0.0;
+                    for (int c = 0; c < dk; ++c) acc += qt[c] * s[c * dv + e];
+                    ot[e] = d->scale * acc;
+                    ss += ot[e] * ot[e];
+                }
+                const double r = 1.0 / sqrt(ss / dv + eps);
+                for (int e = 0; e < dv; ++e) ot[e] *= r;
+            }
+            if (state_out)
+                memcpy(state_out + ((size_t)b * H + h) * dk * dv, s, sizeof(double) * dk * dv);
+            free(s);
         }
     }
     return fail ? -1 : 0;

@@ -45,8 +45,9 @@ def test_prefill_full_size_sampled_chains(ctx, name):
         assert rel_err(s[b:b + 1, h:h + 1], s_ref) <= TOL[torch.bfloat16], (b, h)
 
 
-def test_gated_prefill_full_size_sampled_chains(ctx):
-    wl = workloads.WORKLOADS["config3"]
+@pytest.mark.parametrize("name", ["config3", "config5b"])
+def test_gated_prefill_full_size_sampled_chains(ctx, name):
+    wl = workloads.WORKLOADS[name]
     q, k, v = workloads.make_qkv(wl)
     lam = workloads.make_gate(wl)
     o, s = ctx.lasad_forward_gated(q.cuda(), k.cuda(), v.cuda(), lam.cuda(), wl.grid_w, prefix_len=wl.prefix_len)
@@ -62,9 +63,10 @@ def test_gated_prefill_full_size_sampled_chains(ctx):
 
 def test_decode_full_size_config4_sampled_chains(ctx):
     """Config 4 as the bench runs it: one prefill call for the class token, then one decode step per
-    grid token on all 256 x 20 states; sampled chains against the oracle over the whole sequence."""
+    grid token (all 256 of them) on all 256 x 20 states; sampled chains against the oracle over the
+    whole 257-token sequence."""
     wl = workloads.WORKLOADS["config4"]
-    T = wl.prefix_len + 64                     # class token + four grid rows: every kind of step occurs
+    T = wl.T                                   # class token + all 256 grid positions
     q, k, v = workloads.make_qkv(wl, T)
     g = workloads.make_decay(wl)
     dq, dk, dv, dg = q.cuda(), k.cuda(), v.cuda(), g.cuda()

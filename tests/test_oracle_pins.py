@@ -200,6 +200,43 @@ def test_data_dependent_decay_bruteforce(form):
         np.testing.assert_allclose(o[0, t, 0], acc, rtol=1e-12, atol=1e-13)
 
 
+@pytest.mark.parametrize("form", FORMS, ids=FORM_IDS)
+def test_data_dependent_decay_with_incoming_state_bruteforce(form):
+    """Per-token, per-channel decays on top of a non-zero incoming state, a prefix token and a start
+    in mid-row: outputs and the final state from explicit products over the steps (Section 3.4,
+    the SAD recurrence unrolled; the boundary step multiplies by exactly 1)."""
+    w, T, dk, dv, P, t0, scale = 3, 8, 2, 3, 1, 2, 0.5
+    rng = np.random.default_rng(116)
+    q, k, v = _rand((1, T, 1, dk), 117), _rand((1, T, 1, dk), 118), _rand((1, T, 1, dv), 119)
+    lam = rng.uniform(0.2, 1.0, size=(1, T, 1, dk))
+    s_in = _rand((1, 1, dk, dv), 120)
+    o, s_out = form(q, k, v, lam, w, P, t0, scale, s_in)
+
+    def step_decay(u, c):       # decay of local step u (absolute index t0 + u), channel c
+        i = t0 + u
+        boundary = i >= P and (i - P + 1) % w == 0
+        return 1.0 if boundary else lam[0, u, 0, c]
+
+    def prod(lo, hi, c):        # product over local steps lo .. hi (inclusive)
+        p = 1.0
+        for u in range(lo, hi + 1):
+            p *= step_decay(u, c)
+        return p
+
+    for t in range(T):
+        acc = np.zeros(dv)
+        for c in range(dk):
+            acc += q[0, t, 0, c] * prod(0, t, c) * s_in[0, 0, c]
+            for j in range(t + 1):
+                acc += q[0, t, 0, c] * k[0, j, 0, c] * prod(j + 1, t, c) * v[0, j, 0]
+        np.testing.assert_allclose(o[0, t, 0], scale * acc, rtol=1e-12, atol=1e-13)
+    for c in range(dk):
+        row = prod(0, T - 1, c) * s_in[0, 0, c]
+        for j in range(T):
+            row = row + prod(j + 1, T - 1, c) * k[0, j, 0, c] * v[0, j, 0]
+        np.testing.assert_allclose(s_out[0, 0, c], row, rtol=1e-12, atol=1e-13)
+
+
 # ---------------------------------------------------------------------------------------------
 # the two statements of the method agree (equation vs algorithm)
 # ---------------------------------------------------------------------------------------------
@@ -316,3 +353,65 @@ def test_zero_decay_keeps_only_current_row_segment(form):
     ones = np.ones((1, T, 1, 1))
     o, _ = form(ones, ones, ones, np.array([0.0]), w)
     np.testing.assert_array_equal(o[0, :, 0, 0], [1, 1, 2, 1, 1, 2])
+
+
+# ---------------------------------------------------------------------------------------------
+# Algorithm 1's loop body with its neighbours (SiLU, Sigmoid, tied key, Norm)
+# ---------------------------------------------------------------------------------------------
+def _np_silu(x):
+    return x / (1.0 + np.exp(-x))
+
+
+def _np_sigmoid(x):
+    return 1.0 / (1.0 + np.exp(-x))
+
+
+def test_layer_core_single_token_closed_form():
+    """One token from a zero state: s = k v^T, o = (q . k) v, so the normalised output is
+    v / rms(v) times the sign of q . k, whatever the gate's decay (s_0 = 0 makes it moot)."""
+    dk, dv = 3, 4
+    q_pre = np.array([0.3, -1.2, 2.0]).reshape(1, 1, 1, dk)
+    g_pre = np.array([1.5, -0.4, 0.0]).reshape(1, 1, 1, dk)
+    v = np.array([0.5, -1.0, 2.0, 0.25]).reshape(1, 1, 1, dv)
+    o, s = orc.layer_core(q_pre, None, v, g_pre, grid_w=4, eps=0.0)
+    q = _np_silu(q_pre[0, 0, 0])
+    k = 1.0 - _np_sigmoid(g_pre[0, 0, 0])
+    np.testing.assert_allclose(s[0, 0], np.outer(k, v[0, 0, 0]), rtol=1e-13)
+    dot = float(q @ k)
+    expect = np.sign(dot) * v[0, 0, 0] / np.sqrt(np.mean(v[0, 0, 0] ** 2))
+    np.testing.assert_allclose(o[0, 0, 0], expect, rtol=1e-12)
+    # known values of the activations: SiLU(0) = 0, Sigmoid(0) = 1/2 -> k = 1/2
+    np.testing.assert_allclose(k[2], 0.5, rtol=0, atol=1e-15)
+    o0, _ = orc.layer_core(np.zeros((1, 1, 1, dk)), None, v, g_pre, grid_w=4, eps=1.0)
+    np.testing.assert_allclose(o0, 0.0, atol=1e-15)      # q = SiLU(0) = 0, and eps keeps 0/0 away
+
+
+@pytest.mark.parametrize("tied", [True, False])
+def test_layer_core_is_activations_then_the_recurrence_then_the_norm(tied):
+    """The fused statement against its parts: numpy's SiLU / Sigmoid / RMS norm around the
+    (separately pinned) recurrent form with the gate as a per-token, per-channel decay; prefix,
+    start in mid-row, incoming state, scale and eps all in play."""
+    B, T, H, dk, dv, w, P, t0, scale, eps = 2, 19, 3, 4, 5, 4, 1, 3, 0.7, 1e-3
+    q_pre, g_pre, v = _rand((B, T, H, dk), 301) * 2, _rand((B, T, H, dk), 302) * 2 + 1.0, _rand((B, T, H, dv), 303)
+    k_in = None if tied else _rand((B, T, H, dk), 304)
+    s_in = _rand((B, H, dk, dv), 305)
+    o, s = orc.layer_core(q_pre, k_in, v, g_pre, w, P, t0, scale, s_in, eps)
+    lam = _np_sigmoid(g_pre)
+    k = 1.0 - lam if tied else k_in
+    o_raw, s_ref = orc.recurrent(_np_silu(q_pre), k, v, lam, w, P, t0, scale, s_in)
+    o_ref = o_raw / np.sqrt(np.mean(o_raw ** 2, axis=-1, keepdims=True) + eps)
+    np.testing.assert_allclose(o, o_ref, rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(s, s_ref, rtol=1e-11, atol=1e-12)
+
+
+def test_layer_core_norm_properties():
+    """Each head's normalised output has unit RMS when eps = 0, and scaling v (hence o) leaves it
+    unchanged; with eps > 0 a small output is shrunk, not blown up."""
+    B, T, H, dk, dv = 1, 12, 2, 4, 8
+    q_pre, g_pre, v = _rand((B, T, H, dk), 311), _rand((B, T, H, dk), 312) + 2.0, _rand((B, T, H, dv), 313)
+    o, _ = orc.layer_core(q_pre, None, v, g_pre, 3, eps=0.0)
+    np.testing.assert_allclose(np.sqrt(np.mean(o ** 2, axis=-1)), 1.0, rtol=1e-12)
+    o10, _ = orc.layer_core(q_pre, None, 10.0 * v, g_pre, 3, eps=0.0)
+    np.testing.assert_allclose(o10, o, rtol=1e-11, atol=1e-13)
+    o_eps, _ = orc.layer_core(q_pre, None, 1e-6 * v, g_pre, 3, eps=1.0)
+    assert np.abs(o_eps).max() < 1e-4

@@ -433,6 +433,37 @@ def gated_sweep(ctx, peaks, dev, wls=None, decode: bool = True, reps: int = 10):
                                "frac_of_hbm_peak": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
                                "l2_policy": flush.policy(nbytes)})
         del q, k, v, lam, o, s_out
+    # Algorithm 1's loop body as one call (SiLU, Sigmoid, tied key, operator, RMS norm) against the
+    # same computation as separate kernels: torch's element-wise kernels around lasad_forward_gated
+    out["fused"] = []
+    for wl in wls[1:]:
+        gen = torch.Generator().manual_seed(wl.seed + 11)
+        qp = torch.randn(wl.B, wl.T, wl.H, wl.d, generator=gen).to(wl.torch_dtype).to(dev)
+        gp = (torch.randn(wl.B, wl.T, wl.H, wl.d, generator=gen) + 2.0).to(wl.torch_dtype).to(dev)
+        v = workloads.make_qkv(wl)[2].to(dev)
+        o = torch.empty_like(v)
+        s_out = torch.empty(wl.B, wl.H, wl.d, wl.d, dtype=torch.float32, device=dev)
+        unit = wl.B * wl.T * wl.H * wl.d * wl.elem_bytes       # one [B,T,H,d] tensor
+        state_b = wl.B * wl.H * wl.d * wl.d * 4
+        fused_bytes = 4 * unit + state_b                       # q~, gate~, v in, o out
+        unfused_bytes = 2 * unit + 2 * unit + 3 * unit + (4 * unit + state_b) + 2 * unit   # SiLU, Sigmoid, 1 - lambda, operator, norm
+
+        def unfused():
+            lam = torch.sigmoid(gp)
+            oo, _ = ctx.lasad_forward_gated(torch.nn.functional.silu(qp), 1.0 - lam, v, lam, wl.grid_w,
+                                            prefix_len=wl.prefix_len, o=o, state_out=s_out)
+            return torch.nn.functional.rms_norm(oo, (wl.d,), eps=1e-6)
+
+        ms_f = _time_launches(stream, flush, fused_bytes, reps,
+                              lambda: ctx.lasad_forward_fused(qp, None, v, gp, wl.grid_w, prefix_len=wl.prefix_len, o=o,
+                                                              state_out=s_out, norm_eps=1e-6))
+        ms_u = _time_launches(stream, flush, fused_bytes, reps, unfused)
+        out["fused"].append({"workload": f"{wl.name}: B={wl.B} H={wl.H} T={wl.T} d={wl.d} {wl.dtype}, key tied to the gate",
+                             "fused_us": round(ms_f * 1e3, 2), "unfused_us": round(ms_u * 1e3, 2),
+                             "fused_bytes": fused_bytes, "unfused_bytes": unfused_bytes,
+                             "fused_frac_of_hbm_peak": round(fused_bytes / (ms_f * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                             "unfused": "torch.sigmoid, F.silu, 1 - lambda, lasad_forward_gated, F.rms_norm (five kernels + the operator's two)"})
+        del qp, gp, v, o, s_out
     if not decode:
         return out
     dw = workloads.WORKLOADS["config4"]

@@ -234,6 +234,39 @@ int lasad_decode_step_gated(lasad_ctx* ctx, const lasad_params* p,
                             const void* q, const void* k, const void* v, const void* gate,
                             float* state, void* o, void* cuda_stream);
 
+/*
+ * Algorithm 1's loop body as a whole: the operator together with the element-wise steps the
+ * algorithm puts around it, so that q, the gate and o each cross device memory once instead of
+ * three times.  Per token (Algorithm 1, in its order):
+ *
+ *     q_t = SiLU(q_pre_t)            lambda_t = Sigmoid(gate_pre_t)            k_t = 1 - lambda_t  (k == NULL)
+ *     s_t = diag(lambda_t^spatial) s_{t-1} + k_t v_t^T      o_t = scale * q_t^T s_t      (Section 3.4, SAD rule)
+ *     out_t = Norm(o_t)
+ *
+ * The paper does not say which norm follows the operator; the reading taken here is a weight-free
+ * RMS norm over the dv channels of each head, out = o / sqrt(mean(o^2) + norm_eps), norm_eps >= 0
+ * (a learned per-channel weight, if the model has one, folds into the output projection that
+ * follows).  The output projection itself and the input projections are dense matrix products and
+ * are not part of these calls.
+ *
+ *   q_pre, gate_pre   pre-activations, with the layouts, dtypes and strides of q and gate in
+ *                     lasad_forward_gated / lasad_decode_step_gated (gate_pre is described by k_stride)
+ *   k                 an explicit key (then not tied to the gate), or NULL for Algorithm 1's k = 1 - lambda
+ *   o                 receives the normalised output; state, state_in, state_out as in the gated calls
+ *
+ * Arithmetic: activations, decay products, accumulation, state and norm in fp32; with BF16 I/O
+ * and dk == dv == 64 the contractions run on the tensor cores with bf16 operands, as in
+ * lasad_forward_gated, and the same two-launch scheme covers every gate value.  1 - lambda is
+ * formed as Sigmoid(-gate_pre), not by subtraction, so a gate close to 1 keeps its precision.
+ */
+int lasad_forward_fused(lasad_ctx* ctx, const lasad_params* p,
+                        const void* q_pre, const void* k, const void* v, const void* gate_pre,
+                        const float* state_in, void* o, float* state_out, float norm_eps,
+                        void* cuda_stream);
+int lasad_decode_step_fused(lasad_ctx* ctx, const lasad_params* p,
+                            const void* q_pre, const void* k, const void* v, const void* gate_pre,
+                            float* state, void* o, float norm_eps, void* cuda_stream);
+
 /* After the caller has synchronised the stream: 0, or LASAD_ERR_TIMEOUT if a kernel gave up a
  * bounded wait since the last query (the flag is cleared by the query).  Synchronous copy. */
 int lasad_last_device_status(lasad_ctx* ctx, int* status);

@@ -29,6 +29,7 @@ LASAD_OPT_WAIT_LIMIT = 3
 EXPORTS = (
     "lasad_create", "lasad_destroy", "lasad_set_option", "lasad_reserve", "lasad_forward", "lasad_forward_host", "lasad_forward_static",
     "lasad_decode_step", "lasad_decode_step_pos", "lasad_forward_gated", "lasad_decode_step_gated",
+    "lasad_forward_fused", "lasad_decode_step_fused",
     "lasad_last_device_status", "lasad_last_cuda_error", "lasad_launch_count", "lasad_strerror",
 )
 
@@ -88,6 +89,10 @@ def load_library() -> ctypes.CDLL:
         lib.lasad_forward_gated.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.lasad_decode_step_gated.restype = i32
         lib.lasad_decode_step_gated.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp]
+        lib.lasad_forward_fused.restype = i32
+        lib.lasad_forward_fused.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp]
+        lib.lasad_decode_step_fused.restype = i32
+        lib.lasad_decode_step_fused.argtypes = [vp, pp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp]
         lib.lasad_last_device_status.restype = i32
         lib.lasad_last_device_status.argtypes = [vp, ctypes.POINTER(i32)]
         lib.lasad_last_cuda_error.restype = i32
@@ -244,29 +249,6 @@ class Lasad:
             self._raise(rc, "lasad_decode_step")
         return o
 
-
-def lasad_forward_static(q, k, v, decay, grid_w, o, state_out=None, prefix_len=0, t0=0, scale=1.0,
-                         state_in=None, device_status=None, stream=None):
-    """``lasad_forward_static``: prefill on q's device with no context and no allocation.
-
-    Every buffer, the output ``o`` included, is the caller's: this wrapper allocates nothing either.
-    ``device_status`` is an optional int32 CUDA tensor of one element.  Raises on an error code."""
-    _check_cuda(q, k, v, decay, state_in, o, state_out, device_status)
-    B, T, H, dk = q.shape
-    dv = v.shape[3]
-    p = LasadParams(B, T, H, dk, dv, grid_w, prefix_len, _dtype_code(q), t0, scale, 0,
-                    _strides3(q), _strides3(k), _strides3(v), _strides3(o))
-    lib = load_library()
-    with torch.cuda.device(q.device):
-        st = torch.cuda.current_stream(q.device).cuda_stream if stream is None else stream
-        rc = lib.lasad_forward_static(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(decay), _ptr(state_in),
-                                      _ptr(o), _ptr(state_out), _ptr(device_status), ctypes.c_void_p(st))
-    if rc != LASAD_OK:
-        raise LasadError(rc, "lasad_forward_static")
-    return o, state_out
-
-
-def _gated_methods():
     def lasad_forward_gated(self, q, k, v, gate, grid_w, prefix_len=0, t0=0, scale=1.0, state_in=None, o=None,
                             state_out=None, want_state=True, stream=None):
         """Prefill with a data-dependent gate [B,T,H,dk]; ``k=None`` ties the key to the gate
@@ -336,12 +318,78 @@ def _gated_methods():
             self._raise(rc, "lasad_decode_step_pos")
         return o
 
-    Lasad.lasad_decode_step_pos = lasad_decode_step_pos
-    Lasad.lasad_forward_gated = lasad_forward_gated
-    Lasad.lasad_decode_step_gated = lasad_decode_step_gated
+    def lasad_forward_fused(self, q_pre, k, v, gate_pre, grid_w, prefix_len=0, t0=0, scale=1.0, state_in=None,
+                            o=None, state_out=None, want_state=True, norm_eps=1e-6, stream=None):
+        """Algorithm 1's loop body as one call: SiLU on ``q_pre``, Sigmoid on ``gate_pre``, ``k=None``
+        ties the key to the gate, RMS norm on the output.  Returns (normalised o, state_out)."""
+        _check_cuda(q_pre, k, v, gate_pre, state_in, o, state_out)
+        B, T, H, dk = q_pre.shape
+        dv = v.shape[3]
+        if o is None:
+            o = torch.empty((B, T, H, dv), dtype=q_pre.dtype, device=q_pre.device)
+        if state_out is None and want_state:
+            state_out = torch.empty((B, H, dk, dv), dtype=torch.float32, device=q_pre.device)
+        if gate_pre.dtype != q_pre.dtype or tuple(gate_pre.shape) != tuple(q_pre.shape):
+            raise ValueError("gate_pre must have q_pre's shape and dtype")
+        if k is not None and tuple(k.stride()) != tuple(gate_pre.stride()):
+            raise ValueError("k and gate_pre must share strides")
+        p = LasadParams(B, T, H, dk, dv, grid_w, prefix_len, _dtype_code(q_pre), t0, scale, 0,
+                        _strides3(q_pre), _strides3(gate_pre), _strides3(v), _strides3(o))
+        st = torch.cuda.current_stream(q_pre.device).cuda_stream if stream is None else stream
+        rc = self._lib.lasad_forward_fused(self._h, ctypes.byref(p), _ptr(q_pre), _ptr(k), _ptr(v), _ptr(gate_pre),
+                                           _ptr(state_in), _ptr(o), _ptr(state_out), float(norm_eps),
+                                           ctypes.c_void_p(st))
+        if rc != LASAD_OK:
+            self._raise(rc, "lasad_forward_fused")
+        return o, state_out
+
+    def lasad_decode_step_fused(self, q_pre, k, v, gate_pre, state, grid_w, prefix_len, t, scale=1.0, o=None,
+                                norm_eps=1e-6, stream=None):
+        """One generation step of Algorithm 1's loop body (activations, state update, readout, norm);
+        ``state`` is updated in place.  q_pre, gate_pre, v are [B,H,d]."""
+        _check_cuda(q_pre, k, v, gate_pre, state, o)
+        B, H, dk = q_pre.shape
+        dv = v.shape[2]
+        if o is None:
+            o = torch.empty((B, H, dv), dtype=q_pre.dtype, device=q_pre.device)
+        if state.dtype != torch.float32 or not state.is_contiguous() or tuple(state.shape) != (B, H, dk, dv):
+            raise ValueError("state must be contiguous float32 [B,H,dk,dv]")
+        if gate_pre.dtype != q_pre.dtype or tuple(gate_pre.shape) != tuple(q_pre.shape):
+            raise ValueError("gate_pre must have q_pre's shape and dtype")
+        if k is not None and tuple(k.stride()) != tuple(gate_pre.stride()):
+            raise ValueError("k and gate_pre must share strides")
+        p = LasadParams(B, 1, H, dk, dv, grid_w, prefix_len, _dtype_code(q_pre), t, scale, 0,
+                        _strides_decode(q_pre), _strides_decode(gate_pre), _strides_decode(v), _strides_decode(o))
+        st = torch.cuda.current_stream(q_pre.device).cuda_stream if stream is None else stream
+        rc = self._lib.lasad_decode_step_fused(self._h, ctypes.byref(p), _ptr(q_pre), _ptr(k), _ptr(v),
+                                               _ptr(gate_pre), _ptr(state), _ptr(o), float(norm_eps),
+                                               ctypes.c_void_p(st))
+        if rc != LASAD_OK:
+            self._raise(rc, "lasad_decode_step_fused")
+        return o
 
 
-_gated_methods()
+def lasad_forward_static(q, k, v, decay, grid_w, o, state_out=None, prefix_len=0, t0=0, scale=1.0,
+                         state_in=None, device_status=None, stream=None):
+    """``lasad_forward_static``: prefill on q's device with no context and no allocation.
+
+    Every buffer, the output ``o`` included, is the caller's: this wrapper allocates nothing either.
+    ``device_status`` is an optional int32 CUDA tensor of one element.  Raises on an error code."""
+    _check_cuda(q, k, v, decay, state_in, o, state_out, device_status)
+    B, T, H, dk = q.shape
+    dv = v.shape[3]
+    p = LasadParams(B, T, H, dk, dv, grid_w, prefix_len, _dtype_code(q), t0, scale, 0,
+                    _strides3(q), _strides3(k), _strides3(v), _strides3(o))
+    lib = load_library()
+    with torch.cuda.device(q.device):
+        st = torch.cuda.current_stream(q.device).cuda_stream if stream is None else stream
+        rc = lib.lasad_forward_static(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(decay), _ptr(state_in),
+                                      _ptr(o), _ptr(state_out), _ptr(device_status), ctypes.c_void_p(st))
+    if rc != LASAD_OK:
+        raise LasadError(rc, "lasad_forward_static")
+    return o, state_out
+
+
 
 _default = {}
 

@@ -423,8 +423,14 @@ int lasad_decode_step_pos(lasad_ctx* ctx, const lasad_params* p, const void* q, 
     return LASAD_OK;
 }
 
-int lasad_forward_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
-                        const void* gate, const float* state_in, void* o, float* state_out, void* cuda_stream)
+}  // extern "C"
+
+namespace {
+
+// lasad_forward_gated (fused = false) and lasad_forward_fused (fused = true)
+int forward_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
+                  const void* gate, const float* state_in, void* o, float* state_out, bool fused, float norm_eps,
+                  void* cuda_stream)
 {
     int rc = check_common(ctx, p, false);
     if (rc != LASAD_OK) return rc;
@@ -437,6 +443,7 @@ int lasad_forward_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, co
     fill_args(a, ctx, p);
     a.q = q; a.k = k; a.v = v; a.o = o;
     a.decay = nullptr; a.state_in = state_in; a.state_out = state_out;
+    a.fused = fused ? 1 : 0; a.norm_eps = norm_eps;
     // tensor cores where the shape allows it, unless the CUDA-core implementation is asked for
     const bool bf16 = p->dtype == LASAD_BF16;
     const bool tc = ctx->opt_prefill_impl != 1 && lasad::prefill_gated_tc_supported(p->dk, p->dv, bf16);
@@ -461,8 +468,9 @@ int lasad_forward_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, co
     return LASAD_OK;
 }
 
-int lasad_decode_step_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
-                            const void* gate, float* state, void* o, void* cuda_stream)
+// lasad_decode_step_gated (fused = false) and lasad_decode_step_fused (fused = true)
+int decode_step_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
+                      const void* gate, float* state, void* o, bool fused, float norm_eps, void* cuda_stream)
 {
     int rc = check_common(ctx, p, true);
     if (rc != LASAD_OK) return rc;
@@ -475,6 +483,7 @@ int lasad_decode_step_gated(lasad_ctx* ctx, const lasad_params* p, const void* q
     a.T = 1;
     a.q = q; a.k = k; a.v = v; a.o = o;
     a.decay = nullptr; a.state_in = state; a.state_out = state;
+    a.fused = fused ? 1 : 0; a.norm_eps = norm_eps;
     // SAD rule (Algorithm 1's if-statement): the decay is 1 on a row-boundary step
     const bool decay_on = !lasad::is_boundary_step(p->t0, p->grid_w, p->prefix_len);
     int tpu = ctx->opt_decode_tpu;
@@ -484,6 +493,37 @@ int lasad_decode_step_gated(lasad_ctx* ctx, const lasad_params* p, const void* q
     if (e != cudaSuccess) return fail_cuda(ctx, e);
     ctx->launches += 1;
     return LASAD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lasad_forward_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
+                        const void* gate, const float* state_in, void* o, float* state_out, void* cuda_stream)
+{
+    return forward_gated(ctx, p, q, k, v, gate, state_in, o, state_out, false, 0.0f, cuda_stream);
+}
+
+int lasad_forward_fused(lasad_ctx* ctx, const lasad_params* p, const void* q_pre, const void* k, const void* v,
+                        const void* gate_pre, const float* state_in, void* o, float* state_out, float norm_eps,
+                        void* cuda_stream)
+{
+    if (!(norm_eps >= 0.0f) || !std::isfinite(norm_eps)) return LASAD_ERR_INVALID_ARG;
+    return forward_gated(ctx, p, q_pre, k, v, gate_pre, state_in, o, state_out, true, norm_eps, cuda_stream);
+}
+
+int lasad_decode_step_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,
+                            const void* gate, float* state, void* o, void* cuda_stream)
+{
+    return decode_step_gated(ctx, p, q, k, v, gate, state, o, false, 0.0f, cuda_stream);
+}
+
+int lasad_decode_step_fused(lasad_ctx* ctx, const lasad_params* p, const void* q_pre, const void* k, const void* v,
+                            const void* gate_pre, float* state, void* o, float norm_eps, void* cuda_stream)
+{
+    if (!(norm_eps >= 0.0f) || !std::isfinite(norm_eps)) return LASAD_ERR_INVALID_ARG;
+    return decode_step_gated(ctx, p, q_pre, k, v, gate_pre, state, o, true, norm_eps, cuda_stream);
 }
 
 int lasad_forward_host(lasad_ctx* ctx, const lasad_params* p, const void* q, const void* k, const void* v,

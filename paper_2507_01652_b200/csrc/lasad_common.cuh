@@ -28,7 +28,28 @@ struct KernelArgs {
                             // prefill kernels), [2] launches of the balanced prefill so far
     float* seg_state;       // prefill, CTA-per-chain kernel: room for 2 x SMs states, or nullptr (chains are not cut)
     unsigned wait_limit;
+    // gated entry points only: q and the gate are pre-activations (q <- SiLU(q), lambda <- Sigmoid(gate))
+    // and o leaves through a weight-free RMS norm over its dv channels with this epsilon
+    int fused;
+    float norm_eps;
 };
+
+// The operator's neighbours in Algorithm 1, evaluated in fp32 where the fused entry points need
+// them.  sigmoid_pair gives lambda = Sigmoid(x) and its complement 1 - lambda = Sigmoid(-x), each
+// to full relative precision (1 - lambda is the tied key, and it must not be formed by a
+// subtraction when lambda is close to 1).
+__device__ __forceinline__ void sigmoid_pair(float x, float& lam, float& one_minus_lam)
+{
+    const float t = __expf(-fminf(fmaxf(x, -80.0f), 80.0f));     // e^-x, finite
+    const float r = __frcp_rn(1.0f + t);
+    lam = r;
+    one_minus_lam = t * r;
+}
+__device__ __forceinline__ float silu(float x)
+{
+    const float t = __expf(-fminf(fmaxf(x, -80.0f), 80.0f));
+    return x * __frcp_rn(1.0f + t);
+}
 
 // Number of decaying (non-boundary) steps among absolute indices 0..i, from the token's 2-D
 // grid position alone (SAD rule, Section 3.4): a step decays unless it absorbs the last token

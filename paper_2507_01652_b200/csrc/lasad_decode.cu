@@ -43,9 +43,12 @@ template <> __device__ inline void store4<__nv_bfloat16>(__nv_bfloat16* p, const
 // GATED: the decay is the paper's data-dependent gate, a value per (batch, head, key channel)
 // read from `gate` with q's layout, and the key may be tied to it (k = 1 - lambda when a.k is
 // null); otherwise it is the per-head constant a.decay[h].
-template <typename T, int D, int TPU, bool GATED, bool POS>
+// FUSED (with GATED): q and the gate are pre-activations (q <- SiLU(q), lambda <- Sigmoid(gate))
+// and o leaves through a weight-free RMS norm over its D channels (Algorithm 1's loop body whole).
+template <typename T, int D, int TPU, bool GATED, bool POS, bool FUSED = false>
 __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on, const void* gate_v)
 {
+    static_assert(!FUSED || GATED, "the fused form exists for the gated operator");
     constexpr int CG = D / 4;          // threads per state row
     constexpr int RPP = TPU / CG;      // rows covered per pass
     constexpr int PASSES = D / RPP;    // float4s per thread
@@ -93,9 +96,12 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on,
             for (int u = 0; u < BATCH; ++u) {
                 const int row = r0 + (p0 + u) * RPP;
                 qr[u] = io<T>::load(q + row);
+                if (FUSED) qr[u] = silu(qr[u]);
                 if (GATED) {
-                    const float lr = io<T>::load(lam + row);
-                    kr[u] = k ? io<T>::load(k + row) : 1.0f - lr;     // key tied to the gate
+                    float lr = io<T>::load(lam + row);
+                    float tied = 1.0f - lr;
+                    if (FUSED) sigmoid_pair(lr, lr, tied);
+                    kr[u] = k ? io<T>::load(k + row) : tied;          // key tied to the gate
                     gr[u] = decay_on ? lr : 1.0f;                      // SAD rule: 1 on a boundary step
                 } else {
                     kr[u] = io<T>::load(k + row);
@@ -128,6 +134,15 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on,
             T* o = static_cast<T*>(a.o) + b * a.os[0] + h * a.os[2];
 #pragma unroll
             for (int c = 0; c < 4; ++c) acc[c] *= a.scale;
+            if (FUSED) {
+                // Norm(o): the D channels sit in lanes 0 .. CG-1, four each
+                float ss = acc[0] * acc[0] + acc[1] * acc[1] + acc[2] * acc[2] + acc[3] * acc[3];
+#pragma unroll
+                for (int off = CG / 2; off >= 1; off >>= 1) ss += __shfl_xor_sync((1u << CG) - 1u, ss, off);
+                const float nrm = rsqrtf(ss * (1.0f / D) + a.norm_eps);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) acc[c] *= nrm;
+            }
             store4<T>(o + cg * 4, acc);
         }
     } else {
@@ -147,12 +162,20 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on,
             T* o = static_cast<T*>(a.o) + b * a.os[0] + h * a.os[2];
 #pragma unroll
             for (int c = 0; c < 4; ++c) sum[c] *= a.scale;
+            if (FUSED) {
+                float ss = sum[0] * sum[0] + sum[1] * sum[1] + sum[2] * sum[2] + sum[3] * sum[3];
+#pragma unroll
+                for (int off = CG / 2; off >= 1; off >>= 1) ss += __shfl_xor_sync((1u << CG) - 1u, ss, off);
+                const float nrm = rsqrtf(ss * (1.0f / D) + a.norm_eps);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) sum[c] *= nrm;
+            }
             store4<T>(o + cg * 4, sum);
         }
     }
 }
 
-template <typename T, int D, bool GATED, bool POS>
+template <typename T, int D, bool GATED, bool POS, bool FUSED = false>
 cudaError_t launch_decode_t(const KernelArgs& a, bool decay_on, int tpu, const void* gate, cudaStream_t st)
 {
     const long long n_units = (long long)a.B * a.H;
@@ -160,7 +183,7 @@ cudaError_t launch_decode_t(const KernelArgs& a, bool decay_on, int tpu, const v
 #define LASAD_DECODE_CASE(TPU_)                                                               \
     case TPU_: {                                                                              \
         const long long blocks = (n_units + (256 / TPU_) - 1) / (256 / TPU_);                 \
-        decode_kernel<T, D, TPU_, GATED, POS><<<(unsigned)blocks, 256, 0, st>>>(a, on, gate); \
+        decode_kernel<T, D, TPU_, GATED, POS, FUSED><<<(unsigned)blocks, 256, 0, st>>>(a, on, gate); \
         break;                                                                                \
     }
     switch (tpu) {
@@ -199,6 +222,14 @@ cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool d
 cudaError_t launch_decode_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, bool decay_on, int tpu,
                                 cudaStream_t st)
 {
+    if (a.fused) {
+        if (dk == 64) {
+            return bf16 ? launch_decode_t<__nv_bfloat16, 64, true, false, true>(a, decay_on, tpu, gate, st)
+                        : launch_decode_t<float, 64, true, false, true>(a, decay_on, tpu, gate, st);
+        }
+        return bf16 ? launch_decode_t<__nv_bfloat16, 32, true, false, true>(a, decay_on, tpu, gate, st)
+                    : launch_decode_t<float, 32, true, false, true>(a, decay_on, tpu, gate, st);
+    }
     if (dk == 64) {
         return bf16 ? launch_decode_t<__nv_bfloat16, 64, true, false>(a, decay_on, tpu, gate, st)
                     : launch_decode_t<float, 64, true, false>(a, decay_on, tpu, gate, st);

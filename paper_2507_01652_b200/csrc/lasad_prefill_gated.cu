@@ -50,13 +50,20 @@ __global__ void __launch_bounds__(256) prefill_gated_kernel(KernelArgs a, const 
             const int r = x / D, c = x % D;
             const bool in = r < L;
             const long long t = cs + r;
-            float g = 1.0f, kk = 0.0f;
+            float g = 1.0f, kk = 0.0f, qq = 0.0f;
             if (in) {
                 g = io<T>::load(lam + t * a.ks[1] + c);
-                kk = k ? io<T>::load(k + t * a.ks[1] + c) : 1.0f - g;      // key tied to the gate
+                qq = io<T>::load(q + t * a.qs[1] + c);
+                float tied = 1.0f - g;
+                if (a.fused) {
+                    // Algorithm 1's activations: lambda = Sigmoid(gate), q = SiLU(q)
+                    sigmoid_pair(g, g, tied);
+                    qq = silu(qq);
+                }
+                kk = k ? io<T>::load(k + t * a.ks[1] + c) : tied;          // key tied to the gate
                 if (is_boundary_step(a.t0 + t, a.grid_w, a.prefix_len)) g = 1.0f;   // SAD rule
             }
-            Qs[r][c] = in ? io<T>::load(q + t * a.qs[1] + c) : 0.0f;
+            Qs[r][c] = qq;
             Ks[r][c] = kk;
             Vs[r][c] = in ? io<T>::load(v + t * a.vs[1] + c) : 0.0f;
             Ls[r][c] = g > 0.0f ? fmaxf(log2f(g), kMinLog2) : kMinLog2;   // log2 Lambda for now
@@ -104,10 +111,20 @@ __global__ void __launch_bounds__(256) prefill_gated_kernel(KernelArgs a, const 
 #pragma unroll
                 for (int m = 0; m < D / 16; ++m) acc[m] = fmaf(qc, Ss[c * LD + e0 + 16 * m], acc[m]);
             }
+            float norm = 1.0f;
+            if (a.fused) {
+                // Norm(o_t): weight-free RMS over the row's D channels, which sit in 16 adjacent lanes
+                float ss = 0.0f;
+#pragma unroll
+                for (int m = 0; m < D / 16; ++m) ss = fmaf(a.scale * acc[m], a.scale * acc[m], ss);
+#pragma unroll
+                for (int off = 8; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+                norm = rsqrtf(ss * (1.0f / D) + a.norm_eps);
+            }
             if (i < L) {
                 const long long t = cs + i;
 #pragma unroll
-                for (int m = 0; m < D / 16; ++m) io<T>::store(o + t * a.os[1] + e0 + 16 * m, a.scale * acc[m]);
+                for (int m = 0; m < D / 16; ++m) io<T>::store(o + t * a.os[1] + e0 + 16 * m, a.scale * acc[m] * norm);
             }
         }
         __syncthreads();

@@ -36,6 +36,14 @@
 // the warp's last row; log2 and exp2 only appear for the eight partial products per channel that
 // cross warps.
 //
+// Fused form (kFused; Algorithm 1's loop body whole): q and the gate arrive as pre-activations.
+// The first sweep turns the gate tile into u = Sigmoid(-g~) = 1 - lambda in place (bf16): the
+// complement keeps full relative precision where lambda is close to 1, which is where a rounding
+// of lambda itself would be felt over long ranges, and it is the tied key as it stands.  The
+// second sweep forms lambda = 1 - u in fp32 for its running products and applies SiLU to the
+// query as it scales it; the output tile leaves through a weight-free RMS norm over the head's
+// 64 channels (the two threads that hold a row exchange their sums of squares).
+//
 // Warp roles: warps 0-7 do the element-wise work.  For the scaling they split the chunk by rows
 // (warp w: rows 16 w ..), lanes across channel pairs, so the running sum b needs no exchange
 // inside a warp and only eight partial sums per channel cross warps through shared memory; for
@@ -88,6 +96,7 @@ struct Smem {
     unsigned char kt[kTileBytes];   // K~; after the MMAs the staging buffer of the output tile
     unsigned char sb[kD * kD * 2];  // bf16 copy of diag(2^r) state, [dk][dv], 128 B rows, swizzled
     float segsum[8][kD];            // log2 of the product of Lambda over rows 16 x .. 16 x + 15, per channel
+    float ssq[2][kC];               // fused form: sum of squares of each output row's two halves
     Barriers bar;
     uint32_t tmem_base;
     int abort_flag;
@@ -104,7 +113,21 @@ struct GatedParams {
     int* redo;               // [B*H]: 1 where this kernel gave the chain up (decay too strong), else 0
     int* status;
     unsigned wait_limit;
+    float norm_eps;          // fused form: epsilon of the output norm
 };
+
+__device__ __forceinline__ float rcp_approx(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float tanh_approx(float x)
+{
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 __device__ __forceinline__ float ex2(float x)
 {
@@ -127,6 +150,7 @@ __device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b)
     return r;
 }
 
+template <bool kFused>
 __global__ void __launch_bounds__(kThreads, 2)
 prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                         const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g,
@@ -352,6 +376,17 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             uint32_t ov[32];
             tmem_ld32(tmem + lane_base + kColO + 32 * grp, ov);
             tmem_wait_ld();
+            if (kFused) {
+                // Norm(o_i): sum of squares of this thread's 32 columns, the other 32 from the
+                // thread of warp (warp ^ 4) that holds the same row
+                float ss = 0.0f;
+#pragma unroll
+                for (int c = 0; c < 32; ++c) ss = fmaf(__uint_as_float(ov[c]), __uint_as_float(ov[c]), ss);
+                sm.ssq[grp][i] = ss;
+                asm volatile("bar.sync %0, 64;" ::"r"(1 + qd) : "memory");
+                ss += sm.ssq[1 - grp][i];
+                f *= rsqrtf(f * f * ss * (1.0f / kD) + p.norm_eps);
+            }
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t w[4];
@@ -394,6 +429,18 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 #pragma unroll
             for (int rr = 0; rr < 16; ++rr) {
                 uint32_t g2 = *reinterpret_cast<const uint32_t*>(sm.g + row_off(rr));
+                if (kFused) {
+                    // u = Sigmoid(-g~) = 1 - lambda, written back in place; lambda = 1 - u
+                    const float e0 = ex2(-1.4426950408889634f * fminf(fmaxf(bf16_lo(g2), -80.0f), 80.0f));
+                    const float e1 = ex2(-1.4426950408889634f * fminf(fmaxf(bf16_hi(g2), -80.0f), 80.0f));
+                    const uint32_t u2 = pack_bf16(e0 * rcp_approx(1.0f + e0), e1 * rcp_approx(1.0f + e1));
+                    *reinterpret_cast<uint32_t*>(sm.g + row_off(rr)) = u2;
+                    if ((dec >> rr) & 1u) {
+                        p0 *= 1.0f - bf16_lo(u2);
+                        p1 *= 1.0f - bf16_hi(u2);
+                    }
+                    continue;
+                }
                 g2 = ((dec >> rr) & 1u) ? g2 : 0x3f803f80u;
                 p0 *= bf16_lo(g2);
                 p1 *= bf16_hi(g2);
@@ -411,6 +458,18 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             const int Lc = min(kC, p.T - n * kC);
             // the gate pair of row rr of this warp, or (1, 1) where the step does not decay
             auto gate_or_one = [&](uint32_t g2, int rr) { return ((dec16 >> rr) & 1u) ? g2 : 0x3f803f80u; };
+            // the decay pair of row rr of this warp in fp32 (fused form: the tile holds u = 1 - lambda)
+            auto decay_pair = [&](uint32_t g2, int rr, float& l0, float& l1) {
+                if (kFused) {
+                    const bool dec = (dec16 >> rr) & 1u;
+                    l0 = dec ? 1.0f - bf16_lo(g2) : 1.0f;
+                    l1 = dec ? 1.0f - bf16_hi(g2) : 1.0f;
+                } else {
+                    const uint32_t gx = gate_or_one(g2, rr);
+                    l0 = bf16_lo(gx);
+                    l1 = bf16_hi(gx);
+                }
+            };
             if (!(ok = mbar_wait(&sm.bar.scan, n & 1, limit, abort_flag, p.status))) break;
 
             // ---- this warp's place in the chunk, the chunk's total, the range check ----------------
@@ -464,10 +523,19 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                 }
 #pragma unroll
                 for (int x = 0; x < 8; ++x) {
-                    const uint32_t gx = gate_or_one(g2[x], r8 + x);
-                    f0 *= bf16_lo(gx);
-                    f1 *= bf16_hi(gx);
-                    *reinterpret_cast<uint32_t*>(sm.qt + row_off(r8 + x)) = mul_bf16x2(q2[x], pack_bf16(f0, f1));
+                    float l0, l1;
+                    decay_pair(g2[x], r8 + x, l0, l1);
+                    f0 *= l0;
+                    f1 *= l1;
+                    if (kFused) {
+                        // q = SiLU(q~) = q~ (1 + tanh(q~ / 2)) / 2, scaled in the same step
+                        const float x0 = bf16_lo(q2[x]), x1 = bf16_hi(q2[x]);
+                        *reinterpret_cast<uint32_t*>(sm.qt + row_off(r8 + x)) =
+                            pack_bf16(0.5f * x0 * (1.0f + tanh_approx(0.5f * x0)) * f0,
+                                      0.5f * x1 * (1.0f + tanh_approx(0.5f * x1)) * f1);
+                    } else {
+                        *reinterpret_cast<uint32_t*>(sm.qt + row_off(r8 + x)) = mul_bf16x2(q2[x], pack_bf16(f0, f1));
+                    }
                 }
             }
             if (!p.tied) {
@@ -482,9 +550,10 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 #pragma unroll
                     for (int x = 7; x >= 0; --x) {
                         *reinterpret_cast<uint32_t*>(sm.kt + row_off(r8 + x)) = mul_bf16x2(k2[x], pack_bf16(t0, t1));
-                        const uint32_t gx = gate_or_one(g2[x], r8 + x);
-                        t0 *= bf16_lo(gx);
-                        t1 *= bf16_hi(gx);
+                        float l0, l1;
+                        decay_pair(g2[x], r8 + x, l0, l1);
+                        t0 *= l0;
+                        t1 *= l1;
                     }
                 }
             } else {
@@ -497,15 +566,21 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 #pragma unroll
                     for (int x = 7; x >= 0; --x) {
                         const float one = 16 * warp + r8 + x < Lc ? 1.0f : 0.0f;
-                        *reinterpret_cast<uint32_t*>(sm.kt + row_off(r8 + x)) =
-                            pack_bf16((one - bf16_lo(g2[x])) * t0, (one - bf16_hi(g2[x])) * t1);
-                        const uint32_t gx = gate_or_one(g2[x], r8 + x);
-                        t0 *= bf16_lo(gx);
-                        t1 *= bf16_hi(gx);
+                        if (kFused)     // the tile holds u = 1 - lambda: the tied key itself
+                            *reinterpret_cast<uint32_t*>(sm.kt + row_off(r8 + x)) =
+                                pack_bf16(one * bf16_lo(g2[x]) * t0, one * bf16_hi(g2[x]) * t1);
+                        else
+                            *reinterpret_cast<uint32_t*>(sm.kt + row_off(r8 + x)) =
+                                pack_bf16((one - bf16_lo(g2[x])) * t0, (one - bf16_hi(g2[x])) * t1);
+                        float l0, l1;
+                        decay_pair(g2[x], r8 + x, l0, l1);
+                        t0 *= l0;
+                        t1 *= l1;
                     }
                 }
             }
             write_state_bf16(m_a, m_b);
+            if (kFused) fence_proxy_async();      // the gate tile was rewritten in place: order that before its refill
             mbar_arrive(&sm.bar.in_free);
             fence_proxy_async();
             tc_fence_before();
@@ -612,10 +687,12 @@ cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, int* 
     p.state_in = a.state_in; p.state_out = a.state_out;
     p.redo = redo;
     p.status = a.status; p.wait_limit = a.wait_limit;
+    p.norm_eps = a.norm_eps;
     const size_t smem = sizeof(Smem) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(prefill_gated_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    auto* kernel = a.fused ? prefill_gated_tc_kernel<true> : prefill_gated_tc_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    prefill_gated_tc_kernel<<<(unsigned)(a.B * a.H), kThreads, smem, st>>>(mq, mk, mv, mg, mo, p);
+    kernel<<<(unsigned)(a.B * a.H), kThreads, smem, st>>>(mq, mk, mv, mg, mo, p);
     return cudaGetLastError();
 }
 

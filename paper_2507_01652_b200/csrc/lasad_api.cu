@@ -86,6 +86,7 @@ int reserve_redo(lasad_ctx* ctx, int64_t units)
     if (e == cudaSuccess) e = cudaDeviceSynchronize();   // an earlier launch may still use the old array
     int* nr = nullptr;
     if (e == cudaSuccess) e = cudaMalloc(&nr, (size_t)units * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(nr, 0, (size_t)units * sizeof(int));   // the kernels keep it zero between launches
     if (e == cudaSuccess) {
         if (ctx->d_redo) cudaFree(ctx->d_redo);
         ctx->d_redo = nr;
@@ -458,7 +459,12 @@ int forward_gated(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
     // scaling, and the CUDA-core kernel behind it computes exactly those (none, as a rule).
     rc = reserve_redo(ctx, (int64_t)p->B * p->H);
     if (rc != LASAD_OK) return rc;
-    cudaError_t e = lasad::launch_prefill_gated_tc(a, gate, ctx->d_redo, st);
+    // which tensor-core kernel: the balanced one (option 5, and the default where the plain prefill
+    // would take its counterpart) or the CTA-per-chain one (option 2 and the other defaults)
+    bool pair = ctx->opt_prefill_impl == 5;
+    if (ctx->opt_prefill_impl == 0) pair = auto_prefill_impl(ctx, p, p->B, true) == 5;
+    cudaError_t e = pair ? lasad::launch_prefill_gated_pair(a, gate, ctx->d_redo, ctx->d_pair, ctx->sm_count, st)
+                         : lasad::launch_prefill_gated_tc(a, gate, ctx->d_redo, st);
     if (e == cudaSuccess) {
         ctx->launches += 1;
         e = lasad::launch_prefill_gated(a, gate, p->dk, bf16, ctx->d_redo, st);

@@ -88,9 +88,15 @@ cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool d
 // null (key tied to the gate, k = 1 - lambda); a.decay is unused.
 cudaError_t launch_decode_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, bool decay_on, int tpu,
                                 cudaStream_t st);
-// `only` (device, [B*H], or null): compute just the chains whose entry is non-zero.
-cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, const int* only,
+// `only` (device, [B*H], or null): compute just the chains whose entry is non-zero, and put those
+// entries back to zero.
+cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, int* only,
                                  cudaStream_t st);
+// Balanced tensor-core form of the gated prefill (one CTA per SM, two chunk pipelines on one chain;
+// bf16, dk = dv = 64).  redo ([B*H], zero on entry): set to 1 for every chain given up; the caller
+// launches launch_prefill_gated(..., only = redo, ...) behind it.  scratch as for launch_prefill_pair.
+cudaError_t launch_prefill_gated_pair(const KernelArgs& a, const void* gate, int* redo, void* scratch, int sms,
+                                      cudaStream_t st);
 // Tensor-core form of the gated prefill (bf16, dk = dv = 64).  It writes redo[chain] = 1 for every
 // chain it gave up (decay too strong for its scaling) and 0 for the others; the caller launches
 // launch_prefill_gated(..., only = redo, ...) behind it.

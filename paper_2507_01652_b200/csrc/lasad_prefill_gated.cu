@@ -22,7 +22,7 @@ constexpr int kGC = 16;          // chunk length
 constexpr float kMinLog2 = -150.0f;
 
 template <typename T, int D>
-__global__ void __launch_bounds__(256) prefill_gated_kernel(KernelArgs a, const void* gate_v, const int* only)
+__global__ void __launch_bounds__(256) prefill_gated_kernel(KernelArgs a, const void* gate_v, int* only)
 {
     // behind the tensor-core kernel: only the chains it gave up are computed here
     if (only && only[blockIdx.x] == 0) return;
@@ -152,10 +152,11 @@ __global__ void __launch_bounds__(256) prefill_gated_kernel(KernelArgs a, const 
     __syncthreads();
     if (a.state_out)
         for (int x = tid; x < D * D; x += 256) a.state_out[unit + x] = Ss[(x / D) * LD + (x % D)];
+    if (only && tid == 0) only[blockIdx.x] = 0;      // the mark has been served
 }
 
 template <typename T, int D>
-cudaError_t launch_gated_t(const KernelArgs& a, const void* gate, const int* only, cudaStream_t st)
+cudaError_t launch_gated_t(const KernelArgs& a, const void* gate, int* only, cudaStream_t st)
 {
     const size_t smem = sizeof(float) * D * (D + 1);
     prefill_gated_kernel<T, D><<<(unsigned)(a.B * a.H), 256, smem, st>>>(a, gate, only);
@@ -164,7 +165,7 @@ cudaError_t launch_gated_t(const KernelArgs& a, const void* gate, const int* onl
 
 }  // namespace
 
-cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, const int* only,
+cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, int* only,
                                  cudaStream_t st)
 {
     if (dk == 64)

@@ -52,13 +52,13 @@ def test_gated_prefill_matches_oracle(ctx, dtype, d, T, w, P):
 
 @pytest.mark.parametrize("T,w,P", [(1, 4, 0), (100, 7, 0), (128, 16, 0), (257, 16, 1), (700, 24, 0)])
 def test_gated_prefill_both_implementations(ctx, T, w, P):
-    """bf16, d = 64: the tensor-core kernel (default) and the CUDA-core kernel (option 1) against the
-    oracle on the same inputs."""
+    """bf16, d = 64: the default, the CUDA-core kernel (option 1), the CTA-per-chain tensor-core kernel
+    (option 2) and the balanced tensor-core kernel (option 5) against the oracle on the same inputs."""
     B, H, d = 3, 5, 64
     q, k, v, lam = _inputs(900 + T, B, T, H, d, torch.bfloat16)
     s_in = torch.randn(B, H, d, d, generator=torch.Generator().manual_seed(T))
     o_ref, s_ref = oracle(q, k, v, lam, w, P, 3, 0.25, s_in)
-    for impl in (0, 1):
+    for impl in (0, 1, 2, 5):
         ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, impl)
         try:
             o, s = ctx.lasad_forward_gated(*_dev(q, k, v, lam), w, prefix_len=P, t0=3, scale=0.25, state_in=s_in.cuda())
@@ -70,8 +70,9 @@ def test_gated_prefill_both_implementations(ctx, T, w, P):
         assert rel_err(s, s_ref) <= TOL[torch.bfloat16], impl
 
 
+@pytest.mark.parametrize("impl", [2, 5])
 @pytest.mark.parametrize("level,tied", [(0.35, False), (0.05, False), (0.003, True), (1e-5, False), (0.0, False)])
-def test_gated_tensor_core_path_strong_decay(ctx, level, tied):
+def test_gated_tensor_core_path_strong_decay(ctx, impl, level, tied):
     """Gates so small that a 128-token chunk cannot be scaled around one reference point: the
     tensor-core kernel cuts such chunks into segments of 64, 32, 16 or single tokens.  The middle
     chunk of three is the strong one, with exact zeros sprinkled in; the others are ordinary."""
@@ -83,8 +84,12 @@ def test_gated_tensor_core_path_strong_decay(ctx, level, tied):
     lam[:, 128:256] = strong.to(torch.bfloat16)
     k_used = torch.from_numpy(1.0 - to64(lam)) if tied else k
     o_ref, s_ref = oracle(q, k_used, v, lam, w)
-    o, s = ctx.lasad_forward_gated(q.cuda(), None if tied else k.cuda(), v.cuda(), lam.cuda(), w)
-    torch.cuda.synchronize()
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, impl)
+    try:
+        o, s = ctx.lasad_forward_gated(q.cuda(), None if tied else k.cuda(), v.cuda(), lam.cuda(), w)
+        torch.cuda.synchronize()
+    finally:
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
     assert ctx.device_status() == 0
     assert torch.isfinite(o.float()).all() and torch.isfinite(s).all()
     assert rel_err(o, o_ref) <= TOL[torch.bfloat16]
@@ -167,11 +172,13 @@ def test_gated_state_handoff(ctx):
         assert rel_err(s2, s_ref) <= TOL[torch.bfloat16]
 
 
-def test_gated_prefill_recorded_into_a_cuda_graph_and_replayed(ctx):
+@pytest.mark.parametrize("impl,H", [(2, 3), (5, 3), (5, 80)])
+def test_gated_prefill_recorded_into_a_cuda_graph_and_replayed(ctx, impl, H):
     """Both launches of the gated prefill (tensor-core kernel, CUDA-core kernel for flagged chains)
     captured into a CUDA graph and replayed on new inputs; the second replay has a strong-decay
-    stretch, so the replayed CUDA-core launch has chains to redo."""
-    B, T, H, d, w = 2, 300, 3, 64, 10
+    stretch, so the replayed CUDA-core launch has chains to redo (and, with the balanced kernel and
+    160 chains, chains that were given up on one CTA and finished on another)."""
+    B, T, d, w = 2, (1100 if H > 3 else 300), 64, 10
     dq, dk, dv, dl = [torch.empty(B, T, H, d, dtype=torch.bfloat16, device="cuda") for _ in range(4)]
     o = torch.empty_like(dv)
     s = torch.empty(B, H, d, d, device="cuda")
@@ -180,11 +187,15 @@ def test_gated_prefill_recorded_into_a_cuda_graph_and_replayed(ctx):
         dst.copy_(src)
     stream = torch.cuda.Stream()
     graph = torch.cuda.CUDAGraph()
-    with torch.cuda.stream(stream):
-        ctx.lasad_forward_gated(dq, dk, dv, dl, w, o=o, state_out=s)     # warm-up outside the capture
-        torch.cuda.synchronize()
-        with torch.cuda.graph(graph, stream=stream):
-            ctx.lasad_forward_gated(dq, dk, dv, dl, w, o=o, state_out=s)
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, impl)
+    try:
+        with torch.cuda.stream(stream):
+            ctx.lasad_forward_gated(dq, dk, dv, dl, w, o=o, state_out=s)     # warm-up outside the capture
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph, stream=stream):
+                ctx.lasad_forward_gated(dq, dk, dv, dl, w, o=o, state_out=s)
+    finally:
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
     for rep in range(3):
         q, k, v, lam = _inputs(32 + rep, B, T, H, d, torch.bfloat16)
         if rep == 1:
@@ -197,3 +208,33 @@ def test_gated_prefill_recorded_into_a_cuda_graph_and_replayed(ctx):
         o_ref, s_ref = oracle(q, k, v, lam, w)
         assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
         assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
+
+
+@pytest.mark.parametrize("B,H,T,tied", [(1, 160, 1100, False), (2, 163, 700, True), (1, 151, 260, False), (1, 149, 2500, True)])
+def test_gated_balanced_prefill_left_over_chains(ctx, B, H, T, tied):
+    """The balanced gated kernel (option 5) with more chains than SMs: left-over chains cut into
+    pieces whose state crosses CTAs; some heads with a decay too strong for the kernel's scaling in
+    the second half of the sequence only, so that a chain is given up on one CTA after an earlier
+    piece of it was taken normally, and the mark has to travel with the state; an incoming state,
+    state_out aliasing state_in; twice in a row."""
+    d, w = 64, 13
+    q, k, v, lam = _inputs(2100 + H + T, B, T, H, d, torch.bfloat16)
+    lam[:, T // 2:, 0] = 0.01
+    lam[:, :, H - 1] = 0.02
+    lam[:, T // 3:, H // 2] = 0.0
+    k_used = torch.from_numpy(1.0 - to64(lam)) if tied else k
+    s_in = torch.randn(B, H, d, d, generator=torch.Generator().manual_seed(T)) * 0.3
+    o_ref, s_ref = oracle(q, k_used, v, lam, w, 1, 5, 0.5, s_in)
+    dq, dk, dv, dl = _dev(q, k, v, lam)
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 5)
+    try:
+        for rep in range(2):
+            ds = s_in.cuda()
+            o, s = ctx.lasad_forward_gated(dq, None if tied else dk, dv, dl, w, prefix_len=1, t0=5, scale=0.5,
+                                           state_in=ds, state_out=ds)
+            torch.cuda.synchronize()
+            assert ctx.device_status() == 0
+            assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+            assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
+    finally:
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)

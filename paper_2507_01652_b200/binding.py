@@ -114,7 +114,50 @@ def _dtype_code(t: torch.Tensor) -> int:
 
 
 def _ptr(t):
-    return None if t is None else ctypes.c_void_p(t.data_ptr())
+    # (an int is accepted where the prototype says c_void_p; None is a null pointer)
+    return None if t is None else t.data_ptr()
+
+
+try:
+    _raw_stream = torch._C._cuda_getCurrentRawStream     # the current stream's handle without a Stream object
+except AttributeError:       # pragma: no cover - older torch
+    _raw_stream = None
+
+
+def _stream(device, stream):
+    if stream is not None:
+        return stream
+    if _raw_stream is not None:
+        return _raw_stream(device.index if device.index is not None else torch.cuda.current_device())
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+_params_cache = {}
+
+
+def _params(kind, q, k, v, o, grid_w, prefix_len, t0, scale):
+    """The call's ``lasad_params``.  The struct is cached per (shape, strides, dtype) -- building
+    its ctypes arrays costs more than the rest of the marshalling -- and only its scalars are
+    refreshed.  kind: "prefill" ([B,T,H,d] tensors) or "decode" ([B,H,d])."""
+    key = (kind, q.shape, q.stride(), k.stride(), v.stride(), o.stride(), v.shape[-1], q.dtype)
+    p = _params_cache.get(key)
+    if p is None:
+        if kind == "prefill":
+            B, T, H, dk = q.shape
+            p = LasadParams(B, T, H, dk, v.shape[3], 0, 0, _dtype_code(q), 0, 1.0, 0,
+                            _strides3(q), _strides3(k), _strides3(v), _strides3(o))
+        else:
+            B, H, dk = q.shape
+            p = LasadParams(B, 1, H, dk, v.shape[2], 0, 0, _dtype_code(q), 0, 1.0, 0,
+                            _strides_decode(q), _strides_decode(k), _strides_decode(v), _strides_decode(o))
+        if len(_params_cache) > 256:
+            _params_cache.clear()
+        _params_cache[key] = p
+    p.grid_w = grid_w
+    p.prefix_len = prefix_len
+    p.t0 = t0
+    p.scale = scale
+    return p
 
 
 def _check_cuda(*ts):
@@ -199,12 +242,10 @@ class Lasad:
             o = torch.empty((B, T, H, dv), dtype=q.dtype, device=q.device)
         if state_out is None and want_state:
             state_out = torch.empty((B, H, dk, dv), dtype=torch.float32, device=q.device)
-        p = LasadParams(B, T, H, dk, dv, grid_w, prefix_len, _dtype_code(q), t0, scale, 0,
-                        _strides3(q), _strides3(k), _strides3(v), _strides3(o))
-        st = torch.cuda.current_stream(q.device).cuda_stream if stream is None else stream
+        p = _params("prefill", q, k, v, o, grid_w, prefix_len, t0, scale)
         rc = self._lib.lasad_forward(self._h, ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v),
                                      _ptr(decay), _ptr(state_in), _ptr(o), _ptr(state_out),
-                                     ctypes.c_void_p(st))
+                                     _stream(q.device, stream))
         if rc != LASAD_OK:
             self._raise(rc, "lasad_forward")
         return o, state_out
@@ -240,11 +281,9 @@ class Lasad:
             o = torch.empty((B, H, dv), dtype=q.dtype, device=q.device)
         if state.dtype != torch.float32 or not state.is_contiguous() or tuple(state.shape) != (B, H, dk, dv):
             raise ValueError("state must be contiguous float32 [B,H,dk,dv]")
-        p = LasadParams(B, 1, H, dk, dv, grid_w, prefix_len, _dtype_code(q), t, scale, 0,
-                        _strides_decode(q), _strides_decode(k), _strides_decode(v), _strides_decode(o))
-        st = torch.cuda.current_stream(q.device).cuda_stream if stream is None else stream
+        p = _params("decode", q, k, v, o, grid_w, prefix_len, t, scale)
         rc = self._lib.lasad_decode_step(self._h, ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v),
-                                         _ptr(decay), _ptr(state), _ptr(o), ctypes.c_void_p(st))
+                                         _ptr(decay), _ptr(state), _ptr(o), _stream(q.device, stream))
         if rc != LASAD_OK:
             self._raise(rc, "lasad_decode_step")
         return o

@@ -183,6 +183,14 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         sm.tag = ((unsigned)*reinterpret_cast<volatile int*>(p.work + 2) & 0x3fffffffu) + 1u;   // never 0, the slots' initial content
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (warp == 9 && lane == 0) {
+        // the descriptors' first use then finds them in the descriptor cache
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_q)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_g)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_o)) : "memory");
+    }
     if (threadIdx.x >> 5 == 8) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
                      "r"(2 * kPipeTmemCols)
@@ -415,6 +423,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             if (g >= nx.u.g1) {
                 nx.u = unit_of(plan, g);
                 nx.n = nx.u.n0 + g - nx.u.g0;
+                if (nx.u.recv >= 0) slot_prefetch(p.slots + (size_t)nx.u.recv * kSlotBytes, tid);
                 nx.gp = grid_pos_init(p.grid_w, p.prefix_len, p.t0 + (long long)nx.n * kC, lane);
                 nx.cs = 0;
             } else {
@@ -779,7 +788,8 @@ cudaError_t launch_prefill_gated_pair(const KernelArgs& a, const void* gate, int
     p.norm_eps = a.norm_eps;
     const size_t smem = sizeof(Smem) + 1024;
     auto* kernel = a.fused ? prefill_gated_pair_kernel<true> : prefill_gated_pair_kernel<false>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static bool smem_ok[2][64];      // one set of flags per kernel variant
+    cudaError_t e = allow_dynamic_smem(kernel, smem, smem_ok[a.fused ? 1 : 0]);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(chains < sms ? chains : sms);
     kernel<<<grid, kPairThreads, smem, st>>>(mq, mk, mv, mg, mo, p);

@@ -690,7 +690,8 @@ cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, int* 
     p.norm_eps = a.norm_eps;
     const size_t smem = sizeof(Smem) + 1024;
     auto* kernel = a.fused ? prefill_gated_tc_kernel<true> : prefill_gated_tc_kernel<false>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static bool smem_ok[2][64];      // one set of flags per kernel variant
+    cudaError_t e = allow_dynamic_smem(kernel, smem, smem_ok[a.fused ? 1 : 0]);
     if (e != cudaSuccess) return e;
     kernel<<<(unsigned)(a.B * a.H), kThreads, smem, st>>>(mq, mk, mv, mg, mo, p);
     return cudaGetLastError();

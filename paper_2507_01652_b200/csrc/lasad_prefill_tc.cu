@@ -995,9 +995,9 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, int sms, cudaStream_t st)
     p.n_segs = 1; p.seg_chunks = (a.T + kC - 1) / kC; p.seg_state = nullptr;
     p.status = a.status; p.wait_limit = a.wait_limit;
     const size_t smem = sizeof(Smem) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static bool smem_ok_1[64], smem_ok_2[64];
+    cudaError_t e = allow_dynamic_smem(prefill_tc_kernel<false>, smem, smem_ok_1);
+    if (e == cudaSuccess) e = allow_dynamic_smem(prefill_tc_kernel<true>, smem, smem_ok_2);
     if (e != cudaSuccess) return e;
     // Two CTAs fit on an SM; with more chains than that, the CTAs stay and draw further chains
     // from the work counter, so a chain's first loads overlap the previous chain's last chunk.
@@ -1012,7 +1012,8 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, int sms, cudaStream_t st)
             p.n_segs = segs;
             p.seg_state = a.seg_state;
             const size_t ssmem = sizeof(StateSmem) + 1024;
-            e = cudaFuncSetAttribute(prefill_seg_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssmem);
+            static bool smem_ok_3[64];
+            e = allow_dynamic_smem(prefill_seg_state_kernel, ssmem, smem_ok_3);
             if (e != cudaSuccess) return e;
             SegSteps steps;
             for (int sg = 0; sg + 1 < segs; ++sg) {

@@ -145,6 +145,13 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         sm.tag = ((unsigned)*reinterpret_cast<volatile int*>(p.work + 2) & 0x3fffffffu) + 1u;   // never 0, the slots' initial content
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (warp == 9 && lane == 0) {
+        // the descriptors' first use then finds them in the descriptor cache
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_q)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_o)) : "memory");
+    }
     if (threadIdx.x >> 5 == 8) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
                      "r"(2 * kPipeTmemCols)
@@ -348,6 +355,8 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (g >= u.g1) {
                 u = unit_of(plan, g);
                 n = u.n0 + g - u.g0;
+                if (u.recv >= (int)gridDim.x) park_prefetch(p.slots + (size_t)u.recv * kSlotBytes, tid);
+                else if (u.recv >= 0) slot_prefetch(p.slots + (size_t)u.recv * kSlotBytes, tid);
                 const int h = u.chain % p.H;
                 gamma = p.decay[h];
                 fast = gamma >= kFastPathMinDecay;
@@ -483,7 +492,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                 } else {
                     // the chain was cut here: its state comes from where the part before it was done
-                    if (!(ok = slot_receive(p.slots + (size_t)u.recv * kSlotBytes, tid, st, sm.tag, limit, abort_flag, p.status)))
+                    if (u.recv >= (int)gridDim.x)
+                        park_receive(p.slots + (size_t)u.recv * kSlotBytes, tid, st);
+                    else if (!(ok = slot_receive(p.slots + (size_t)u.recv * kSlotBytes, tid, st, sm.tag, limit, abort_flag, p.status)))
                         break;
                 }
             } else {
@@ -520,7 +531,8 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                 } else {
                     // the chain is cut here: the state goes to where its next part will be done
-                    slot_send(p.slots + (size_t)u.send * kSlotBytes, tid, st, sm.tag);
+                    if (u.send >= (int)gridDim.x) park_send(p.slots + (size_t)u.send * kSlotBytes, tid, st);
+                    else slot_send(p.slots + (size_t)u.send * kSlotBytes, tid, st, sm.tag);
                 }
             } else {
 #pragma unroll
@@ -597,7 +609,8 @@ cudaError_t launch_prefill_pair(const KernelArgs& a, void* scratch, int sms, cud
     p.chains = (int)chains;
     p.status = a.status; p.wait_limit = a.wait_limit;
     const size_t smem = sizeof(Smem) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(prefill_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static bool smem_ok_1[64];
+    cudaError_t e = allow_dynamic_smem(prefill_pair_kernel, smem, smem_ok_1);
     if (e != cudaSuccess) return e;
     // Fewer chains than SMs: one chain per CTA, nothing is cut.  Otherwise one CTA per SM.
     const unsigned grid = (unsigned)(chains < sms ? chains : sms);

@@ -781,7 +781,8 @@ cudaError_t launch_prefill_stream(const KernelArgs& a, const TcRelay& r, cudaStr
     p.status = a.status; p.wait_limit = a.wait_limit;
     if (r.max_ctas <= 0 || (p.n_chunks > 1 && !p.relay)) return cudaErrorInvalidValue;
     const size_t smem = sizeof(Smem) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(prefill_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static bool smem_ok_1[64];
+    cudaError_t e = allow_dynamic_smem(prefill_stream_kernel, smem, smem_ok_1);
     if (e != cudaSuccess) return e;
     const int grid = p.n_tasks < r.max_ctas ? p.n_tasks : r.max_ctas;
     prefill_stream_kernel<<<(unsigned)grid, kThreads, smem, st>>>(mq, mk, mv, mo, p);

@@ -32,7 +32,7 @@ struct Plan {
     int stride;       // chains per round (= CTAs)
     Unit special[kMaxSpecial];
 };
-constexpr int kHandoffMargin = 2;   // chunks a CTA stays on its own chain beyond the nominal start of its piece, per hop
+constexpr int kHandoffMargin = 3;   // chunks a CTA stays on its own chain beyond the nominal start of its piece, per hop
 constexpr int kMinPiece = 4;        // shortest piece (chunks) a left-over chain is cut into
 
 __device__ __forceinline__ Unit unit_of(const Plan& pl, int g)
@@ -84,6 +84,16 @@ __device__ __forceinline__ void slot_send(unsigned char* slot, int t, const floa
     for (int k = 0; k < 8; ++k)
         st_cg_v2u64(slot + ((size_t)k * kEThreads + t) * 16, hi | __float_as_uint(st[2 * k]), hi | __float_as_uint(st[2 * k + 1]));
 }
+// Asks for this thread's part of a slot to be brought into L2.  A slot that was written tens of
+// microseconds ago has been pushed out to DRAM by the kernel's own traffic, and a DRAM read under
+// that load takes several microseconds: issued one chunk ahead, it is over by the time the state
+// is wanted.
+__device__ __forceinline__ void slot_prefetch(const unsigned char* slot, int t)
+{
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(slot + ((size_t)k * kEThreads + t) * 16));
+}
 // Bounded: polls until all sixteen packets carry `tag`; `flag` (if given) receives the sender's flag.
 __device__ __forceinline__ bool slot_receive(const unsigned char* slot, int t, float (&st)[16], unsigned tag, unsigned limit,
                                              volatile int* abort_flag, int* status, bool* flag = nullptr)
@@ -111,6 +121,35 @@ __device__ __forceinline__ bool slot_receive(const unsigned char* slot, int t, f
     *abort_flag = 1;
     atomicExch(status, 1);
     return false;
+}
+
+// A CTA's own chain waits in its own slot while the CTA works on a piece.  Nobody else touches
+// that slot, so it needs no tags: plain fp32 (the first 16 KiB of the slot, thread t's values
+// 4k .. 4k+3 at (k * 256 + t) * 16), ordered between writer and reader by the mbarriers that the
+// chunks in between pass through.  Its read is asked for one chunk ahead, into L1: a load issued
+// when the state is wanted would queue behind the SM's bulk copies for microseconds.
+__device__ __forceinline__ void park_send(unsigned char* slot, int t, const float (&st)[16])
+{
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        *reinterpret_cast<float4*>(slot + ((size_t)k * kEThreads + t) * 16) = make_float4(st[4 * k], st[4 * k + 1], st[4 * k + 2], st[4 * k + 3]);
+}
+__device__ __forceinline__ void park_prefetch(const unsigned char* slot, int t)
+{
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        asm volatile("prefetch.global.L1 [%0];" ::"l"(slot + ((size_t)k * kEThreads + t) * 16));
+}
+__device__ __forceinline__ void park_receive(const unsigned char* slot, int t, float (&st)[16])
+{
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        float4 x;
+        asm volatile("ld.global.ca.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w)
+                     : "l"(slot + ((size_t)k * kEThreads + t) * 16));
+        st[4 * k] = x.x; st[4 * k + 1] = x.y; st[4 * k + 2] = x.z; st[4 * k + 3] = x.w;
+    }
 }
 
 // Fills `plan` (shared memory) for the CTA with start-order number `cta`; every thread of the CTA

@@ -3,6 +3,7 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <stdint.h>
 
 namespace lasad {
 namespace tcx {
@@ -27,7 +28,7 @@ inline EncodeTiledFn get_encode_fn()
 
 // [B,T,H,64] bf16 with element strides (b,t,h) -> 4-D map (d, h, t, b); box = 128 tokens of one
 // head, rows of 128 bytes with the 128-byte swizzle; rows past T read as zeros and are not stored.
-inline bool encode_chunk_map(CUtensorMap* map, const void* base, int B, int T, int H, const long long* strides)
+inline bool encode_chunk_map_uncached(CUtensorMap* map, const void* base, int B, int T, int H, const long long* strides)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
@@ -39,6 +40,49 @@ inline bool encode_chunk_map(CUtensorMap* map, const void* base, int B, int T, i
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, gstr, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The same through a small per-thread cache: a descriptor depends on nothing but the arguments
+// below, and callers come back with the same tensors call after call (a layer's buffers, the
+// slots of a host pipeline), so the driver call is made once per tensor, not once per launch.
+inline bool encode_chunk_map(CUtensorMap* map, const void* base, int B, int T, int H, const long long* strides)
+{
+    struct Entry {
+        const void* base;
+        int B, T, H;
+        long long s[3];
+        bool valid;
+        CUtensorMap map;
+    };
+    constexpr int kEntries = 32;
+    thread_local Entry cache[kEntries];
+    const unsigned long long x = (unsigned long long)reinterpret_cast<uintptr_t>(base);
+    Entry& e = cache[((x >> 8) ^ (x >> 20) ^ (unsigned)T) % kEntries];
+    if (e.valid && e.base == base && e.B == B && e.T == T && e.H == H && e.s[0] == strides[0] && e.s[1] == strides[1] &&
+        e.s[2] == strides[2]) {
+        *map = e.map;
+        return true;
+    }
+    if (!encode_chunk_map_uncached(map, base, B, T, H, strides)) return false;
+    e.base = base; e.B = B; e.T = T; e.H = H;
+    e.s[0] = strides[0]; e.s[1] = strides[1]; e.s[2] = strides[2];
+    e.map = *map;
+    e.valid = true;
+    return true;
+}
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per device and kernel instead of once per
+// launch.  `done` is the call site's own flag array.
+template <typename Kernel>
+inline cudaError_t allow_dynamic_smem(Kernel kernel, size_t bytes, bool (&done)[64])
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+    return e;
 }
 
 }  // namespace tcx

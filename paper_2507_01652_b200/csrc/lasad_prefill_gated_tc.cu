@@ -51,6 +51,7 @@
 // issues the MMAs, warp 9 the TMA loads and stores.  All waits are bounded: a wait that runs out
 // raises a status word the host can read and the CTA leaves through the normal exit.
 #include "lasad_common.cuh"
+#include "lasad_tc_chunk.cuh"
 #include "lasad_tc_ptx.cuh"
 #include "lasad_tc_tma.cuh"
 
@@ -59,16 +60,8 @@ namespace {
 
 using namespace tcx;
 
-constexpr int kC = 128;                    // chunk length (tokens) = MMA M
-constexpr int kD = 64;                     // d_k = d_v
-constexpr int kEThreads = 256;             // element-wise warps 0-7
-constexpr int kThreads = kEThreads + 64;   // + the MMA warp and the TMA warp
-constexpr int kTileBytes = kC * kD * 2;    // 16 KB: one [128 x 64] bf16 tile, 128 B rows
+constexpr int kThreads = kEThreads + 64;   // element-wise warps, the MMA warp and the TMA warp
 constexpr int kTmemCols = 256;
-constexpr uint32_t kColS = 0;      // S (fp32, 128 columns); A (bf16 pairs) aliases columns 0..31 and 64..95
-constexpr uint32_t kColO = 128;    // O accumulator, 64 columns
-constexpr uint32_t kColDS = 192;   // dS accumulator (M = 64 layout), 64 columns
-constexpr unsigned kTeardownLimit = 1u << 26;
 constexpr float kSafeRange = 200.0f;   // largest |sum of log2 decays| one pass may span
 
 struct __align__(8) Barriers {

@@ -36,6 +36,7 @@
 // bounded: a wait that runs out raises a status word the host can read and the CTA leaves
 // through the normal exit (copies in flight are waited for, TMEM is freed).
 #include "lasad_common.cuh"
+#include "lasad_tc_chunk.cuh"
 #include "lasad_tc_ptx.cuh"
 #include "lasad_tc_tma.cuh"
 
@@ -44,18 +45,9 @@ namespace {
 
 using namespace tcx;
 
-constexpr int kC = 128;                    // chunk length (tokens) = MMA M
-constexpr int kD = 64;                     // d_k = d_v
-constexpr int kEThreads = 256;             // element-wise warps 0-7
-constexpr int kThreads = kEThreads + 64;   // + the MMA warp and the TMA warp
-constexpr int kTileBytes = kC * kD * 2;    // 16 KB: one [128 x 64] bf16 tile, 128 B rows
+constexpr int kThreads = kEThreads + 64;   // element-wise warps, the MMA warp and the TMA warp
 constexpr int kStages = 2;
 constexpr int kTmemCols = 256;
-constexpr uint32_t kColS = 0;      // S (fp32, 128 columns); A/P (bf16 pairs) aliases columns 0..31 and 64..95
-constexpr uint32_t kColO = 128;    // O accumulator, 64 columns
-constexpr uint32_t kColDS = 192;   // dS accumulator (M = 64 layout), 64 columns
-constexpr unsigned kTeardownLimit = 1u << 26;
-constexpr float kFastPathMinDecay = 0.6f;
 
 struct __align__(8) Barriers {
     unsigned long long full[kStages];   // TMA loads of a stage have landed
@@ -86,15 +78,6 @@ struct Smem {
 };
 
 
-#ifdef LASAD_TC_TRACE
-// Debug builds only: per-phase clock64() stamps of CTA 0 (E-thread 0: slots 0..; MMA thread: slots 2048..).
-__device__ long long g_trace[4096];
-#define TRACE_E(slot) do { if (blockIdx.x == 0 && tid == 0) g_trace[(slot)] = clock64(); } while (0)
-#define TRACE_M(slot) do { if (blockIdx.x == 0 && lane == 0) g_trace[2048 + (slot)] = clock64(); } while (0)
-#else
-#define TRACE_E(slot) do { } while (0)
-#define TRACE_M(slot) do { } while (0)
-#endif
 
 struct TcParams {
     int B, T, H;
@@ -114,89 +97,10 @@ struct TcParams {
     unsigned wait_limit;
 };
 
-// Decay bookkeeping of one chunk, computed by every warp on its own with four ballots (one per
-// 32-token block): which steps decay, and from their popcounts n_i for the thread's own row.
-struct ChunkDecay {
-    unsigned m0, m1, m2, m3;   // bit l of m<x>: token 32 x + l of the chunk is a decaying step
-    int c0, c1, c2;            // decaying steps up to the end of block 0, 1, 2
-    int ni;                    // n of the thread's own row
-    int n_last;                // n of the chunk's last token
-    // n of chunk column j (warp-uniform j)
-    __device__ __forceinline__ int n_of(int j) const
-    {
-        const int x = j >> 5;
-        const unsigned m = x == 0 ? m0 : x == 1 ? m1 : x == 2 ? m2 : m3;
-        const int before = x == 0 ? 0 : x == 1 ? c0 : x == 2 ? c1 : c2;
-        return before + __popc(m & (0xffffffffu >> (31 - (j & 31))));
-    }
-};
-
-// Where the chunks of this call sit on the token grid, in a form that needs no division inside
-// the chunk loop: token `tok` of the chunk that starts at call offset cs absorbs the last token
-// of a grid row (a boundary step, SAD rule of Section 3.4) iff it lies on the grid
-// (cs + tok >= pre) and (phase + r[tok / 32]) is 0 or w, where r = (tok mod w) is fixed per
-// thread and phase = (grid column of the chunk's first token + 1) mod w advances by
-// (128 mod w) per chunk.
-struct GridPos {
-    int grid_w;
-    int pre;         // tokens of this call that precede the grid (class-token prefix)
-    int r[4];        // (32 x + lane) mod w
-    int step;        // 128 mod w
-    int phase;       // ((grid index of the current chunk's first token) + 1) mod w
-};
-
-__device__ __forceinline__ GridPos grid_pos_init(int grid_w, int prefix_len, long long t0, int lane)
-{
-    GridPos g;
-    g.grid_w = grid_w;
-    const long long g0 = t0 - prefix_len;   // grid index of the call's first token (may be < 0)
-    g.pre = g0 < 0 ? (int)min(-g0, (long long)0x7fffffff) : 0;
-    g.step = 0; g.phase = 0;
-#pragma unroll
-    for (int x = 0; x < 4; ++x) g.r[x] = 0;
-    if (grid_w > 0) {
-        long long ph = (g0 + 1) % grid_w;    // C remainder: may be negative inside the prefix
-        if (ph < 0) ph += grid_w;
-        g.phase = (int)ph;
-        g.step = kC % grid_w;
-#pragma unroll
-        for (int x = 0; x < 4; ++x) g.r[x] = (32 * x + lane) % grid_w;
-    }
-    return g;
-}
-
-// Decay bookkeeping of the chunk at call offset cs (L live tokens); advances g to the next chunk.
-__device__ __forceinline__ ChunkDecay chunk_decay(GridPos& g, int cs, int L, int qd, int lane)
-{
-    ChunkDecay d;
-    unsigned mk[4];
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-        const int tok = 32 * x + lane;
-        const int m = g.phase + g.r[x];
-        const bool boundary = g.grid_w > 0 && cs + tok >= g.pre && (m == 0 || m == g.grid_w);
-        mk[x] = __ballot_sync(0xffffffffu, tok < L && !boundary);
-    }
-    d.m0 = mk[0]; d.m1 = mk[1]; d.m2 = mk[2]; d.m3 = mk[3];
-    d.c0 = __popc(d.m0);
-    d.c1 = d.c0 + __popc(d.m1);
-    d.c2 = d.c1 + __popc(d.m2);
-    d.n_last = d.c2 + __popc(d.m3);
-    g.phase += g.step;
-    if (g.phase >= g.grid_w) g.phase -= g.grid_w;
-    const unsigned own = qd == 0 ? d.m0 : qd == 1 ? d.m1 : qd == 2 ? d.m2 : d.m3;
-    const int before = qd == 0 ? 0 : qd == 1 ? d.c0 : qd == 2 ? d.c1 : d.c2;
-    d.ni = before + __popc(own & (0xffffffffu >> (31 - lane)));
-    return d;
-}
-
-#ifndef LASAD_MINBLOCKS
-#define LASAD_MINBLOCKS 2
-#endif
 // kSegments: work units are segments of chains (see TcParams); false: whole chains, and none of
 // the unit arithmetic below costs anything.
 template <bool kSegments>
-__global__ void __launch_bounds__(kThreads, LASAD_MINBLOCKS)
+__global__ void __launch_bounds__(kThreads, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, TcParams p)
 {
@@ -384,7 +288,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const int s = g % kStages;
             const uint64_t dqs = s ? dq1 : dq0, dks = s ? dk1 : dk0, dvs = s ? dv1 : dv0;
             const bool fast = fast_next;
-            TRACE_M(8 * g + 0);
             if (!mbar_wait(&sm.bar.x_ready, g & 1, limit, abort_flag, p.status)) break;
             tc_fence_after();
             if (elect_one()) {
@@ -402,10 +305,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
             }
             __syncwarp();
-            TRACE_M(8 * g + 1);
             if (!mbar_wait(&sm.bar.p_ready, g & 1, limit, abort_flag, p.status)) break;
             tc_fence_after();
-            TRACE_M(8 * g + 2);
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kC / 16; ++kk)  // A/P: 8 TMEM columns per step (tokens 0..63 at columns
@@ -421,9 +322,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 mma_commit(&sm.bar.o_done[s]);
             }
             __syncwarp();
-            TRACE_M(8 * g + 3);
             more = issue_m1(g + 1);
-            TRACE_M(8 * g + 4);
         }
         // make sure nothing is still running on the tensor pipe before TMEM is freed
         if (elect_one()) {
@@ -550,10 +449,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 mbar_arrive(&sm.bar.x_ready);
                 for (int n = 0; ok && n < n_here; ++n, ++g) {
                     const int s = g % kStages;
-                    TRACE_E(8 * g + 0);
                     if (!(ok = mbar_wait(&sm.bar.s_done, g & 1, limit, abort_flag, p.status))) break;
                     tc_fence_after();
-                    TRACE_E(8 * g + 1);
                     // ---- E1: A = tril(S) -> bf16 over S's own columns.  This warp converts the
                     //      32-column blocks 2 grp and 2 grp + 1 of its rows and keeps the result inside
                     //      its own half of S's columns (block pc -> columns 64 grp + 16 (pc & 1), always
@@ -585,14 +482,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(&sm.bar.p_ready);
-                    TRACE_E(8 * g + 2);
 
                     // ---- while the O MMAs run: the state recurrence in fp32 registers ----------------
                     const float out_f = p.scale * gpow(-(cd.n_last - cd.ni));   // scale * gamma^-(N - n_i)
                     if (!(ok = mbar_wait(&sm.bar.ds_done, g & 1, limit, abort_flag, p.status))) break;
                     tc_fence_after();
                     update_state(gpow(cd.n_last));
-                    TRACE_E(8 * g + 3);
                     const bool more = n + 1 < n_here;
                     if (more) {
                         const int cs1 = (n + 1) * kC;
@@ -600,18 +495,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     } else {
                         state_leaves();
                     }
-                    TRACE_E(8 * g + 4);
 
                     // ---- E2: o_i = scale * gamma^-(N - n_i) * O'_i ------------------------------------
                     if (!(ok = mbar_wait(&sm.bar.o_done[s], (g / kStages) & 1, limit, abort_flag, p.status))) break;
                     tc_fence_after();
-                    TRACE_E(8 * g + 5);
                     stage_output(s, out_f);
                     if (more) write_state_bf16(gpow(cd.n_last));   // gamma^N(next) * S_new
                     fence_proxy_async();
                     tc_fence_before();
                     mbar_arrive(&sm.bar.st_ready[s]);
-                    TRACE_E(8 * g + 6);
 
                     // ---- V~ of the chain's next chunk, once its loads have landed.  This stage is
                     //      released (st_ready above) before the wait, so the wait never holds a buffer
@@ -960,13 +852,6 @@ prefill_seg_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
 }
 
 }  // namespace
-
-#ifdef LASAD_TC_TRACE
-extern "C" int lasad_debug_read_trace(long long* host, int n)
-{
-    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * n);
-}
-#endif
 
 bool prefill_tc_supported(int dk, int dv, bool bf16) { return bf16 && dk == kD && dv == kD; }
 

@@ -3,17 +3,21 @@
 //
 // Work decomposition.  The sequence of one (batch, head) -- a chain -- is cut into chunks of
 // C = 128 tokens.  One task = one chunk of one chain.  Tasks are numbered chunk-major
-// (id = n * X + x for chunk n of chain x, X = B * H chains) and dealt round-robin to a grid of
-// persistent CTAs, two per SM (256 TMEM columns and ~106 KB of shared memory each): CTA c runs
-// tasks c, c + G, c + 2 G, ...  Everything in a task except the carried state is independent of
-// every other task; the d_k x d_v fp32 state is relayed from the CTA that ran chunk n-1 of the
-// chain to the CTA that runs chunk n through a per-chain slot in global memory (it stays in L2).
-// Consecutive tasks of one CTA belong to different chains, so every SM holds the same amount of
-// work however B * H relates to the SM count, and consecutive chunks of one chain are loaded and
-// multiplied concurrently on different SMs; only the state relay (read 32 KB of packets, fp32
-// update, write 32 KB of packets) is serial along a chain.  Tasks are taken in increasing id and a
-// task only waits for a smaller id, so the grid cannot deadlock as long as all its CTAs are
-// resident (the host sizes the grid from the occupancy query); every wait is bounded anyway.
+// (id = n * X + x for chunk n of chain x, X = B * H chains) and handed out, in increasing order,
+// from a launch-wide counter to a grid of persistent CTAs, two per SM (256 TMEM columns and
+// ~106 KB of shared memory each): a CTA draws its next task when it has room for the task's tiles,
+// two tasks ahead of the one it computes.  Everything in a task except the carried state is
+// independent of every other task; the d_k x d_v fp32 state is relayed from the CTA that ran
+// chunk n-1 of the chain to the CTA that runs chunk n through a per-chain slot in global memory
+// (it stays in L2).  Consecutive tasks of one CTA belong to different chains, so every SM holds
+// the same amount of work however B * H relates to the SM count, and consecutive chunks of one
+// chain are loaded and multiplied concurrently on different SMs; only the state relay (read 32 KB
+// of packets, fp32 update, write 32 KB of packets) is serial along a chain.
+// Forward progress: a task waits only for a task with a smaller number; numbers are drawn by CTAs
+// that are running, each of which works through what it has drawn in increasing order.  So the
+// smallest unfinished number is always held by a running CTA that waits for nothing, whatever
+// part of the grid is resident at the time: the grid size (the host's estimate of what fits on
+// the device) is a matter of speed, not of correctness.  Every wait is bounded anyway.
 //
 // Relay packets.  A state value travels as one 64-bit word (tag in the high half, value in the low
 // half), two words per 16-byte vector access.  A 64-bit element is read and written as a unit, so
@@ -54,32 +58,22 @@
 // through the normal exit (copies in flight are waited for, TMEM is freed).
 #include "../../include/lasad.h"
 #include "lasad_common.cuh"
+#include "lasad_tc_chunk.cuh"
 #include "lasad_tc_ptx.cuh"
 #include "lasad_tc_tma.cuh"
 
 #include <cmath>
 #include <mutex>
 
-#include <cstdio>
-#include <cstdlib>
 
 namespace lasad {
 namespace {
 
 using namespace tcx;
 
-constexpr int kC = 128;                    // chunk length (tokens) = MMA M
-constexpr int kD = 64;                     // d_k = d_v
-constexpr int kEThreads = 256;             // element-wise warps 0-7
-constexpr int kThreads = kEThreads + 64;   // + the MMA warp and the TMA warp
-constexpr int kTileBytes = kC * kD * 2;    // 16 KB: one [128 x 64] bf16 tile, 128 B rows
+constexpr int kThreads = kEThreads + 64;   // element-wise warps, the MMA warp and the TMA warp
 constexpr int kStages = 2;
 constexpr int kTmemCols = 256;
-constexpr uint32_t kColS = 0;      // S (fp32, 128 columns); A/P (bf16 pairs) aliases columns 0..31 and 64..95
-constexpr uint32_t kColO = 128;    // O accumulator, 64 columns
-constexpr uint32_t kColDS = 192;   // dS accumulator (M = 64 layout), 64 columns
-constexpr unsigned kTeardownLimit = 1u << 26;
-constexpr float kFastPathMinDecay = 0.6f;
 constexpr int kHeadCache = 256;
 
 struct __align__(8) Barriers {
@@ -107,18 +101,17 @@ struct Smem {
     float pw[kC + 4];               // gamma^m, m = 0..128 (exact path only, rebuilt per task)
     float gam[kHeadCache];          // the heads' decays and their base-2 logarithms (when H <= kHeadCache)
     float lgam[kHeadCache];
+    // the tasks this CTA has drawn, by position in its sequence modulo 4 (n < 0: the work has run out);
+    // written by the TMA warp before it issues (or, for the end marker, completes by hand) the `full`
+    // barrier of that position's stage, read by the other roles after that wait
+    struct Drawn {
+        int n, x, b, h;     // chunk, chain, batch, head
+        int phase;          // (grid index of the chunk's first token + 1) mod w
+    } ring[4];
     Barriers bar;
     uint32_t tmem_base;
     int abort_flag;
 };
-
-#ifdef LASAD_TC_TRACE
-// Debug builds only: clock64() stamps of CTA 0's first element-wise thread, 8 slots per task.
-__device__ long long g_stream_trace[4096];
-#define TRACE_E(slot) do { if (blockIdx.x == 0 && tid == 0 && g < 500) g_stream_trace[8 * g + (slot)] = clock64(); } while (0)
-#else
-#define TRACE_E(slot) do { } while (0)
-#endif
 
 struct StreamParams {
     int B, T, H;
@@ -133,6 +126,7 @@ struct StreamParams {
     float* state_out;
     uint4* relay;              // [X][dk * dv / 2]: two (value, tag) packets per element
     unsigned epoch16;          // launch number folded into 1..65535: high half of the packets' tag
+    int* work;                 // [2], zero between launches: tasks drawn so far, CTAs that have left
     int* status;
     unsigned wait_limit;
 };
@@ -151,80 +145,6 @@ __device__ __forceinline__ Task decode_task(int id, int X, int H)
     return t;
 }
 
-// Decay bookkeeping of one chunk, computed by every warp on its own with four ballots (one per
-// 32-token block): which steps decay, and from their popcounts n_i for the thread's own row.
-struct ChunkDecay {
-    unsigned m0, m1, m2, m3;   // bit l of m<x>: token 32 x + l of the chunk is a decaying step
-    int c0, c1, c2;            // decaying steps up to the end of block 0, 1, 2
-    int ni;                    // n of the thread's own row
-    int n_last;                // n of the chunk's last token
-    // n of chunk column j (warp-uniform j)
-    __device__ __forceinline__ int n_of(int j) const
-    {
-        const int x = j >> 5;
-        const unsigned m = x == 0 ? m0 : x == 1 ? m1 : x == 2 ? m2 : m3;
-        const int before = x == 0 ? 0 : x == 1 ? c0 : x == 2 ? c1 : c2;
-        return before + __popc(m & (0xffffffffu >> (31 - (j & 31))));
-    }
-};
-
-// Where the call sits on the token grid, in a form that needs no division per token: token `tok`
-// of the chunk that starts at call offset cs absorbs the last token of a grid row (a boundary
-// step, SAD rule of Section 3.4) iff it lies on the grid (cs + tok >= pre) and phase + r[tok / 32]
-// is 0 or w, where r = (tok mod w) is fixed per thread and
-// phase = (grid index of the chunk's first token + 1) mod w.
-struct GridPos {
-    int grid_w;
-    int pre;         // tokens of this call that precede the grid (class-token prefix)
-    int r[4];        // (32 x + lane) mod w
-    int step;        // 128 mod w
-    int phase0;      // (grid index of the call's first token + 1) mod w
-};
-
-__device__ __forceinline__ GridPos grid_pos_init(int grid_w, int prefix_len, long long t0, int lane)
-{
-    GridPos g;
-    g.grid_w = grid_w;
-    const long long g0 = t0 - prefix_len;   // grid index of the call's first token (may be < 0)
-    g.pre = g0 < 0 ? (int)min(-g0, (long long)0x7fffffff) : 0;
-    g.step = 0; g.phase0 = 0;
-#pragma unroll
-    for (int x = 0; x < 4; ++x) g.r[x] = 0;
-    if (grid_w > 0) {
-        long long ph = (g0 + 1) % grid_w;    // C remainder: may be negative inside the prefix
-        if (ph < 0) ph += grid_w;
-        g.phase0 = (int)ph;
-        g.step = kC % grid_w;
-#pragma unroll
-        for (int x = 0; x < 4; ++x) g.r[x] = (32 * x + lane) % grid_w;
-    }
-    return g;
-}
-
-// Decay bookkeeping of chunk n of the call (L live tokens); phase = (phase0 + n * 128) mod w.
-__device__ __forceinline__ ChunkDecay chunk_decay(const GridPos& g, int phase, int n, int L, int qd, int lane)
-{
-    ChunkDecay d;
-    const int cs = n * kC;
-    unsigned mk[4];
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-        const int tok = 32 * x + lane;
-        const int m = phase + g.r[x];
-        const bool boundary = g.grid_w > 0 && cs + tok >= g.pre && (m == 0 || m == g.grid_w);
-        mk[x] = __ballot_sync(0xffffffffu, tok < L && !boundary);
-    }
-    d.m0 = mk[0]; d.m1 = mk[1]; d.m2 = mk[2]; d.m3 = mk[3];
-    d.c0 = __popc(d.m0);
-    d.c1 = d.c0 + __popc(d.m1);
-    d.c2 = d.c1 + __popc(d.m2);
-    d.n_last = d.c2 + __popc(d.m3);
-    const unsigned own = qd == 0 ? d.m0 : qd == 1 ? d.m1 : qd == 2 ? d.m2 : d.m3;
-    const int before = qd == 0 ? 0 : qd == 1 ? d.c0 : qd == 2 ? d.c1 : d.c2;
-    d.ni = before + __popc(own & (0xffffffffu >> (31 - lane)));
-    return d;
-}
-
 __global__ void __launch_bounds__(kThreads, 2)
 prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -235,11 +155,8 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const int G = (int)gridDim.x;
-    const int first = (int)blockIdx.x;
-    // tasks of this CTA: first, first + G, ...
-    const int n_local = first < p.n_tasks ? (p.n_tasks - first + G - 1) / G : 0;
     volatile int* abort_flag = &sm.abort_flag;
+    volatile Smem::Drawn* ring = sm.ring;
     const unsigned limit = p.wait_limit;
 
     // ---- set-up ---------------------------------------------------------------------------
@@ -279,33 +196,64 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     if (warp == 9) {
         // ===================== TMA warp: loads two tasks ahead, stores each output tile ========
         if (elect_one()) {
-            auto issue_loads = [&](int g) {
-                const Task t = decode_task(first + g * G, p.X, p.H);
+            // position of the call's first token relative to the grid (SAD rule, Section 3.4)
+            int step = 0, phase0 = 0;
+            if (p.grid_w > 0) {
+                long long ph = (p.t0 - p.prefix_len + 1) % p.grid_w;    // C remainder: may be negative inside the prefix
+                if (ph < 0) ph += p.grid_w;
+                phase0 = (int)ph;
+                step = kC % p.grid_w;
+            }
+            // Draws the next task from the launch-wide counter for position g of this CTA's sequence,
+            // publishes it and issues its loads; at the end of the work it publishes the end marker
+            // instead (once) and returns false.  Tasks are numbered chunk-major, so a task only
+            // depends on a smaller number, and numbers are handed out in increasing order to CTAs
+            // that are running: whoever holds the task another one waits for is making progress,
+            // whatever part of the grid is resident.
+            auto draw = [&](int g) {
                 const int s = g % kStages;
+                const int id = atomicAdd(p.work, 1);
+                volatile Smem::Drawn& d = ring[g & 3];
+                if (id >= p.n_tasks) {
+                    d.n = -1;
+                    __threadfence_block();
+                    mbar_arrive(&sm.bar.full[s]);     // completes the phase: the waiters find the marker
+                    return false;
+                }
+                const Task t = decode_task(id, p.X, p.H);
+                d.n = t.n; d.x = t.x; d.b = t.b; d.h = t.h;
+                d.phase = p.grid_w > 0 ? (int)(((long long)(t.n % p.grid_w) * step + phase0) % p.grid_w) : 0;
+                __threadfence_block();
                 mbar_arrive_expect_tx(&sm.bar.full[s], 3 * kTileBytes);
                 tma_load_4d(sm.q[s], &tm_q, &sm.bar.full[s], 0, t.h, t.n * kC, t.b);
                 tma_load_4d(sm.k[s], &tm_k, &sm.bar.full[s], 0, t.h, t.n * kC, t.b);
                 tma_load_4d(sm.v[s], &tm_v, &sm.bar.full[s], 0, t.h, t.n * kC, t.b);
+                return true;
             };
-            int loads_issued = min(n_local, kStages);
-            for (int g = 0; g < loads_issued; ++g) issue_loads(g);
-            for (int g = 0; g < n_local; ++g) {
+            int loads_issued = 0;      // positions whose loads have been issued
+            bool more = true;
+            for (int g = 0; g < kStages && more; ++g) {
+                more = draw(g);
+                if (more) loads_issued = g + 1;
+            }
+            for (int g = 0; g < loads_issued; ++g) {
                 const int s = g % kStages;
                 // the output tile of task g sits in the Q buffer of its stage; by now every MMA
                 // that read this stage has retired (the element-wise warps waited for o_done)
                 if (!mbar_wait(&sm.bar.st_ready[s], (g / kStages) & 1, limit, abort_flag, p.status)) break;
-                const Task t = decode_task(first + g * G, p.X, p.H);
-                tma_store_4d(&tm_o, sm.q[s], 0, t.h, t.n * kC, t.b);
+                tma_store_4d(&tm_o, sm.q[s], 0, ring[g & 3].h, ring[g & 3].n * kC, ring[g & 3].b);
                 tma_store_commit();
-                if (g + kStages < n_local) {
+                if (more) {
                     tma_store_wait_read();        // the store has finished reading the buffer
-                    issue_loads(g + kStages);
-                    loads_issued = g + kStages + 1;
+                    more = draw(g + kStages);
+                    if (more) loads_issued = g + kStages + 1;
                 }
             }
             tma_store_wait_all();
             // leave only when every issued load has landed (they write this CTA's shared memory)
-            for (int g = max(0, loads_issued - kStages); g < loads_issued; ++g)
+            // (once the end marker is out, the task before the last loaded one has been computed, and
+            // its stage's barrier has moved on by the marker's phase: only the last one is waited for)
+            for (int g = max(0, more ? loads_issued - kStages : loads_issued - 1); g < loads_issued; ++g)
                 for (unsigned it = 0; it < kTeardownLimit; ++it)
                     if (mbar_try_wait(&sm.bar.full[g % kStages], (g / kStages) & 1)) break;
         }
@@ -331,9 +279,9 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             }
             __syncwarp();
         };
-        bool ok = n_local > 0 && mbar_wait(&sm.bar.full[0], 0, limit, abort_flag, p.status);
+        bool ok = mbar_wait(&sm.bar.full[0], 0, limit, abort_flag, p.status) && ring[0].n >= 0;
         if (ok) issue_m1(0);
-        for (int g = 0; ok && g < n_local; ++g) {
+        for (int g = 0; ok; ++g) {
             const uint64_t dq = (g & 1) ? dq1 : dq0, dk = (g & 1) ? dk1 : dk0, dv = (g & 1) ? dv1 : dv0;
             if (!mbar_wait(&sm.bar.x_ready, g & 1, limit, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
@@ -361,13 +309,12 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             __syncwarp();
             // the scores of the next task (they overwrite A's columns: the tensor pipe runs in
             // issue order, so the A V MMAs above read A first)
-            if (g + 1 < n_local) {
-                if (!mbar_wait(&sm.bar.full[(g + 1) % kStages], ((g + 1) / kStages) & 1, limit, abort_flag, p.status)) {
-                    ok = false;
-                    break;
-                }
-                issue_m1(g + 1);
+            if (!mbar_wait(&sm.bar.full[(g + 1) % kStages], ((g + 1) / kStages) & 1, limit, abort_flag, p.status)) {
+                ok = false;
+                break;
             }
+            if (ring[(g + 1) & 3].n < 0) break;      // the work has run out
+            issue_m1(g + 1);
         }
         // make sure nothing is still running on the tensor pipe before TMEM is freed
         if (elect_one()) {
@@ -495,20 +442,16 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
         bool ok = true;
         unsigned exact_tasks = 0;    // exact-path tasks this CTA has run (phase of the table barriers)
-        // Task ids advance by G; chunk, chain, batch, head and the grid phase of the chunk's first
-        // token are advanced with them instead of being recomputed by division every task.
-        const int dn = G / p.X, dx = G - dn * p.X;
-        Task t = decode_task(first, p.X, p.H);
-        int phase = 0, dphase = 0;
-        if (p.grid_w > 0) {
-            const unsigned long long w = (unsigned long long)p.grid_w;
-            phase = (int)((((unsigned long long)t.n % w) * (unsigned)gp.step + (unsigned)gp.phase0) % w);
-            dphase = (int)((((unsigned long long)dn % w) * (unsigned)gp.step) % w);
-        }
-        for (int g = 0; ok && g < n_local; ++g) {
+        for (int g = 0; ok; ++g) {
             const int s = g % kStages;
             const unsigned par = g & 1;
-            TRACE_E(0);
+            // the task the TMA warp drew for this position (chunk, chain, batch, head, grid phase)
+            if (!(ok = mbar_wait(&sm.bar.full[s], (g / kStages) & 1, limit, abort_flag, p.status))) break;
+            Task t;
+            t.n = ring[g & 3].n;
+            if (t.n < 0) break;                      // the work has run out
+            t.x = ring[g & 3].x; t.b = ring[g & 3].b; t.h = ring[g & 3].h;
+            const int phase = ring[g & 3].phase;
             float gamma, lg;
             if (p.H <= kHeadCache) {
                 gamma = sm.gam[t.h];
@@ -520,7 +463,9 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             const bool fast = gamma >= kFastPathMinDecay;
             const bool last_chunk = t.n + 1 == p.n_chunks;
             const bool relayed_in = t.n > 0;
-            const ChunkDecay cd = chunk_decay(gp, phase, t.n, min(kC, p.T - t.n * kC), qd, lane);
+            GridPos here = gp;          // the task's chunk: offset and phase within the call
+            here.phase = phase;
+            const ChunkDecay cd = chunk_decay(here, t.n * kC, min(kC, p.T - t.n * kC), qd, lane);
             uint4* const slot = p.relay ? p.relay + (size_t)t.x * (kD * kD / 2) : nullptr;
             // tag of the state after chunk n - 1 of this launch (what this task consumes): launch
             // number and chunk index; the state this task produces carries the next tag
@@ -562,7 +507,6 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             }
             fence_proxy_async();
             mbar_arrive(&sm.bar.x_ready);
-            TRACE_E(1);
 
             // ---- E1: A = tril(S) (normal) or P = S o gamma^(n_i - n_j) o [j <= i] (exact) -> bf16
             //      over S's own columns, in 16-column pieces.  This warp converts the blocks 2 grp
@@ -633,14 +577,12 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 mbar_arrive(&sm.bar.tbl_free);    // last use of the table in this task
                 ++exact_tasks;
             }
-            TRACE_E(3);
 
             // ---- state section, the only serial link along a chain: take the incoming state
             //      (waiting for it if it is not here yet), copy it for the Q x state MMAs,
             //      E3: S_new = gamma^N S_prev + dS, hand S_new on at once
             if (!(ok = mbar_wait(&sm.bar.ds_done, par, limit, abort_flag, p.status))) break;
             tc_fence_after();
-            TRACE_E(4);
             // (the request is not issued earlier in the task: holding its 32 registers across E1
             // costs more in spills than the exposed trip from L2)
             unsigned long long rv[16];
@@ -669,7 +611,6 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     break;
                 }
             }
-            TRACE_E(2);
             // gamma^N S_prev (normal) / S_prev (exact: Q~ carries gamma^n_i)
             write_state_bf16(fast ? g_chunk : 1.0f);
             fence_proxy_async();
@@ -680,34 +621,16 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             } else if (p.state_out) {
                 store_state(p.state_out + (size_t)t.x * (kD * kD));
             }
-            TRACE_E(5);
 
             // ---- E2: o_i = scale * gamma^-(N - n_i) * O'_i (normal) / scale * O_i (exact) -----------
             const float out_f = fast ? p.scale * gpow(-(cd.n_last - cd.ni)) : p.scale;
             if (!(ok = mbar_wait(&sm.bar.o_done, par, limit, abort_flag, p.status))) break;
             tc_fence_after();
-            TRACE_E(6);
             stage_output(s, out_f);
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(&sm.bar.st_ready[s]);
-            TRACE_E(7);
 
-            // ---- next task of this CTA -----------------------------------------------------------
-            t.n += dn;
-            t.x += dx;
-            phase += dphase;
-            if (t.x >= p.X) {
-                t.x -= p.X;
-                t.n += 1;
-                phase += gp.step;
-            }
-            if (p.grid_w > 0) {
-                if (phase >= p.grid_w) phase -= p.grid_w;
-                if (phase >= p.grid_w) phase -= p.grid_w;
-            }
-            t.b = t.x / p.H;
-            t.h = t.x - t.b * p.H;
         }
     }
 
@@ -719,27 +642,30 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+    // the last CTA to leave puts the counters back to zero for the next launch
+    if (tid == 0) {
+        __threadfence();
+        if (atomicAdd(p.work + 1, 1) == (int)gridDim.x - 1) {
+            p.work[0] = 0;
+            p.work[1] = 0;
+            __threadfence();
+        }
+    }
 }
 
 }  // namespace
 
-#ifdef LASAD_TC_TRACE
-extern "C" int lasad_debug_read_stream_trace(long long* host, int n)
-{
-    return (int)cudaMemcpyFromSymbol(host, g_stream_trace, sizeof(long long) * n);
-}
-#endif
-
 int prefill_stream_chunks(int T) { return (T + kC - 1) / kC; }
 
-// Largest grid whose CTAs are all resident at once on `device` (the state relay needs that),
-// from the device's shared-memory, register and thread limits and the kernel's own needs.
+// Largest grid whose CTAs are all resident at once on `device`, from the device's shared-memory,
+// register and thread limits and the kernel's own needs: the grid size that keeps every SM busy
+// without CTAs queueing behind one another (the kernel is correct at any grid size).
 int prefill_stream_max_ctas(int device)
 {
     static int cached[64] = {0};
     if (device >= 0 && device < 64 && cached[device] > 0) return cached[device];
     const size_t smem = sizeof(Smem) + 1024;
-    int sms = 0, smem_sm = 0, smem_reserved = 0, regs_sm = 0, threads_sm = 0, api_blocks = 0;
+    int sms = 0, smem_sm = 0, smem_reserved = 0, regs_sm = 0, threads_sm = 0;
     cudaFuncAttributes fa;
     if (cudaFuncSetAttribute(prefill_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
         cudaFuncGetAttributes(&fa, prefill_stream_kernel) != cudaSuccess ||
@@ -749,16 +675,12 @@ int prefill_stream_max_ctas(int device)
         cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, device) != cudaSuccess ||
         cudaDeviceGetAttribute(&threads_sm, cudaDevAttrMaxThreadsPerMultiProcessor, device) != cudaSuccess)
         return 0;
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&api_blocks, prefill_stream_kernel, kThreads, smem);
     const int by_smem = smem_sm / (int)(smem + fa.sharedSizeBytes + smem_reserved);
     const int regs_block = ((fa.numRegs * 32 + 255) / 256 * 256) * (kThreads / 32);   // allocated per warp in units of 256
     const int by_regs = regs_block > 0 ? regs_sm / regs_block : 0;
     const int by_threads = threads_sm / kThreads;
     // TMEM: 512 columns per SM, kTmemCols per CTA
     int per_sm = min(min(by_smem, by_regs), min(by_threads, 512 / kTmemCols));
-    if (getenv("LASAD_DEBUG"))
-        fprintf(stderr, "lasad: stream prefill CTAs/SM: smem %d regs %d threads %d -> %d (occupancy API: %d), %d SMs\n",
-                by_smem, by_regs, by_threads, per_sm, api_blocks, sms);
     const int n = per_sm * sms;
     if (device >= 0 && device < 64) cached[device] = n;
     return n;
@@ -778,8 +700,9 @@ cudaError_t launch_prefill_stream(const KernelArgs& a, const TcRelay& r, cudaStr
     p.grid_w = a.grid_w; p.prefix_len = a.prefix_len; p.t0 = a.t0; p.scale = a.scale;
     p.decay = a.decay; p.state_in = a.state_in; p.state_out = a.state_out;
     p.relay = static_cast<uint4*>(r.relay); p.epoch16 = r.epoch16;
+    p.work = a.work;
     p.status = a.status; p.wait_limit = a.wait_limit;
-    if (r.max_ctas <= 0 || (p.n_chunks > 1 && !p.relay)) return cudaErrorInvalidValue;
+    if (r.max_ctas <= 0 || (p.n_chunks > 1 && !p.relay) || !p.work) return cudaErrorInvalidValue;
     const size_t smem = sizeof(Smem) + 1024;
     static bool smem_ok_1[64];
     cudaError_t e = allow_dynamic_smem(prefill_stream_kernel, smem, smem_ok_1);
@@ -872,6 +795,7 @@ extern "C" int lasad_forward_static(const lasad_params* p, const void* q, const 
     a.q = q; a.k = k; a.v = v; a.o = o;
     a.decay = decay; a.state_in = state_in; a.state_out = state_out;
     a.status = device_status ? device_status : reinterpret_cast<int*>(base + relay_bytes);
+    a.work = reinterpret_cast<int*>(base + relay_bytes) + 16;      // two counters the kernel keeps at zero between launches
     a.wait_limit = 1u << 22;
 
     lasad::TcRelay r{};

@@ -46,9 +46,6 @@ __device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity, unsigned l
 {
     for (unsigned it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-#ifdef LASAD_WAIT_SLEEP
-        __nanosleep(LASAD_WAIT_SLEEP);
-#endif
         if ((it & 63u) == 63u && *abort_flag) return false;
     }
     *abort_flag = 1;

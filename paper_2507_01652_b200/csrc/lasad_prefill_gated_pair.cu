@@ -158,6 +158,9 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     PipeBarriers& bar = sm.bar[X];
 
     // ---- set-up ---------------------------------------------------------------------------
+    // A kernel launched behind this one as a programmatic dependent may start to take SMs as they
+    // become free; it waits for this kernel's completion before it touches device memory.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) {
         for (int x = 0; x < 2; ++x) {
             PipeBarriers& b = sm.bar[x];
@@ -177,6 +180,9 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             mbar_init(&b.state_ready, kEThreads);
             mbar_init(&b.drain, 1);
         }
+        // nothing above reads or writes device memory; everything below may depend on the kernel
+        // before this one in the stream (its outputs, the work counters it puts back to zero)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         sm.abort_flag = 0;
         sm.given_up = -1;
         sm.cta = atomicAdd(p.work, 1);
@@ -792,8 +798,18 @@ cudaError_t launch_prefill_gated_pair(const KernelArgs& a, const void* gate, int
     cudaError_t e = allow_dynamic_smem(kernel, smem, smem_ok[a.fused ? 1 : 0]);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(chains < sms ? chains : sms);
-    kernel<<<grid, kPairThreads, smem, st>>>(mq, mk, mv, mg, mo, p);
-    return cudaGetLastError();
+    // programmatic dependent launch, as in launch_prefill_pair
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kPairThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mg, mo, p);
 }
 
 }  // namespace lasad

@@ -123,6 +123,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     PipeBarriers& bar = sm.bar[X];
 
     // ---- set-up ---------------------------------------------------------------------------
+    // A kernel launched behind this one as a programmatic dependent may start to take SMs as they
+    // become free; it waits for this kernel's completion before it touches device memory.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) {
         for (int x = 0; x < 2; ++x) {
             PipeBarriers& b = sm.bar[x];
@@ -140,6 +143,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             mbar_init(&b.tbl, kEThreads);
             mbar_init(&b.drain, 1);
         }
+        // nothing above reads or writes device memory; everything below may depend on the kernel
+        // before this one in the stream (its outputs, the work counters it puts back to zero)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         sm.abort_flag = 0;
         sm.cta = atomicAdd(p.work, 1);
         sm.tag = ((unsigned)*reinterpret_cast<volatile int*>(p.work + 2) & 0x3fffffffu) + 1u;   // never 0, the slots' initial content
@@ -614,8 +620,22 @@ cudaError_t launch_prefill_pair(const KernelArgs& a, void* scratch, int sms, cud
     if (e != cudaSuccess) return e;
     // Fewer chains than SMs: one chain per CTA, nothing is cut.  Otherwise one CTA per SM.
     const unsigned grid = (unsigned)(chains < sms ? chains : sms);
-    prefill_pair_kernel<<<grid, kPairThreads, smem, st>>>(mq, mk, mv, mo, p);
-    return cudaGetLastError();
+    // Programmatic dependent launch: when the kernel before this one in the stream lets its
+    // dependents go early (this kernel does, see its first lines), the CTAs of this launch may take
+    // their SMs as soon as that kernel's CTAs leave them and do their set-up there; they read
+    // nothing from device memory before griddepcontrol.wait, which returns when the earlier
+    // kernel has completed.  After any other kernel the launch behaves like an ordinary one.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kPairThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel, mq, mk, mv, mo, p);
 }
 
 }  // namespace lasad

@@ -93,7 +93,7 @@ typedef struct lasad_ctx lasad_ctx;
 
 /* Creates a context on CUDA device `device`: a status word, work counters and the scratch storage
  * of the prefill kernels (state slots at the cuts of sequences, relay slots, per-pair flags; about
- * 50 MiB in all).  Which later calls may allocate as well is said at lasad_reserve,
+ * 60 MiB in all).  Which later calls may allocate as well is said at lasad_reserve,
  * lasad_forward_host and lasad_forward_gated; no other call allocates. */
 int lasad_create(lasad_ctx** out, int device);
 int lasad_destroy(lasad_ctx* ctx);
@@ -221,7 +221,10 @@ int lasad_decode_step_pos(lasad_ctx* ctx, const lasad_params* p,
  * tensor-core kernel, which scales each 128-token chunk's queries and keys around a per-channel
  * reference decay and gives up a (batch, head) whose decay over one chunk falls below 2^-200 in
  * some channel, and a CUDA-core kernel that recomputes exactly the pairs given up, so every gate
- * in [0,1] is handled); LASAD_OPT_PREFILL_IMPL = 1 forces the CUDA-core kernel for all pairs.
+ * in [0,1] is handled).  LASAD_OPT_PREFILL_IMPL picks the tensor-core kernel: 5 the balanced one
+ * (one CTA per SM, as for lasad_forward), 2 the one with a CTA per (batch, head), 0 the balanced
+ * one where lasad_forward's default would be 5 and the other elsewhere; 1 forces the CUDA-core
+ * kernel for all pairs.
  * Other shapes and the decode step use fp32 arithmetic on CUDA cores.  The calls of one ctx
  * share a per-pair flag array: two lasad_forward_gated calls on one ctx must not overlap on the
  * device, and a call with more (batch, head) pairs than lasad_create or lasad_reserve provided

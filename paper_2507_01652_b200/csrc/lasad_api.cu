@@ -361,11 +361,24 @@ int lasad_forward(lasad_ctx* ctx, const lasad_params* p, const void* q, const vo
         return LASAD_OK;
     }
     int chunk = ctx->opt_prefill_chunk;
-    if (chunk == 0) chunk = p->dk == 64 ? 32 : 64;
+    const long long chains = (long long)p->B * p->H;
+    // few chains are cut into segments of whole chunks that run side by side: shorter chunks then
+    // give more segments (the default chunk is the one that is fastest when every SM has a chain)
+    if (chunk == 0) {
+        if (chains * 2 <= ctx->sm_count) {
+            // the longest chunk that still yields a segment for every CTA slot, else the shortest
+            const long long want = 2LL * ctx->sm_count / chains;
+            chunk = p->T / 64 >= want ? 64 : p->T / 32 >= want ? 32 : 16;
+        } else {
+            chunk = p->dk == 64 ? 32 : 64;
+        }
+    }
     if (p->T <= 16) chunk = 16;
-    const cudaError_t e = lasad::launch_prefill_simt(a, p->dk, p->dv, bf16, chunk, st);
+    const size_t scratch_floats = (size_t)2 * ctx->sm_count * 64 * 64;      // the state slots of d_segstate
+    const cudaError_t e = lasad::launch_prefill_simt(a, p->dk, p->dv, bf16, chunk, ctx->d_segstate, scratch_floats,
+                                                     ctx->sm_count, st);
     if (e != cudaSuccess) return fail_cuda(ctx, e);
-    ctx->launches += 1;
+    ctx->launches += lasad::prefill_simt_launches(p->T, p->dk, chunk, chains, ctx->sm_count, scratch_floats);
     return LASAD_OK;
 }
 

@@ -123,7 +123,10 @@ constexpr long long kTcRelaySlotBytes = 64 * 64 * 8;   // dk * dv values, each w
 int prefill_stream_chunks(int T);
 int prefill_stream_max_ctas(int device);
 cudaError_t launch_prefill_stream(const KernelArgs& a, const TcRelay& r, cudaStream_t st);
-cudaError_t launch_prefill_simt(const KernelArgs& a, int dk, int dv, bool bf16, int chunk,
-                                cudaStream_t st);
+// scratch (scratch_floats floats of device memory, or null): room for the states at the cuts when few
+// chains are cut into segments that run side by side (two launches then, else one).
+cudaError_t launch_prefill_simt(const KernelArgs& a, int dk, int dv, bool bf16, int chunk, float* scratch,
+                                size_t scratch_floats, int sms, cudaStream_t st);
+int prefill_simt_launches(int T, int dk, int chunk, long long chains, int sms, size_t scratch_floats);
 
 }  // namespace lasad

@@ -390,9 +390,22 @@ def prefill_sweep(ctx, peaks, dev, names, reps: int = 10):
 
 
 def _time_launches(stream, flush, nbytes, reps, launch):
-    """Median CUDA-event time (ms) of `launch()` over `reps` launches after 3 warm-up ones."""
+    """CUDA-event time (ms) of one `launch()`: for workloads that need the L2 cleared, the median over
+    `reps` launches, each between its own pair of events behind the clearing read; for workloads
+    larger than twice the L2, `reps` back-to-back launches between one pair of events, divided by
+    `reps` (as the main timed region does).  3 warm-up launches either way."""
     import torch
 
+    if nbytes > 2 * L2_BYTES:
+        for _ in range(3):
+            launch()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            launch()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
     evs = []
     for it in range(reps + 3):
         flush(nbytes)

@@ -327,13 +327,13 @@ def test_default_prefill_picks_a_kernel_by_the_number_of_chains(ctx):
 
 
 @pytest.mark.parametrize("B,H,T", [(1, 160, 1100), (2, 163, 1100), (1, 151, 260), (40, 5, 130), (1, 149, 2500),
-                                   (3, 7, 900)])
+                                   (3, 7, 900), (1, 150, 100), (2, 148, 300)])
 def test_balanced_prefill_left_over_chains_cut_into_pieces(ctx, B, H, T):
     """Implementation 5 with more chains than SMs: every CTA takes whole chains in rounds and one
     piece of a left-over chain, whose state travels from CTA to CTA (pieces of 4 chunks, two or three
     to a chain, some shares straddling two chains: 160 x 9 chunks; two rounds: 326 chains; chains too
-    short to be cut: 2 and 3 chunks; one long left-over chain over many CTAs: 149 x 20 chunks), and
-    with fewer chains than SMs (one chain per CTA).  Heads on both decay paths, an incoming state, a
+    short to be cut: 1, 2 and 3 chunks; one long left-over chain over many CTAs: 149 x 20 chunks;
+    whole rounds with nothing left over: 296 chains), and with fewer chains than SMs (one chain per CTA).  Heads on both decay paths, an incoming state, a
     prefix token, a start in mid-row, state_out aliasing state_in; twice in a row (the packet tags
     must tell the launches apart)."""
     d, w = 64, 13

@@ -15,10 +15,13 @@
 //
 // Only the last two lines tie a chunk to the one before it, so pipeline X works on chunk n while
 // the other works on n + 1; the fp32 state passes between them through a 16 KiB buffer, and the
-// Q~ S_prev MMAs are issued last in a chunk.  Five tiles per pipeline: gate, query (both free for
+// Q~ S_prev MMAs are issued last in a chunk (the plain form takes the state in and writes its bf16
+// copy while the score MMAs run, the fused form after E1).  Five tiles per pipeline: gate, query (both free for
 // the next chunk's loads once Q~ and K~ are written), key (scaled in place; free once the dS MMAs
-// have retired), value (free when the chunk's MMAs are done) and Q~, which doubles as the staging
-// buffer of the output tile.
+// have retired), Q~ (free for the next chunk's Q~ when the chunk's MMAs are done) and value, which
+// after the chunk's MMAs doubles as the staging buffer of the output tile: the next chunk's
+// scaling sweep then does not have to wait for the output store to have read its buffer, only the
+// next value tile's load does, and that has the whole sweep to arrive.
 //
 // A chunk whose decay is too strong for the scaling (|b_N[c]| > 200 for some channel) cannot be
 // taken this way.  The kernel then marks the chain in `redo` and lets a flag travel with the
@@ -55,7 +58,6 @@ struct __align__(8) PipeBarriers {
     unsigned long long full_v;      // value tile has landed
     unsigned long long scan;        // partial sums of the chunk are in shared memory (256 arrivals)
     unsigned long long in_free;     // last read of the gate and query tiles of the chunk (256 arrivals)
-    unsigned long long stage_free;  // the store of the previous output tile has read its staging buffer
     unsigned long long x_ready;     // Q~ and K~ are written (256 arrivals)
     unsigned long long s_done;      // M1 complete
     unsigned long long ds_done;     // dS MMAs complete (and M1): the key tile is free
@@ -72,8 +74,8 @@ struct Smem {
     unsigned char g[2][kTileBytes];     // gate lambda (fused form: pre-activation, then 1 - lambda)
     unsigned char q[2][kTileBytes];
     unsigned char k[2][kTileBytes];     // keys, scaled in place to K~
-    unsigned char v[2][kTileBytes];
-    unsigned char qt[2][kTileBytes];    // Q~; after the MMAs the staging buffer of the output tile
+    unsigned char v[2][kTileBytes];     // values; after the MMAs the staging buffer of the output tile
+    unsigned char qt[2][kTileBytes];    // Q~
     unsigned char sb[2][kD * kD * 2];   // per pipeline: bf16 copy of diag(2^r) state, [dk][dv], 128 B rows, swizzled
     float4 sf[4][kEThreads];            // the fp32 state between two chunks: element-wise thread t's 16 values
     float segsum[2][8][kD];             // log2 of the product of Lambda over rows 16 x .. 16 x + 15, per channel
@@ -169,7 +171,6 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             mbar_init(&b.full_v, 1);
             mbar_init(&b.scan, kEThreads);
             mbar_init(&b.in_free, kEThreads);
-            mbar_init(&b.stage_free, 1);
             mbar_init(&b.x_ready, kEThreads);
             mbar_init(&b.s_done, 1);
             mbar_init(&b.ds_done, 1);
@@ -216,7 +217,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     if (warp == 9) {
         // ===================== TMA warp ========================================================
         // One set of tiles per pipeline; each is refilled for the pipeline's next chunk as soon as its
-        // last reader is done.  The output tile leaves from the Q~ buffer.
+        // last reader is done.  The output tile leaves from the value buffer.
         if (elect_one() && J > 0) {
             Unit lu;
             lu.g0 = 0; lu.g1 = -1;
@@ -259,21 +260,19 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                         issue_k();
                         k_issued = j + 2;
                     }
-                    if (!mbar_wait(&bar.o_done, j & 1, limit, abort_flag, p.status)) break;
-                    issue_v();
-                    v_issued = j + 2;
                 }
                 if (!mbar_wait(&bar.st_ready, j & 1, limit, abort_flag, p.status)) break;
                 {
                     const int g = 2 * j + X;
                     if (g >= su.g1) su = unit_of(plan, g);
                     const int sb_ = su.chain / p.H, sh = su.chain - sb_ * p.H;
-                    tma_store_4d(&tm_o, sm.qt[X], 0, sh, (su.n0 + g - su.g0) * kC, sb_);
+                    tma_store_4d(&tm_o, sm.v[X], 0, sh, (su.n0 + g - su.g0) * kC, sb_);
                     tma_store_commit();
                 }
                 if (more) {
-                    tma_store_wait_read();        // the store has finished reading the buffer
-                    mbar_arrive(&bar.stage_free);
+                    tma_store_wait_read();        // the store has finished reading the buffer: the next values may land
+                    issue_v();
+                    v_issued = j + 2;
                 }
             }
             tma_store_wait_all();
@@ -385,7 +384,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         };
         // this thread's 32 columns of output row i -> bf16 -> row i of the staging buffer
         auto stage_output = [&](float f) {
-            unsigned char* orow = tqt + i * 128;
+            unsigned char* orow = sm.v[X] + i * 128;
             uint32_t ov[32];
             tmem_ld32(tmem + lane_base + kColO + 32 * grp, ov);
             tmem_wait_ld();
@@ -451,20 +450,17 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             for (int rr = 0; rr < 16; ++rr) {
                 uint32_t g2 = *reinterpret_cast<const uint32_t*>(tg + row_off(rr));
                 if (kFused) {
-                    // u = Sigmoid(-g~) = 1 - lambda, written back in place; lambda = 1 - u
-                    const float e0 = ex2(-1.4426950408889634f * fminf(fmaxf(bf16_lo(g2), -80.0f), 80.0f));
-                    const float e1 = ex2(-1.4426950408889634f * fminf(fmaxf(bf16_hi(g2), -80.0f), 80.0f));
-                    const uint32_t u2 = pack_bf16(e0 * rcp_approx(1.0f + e0), e1 * rcp_approx(1.0f + e1));
+                    // u = Sigmoid(-g~) = 1 / (1 + e^g~) = 1 - lambda, written back in place; lambda = 1 - u
+                    // (e^g~ = inf gives u = 0 and e^g~ = 0 gives u = 1: no clamp is needed)
+                    const uint32_t u2 = pack_bf16(rcp_approx(1.0f + ex2(1.4426950408889634f * bf16_lo(g2))),
+                                                  rcp_approx(1.0f + ex2(1.4426950408889634f * bf16_hi(g2))));
                     *reinterpret_cast<uint32_t*>(tg + row_off(rr)) = u2;
-                    if ((dec >> rr) & 1u) {
-                        p0 *= 1.0f - bf16_lo(u2);
-                        p1 *= 1.0f - bf16_hi(u2);
-                    }
+                    const uint32_t us = ((dec >> rr) & 1u) ? u2 : 0u;
+                    mul2_pair(p0, p1, 1.0f - bf16_lo(us), 1.0f - bf16_hi(us));
                     continue;
                 }
                 g2 = ((dec >> rr) & 1u) ? g2 : 0x3f803f80u;
-                p0 *= bf16_lo(g2);
-                p1 *= bf16_hi(g2);
+                mul2_pair(p0, p1, bf16_lo(g2), bf16_hi(g2));
             }
             // a product that has left the fp32 range reads as -inf and fails the range check
             *reinterpret_cast<float2*>(&segsum[warp][2 * lane]) = make_float2(lg2(p0), lg2(p1));
@@ -480,16 +476,12 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             const Unit u = nx.u;                        // the chunk being worked on
             const int n = nx.n;
             const int Lc = min(kC, p.T - n * kC);
-            // the decay pair of row rr of this warp in fp32 (fused form: the tile holds u = 1 - lambda)
+            // the decay pair of row rr of this warp in fp32 (fused form: the tile holds u = 1 - lambda);
+            // a boundary step or a dead row has decay 1 (one select, on the packed word)
             auto decay_pair = [&](uint32_t g2, int rr, float& l0, float& l1) {
-                const bool dec = (dec16 >> rr) & 1u;
-                if (kFused) {
-                    l0 = dec ? 1.0f - bf16_lo(g2) : 1.0f;
-                    l1 = dec ? 1.0f - bf16_hi(g2) : 1.0f;
-                } else {
-                    l0 = dec ? bf16_lo(g2) : 1.0f;
-                    l1 = dec ? bf16_hi(g2) : 1.0f;
-                }
+                const uint32_t x = ((dec16 >> rr) & 1u) ? g2 : (kFused ? 0u : 0x3f803f80u);
+                l0 = kFused ? 1.0f - bf16_lo(x) : bf16_lo(x);
+                l1 = kFused ? 1.0f - bf16_hi(x) : bf16_hi(x);
             };
             if (!(ok = mbar_wait(&bar.scan, j & 1, limit, abort_flag, p.status))) break;
 
@@ -497,8 +489,9 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             float f0, f1;       // 2^(b - r) just before this warp's first row
             float t0, t1;       // 2^(r - b) at this warp's last row
             bool too_strong;
+            float tot0 = 0.0f, tot1 = 0.0f;     // log2 of the chunk's total decay, this lane's two channels
             {
-                float base0 = 0.0f, base1 = 0.0f, tot0 = 0.0f, tot1 = 0.0f;
+                float base0 = 0.0f, base1 = 0.0f;
 #pragma unroll
                 for (int x = 0; x < 8; ++x) {
                     const float2 bsx = *reinterpret_cast<const float2*>(&segsum[x][2 * lane]);
@@ -514,20 +507,22 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 too_strong = __any_sync(0xffffffffu, !(fabsf(tot0) <= kSafeRange) || !(fabsf(tot1) <= kSafeRange));
             }
             // per-row factors of the state (rows r0 and r0 + 8 are channels): 2^(b_N / 2) = 2^r = 2^(b_N - r)
+            // (channel c's total sits in lane c / 2, component c & 1)
             float m_a, m_b;
             {
-                float ta = 0.0f, tb = 0.0f;
-#pragma unroll
-                for (int x = 0; x < 8; ++x) { ta += segsum[x][r0]; tb += segsum[x][r0 + 8]; }
-                m_a = ex2(0.5f * ta);
-                m_b = ex2(0.5f * tb);
+                const int src = 8 * qd + (lane >> 3);
+                const float a0 = __shfl_sync(0xffffffffu, tot0, src), a1 = __shfl_sync(0xffffffffu, tot1, src);
+                const float b0 = __shfl_sync(0xffffffffu, tot0, src + 4), b1 = __shfl_sync(0xffffffffu, tot1, src + 4);
+                const bool odd = (lane >> 2) & 1;
+                m_a = ex2(0.5f * (odd ? a1 : a0));
+                m_b = ex2(0.5f * (odd ? b1 : b0));
             }
 
             // ---- second sweep: Q~ = Q o 2^(b - r) with the factor carried forward down the rows as a
             //      running product of the gates, K~ = K o 2^(r - b) with its factor carried backward
             //      from the warp's last row, so that no factor is ever inverted.  (Rows in groups of
             //      eight: a group's loads are issued before its stores.)
-            if (j > 0 && !(ok = mbar_wait(&bar.stage_free, (j - 1) & 1, limit, abort_flag, p.status))) break;
+            // (the Q~ buffer is free: this thread has waited for the previous chunk's last MMA)
 #pragma unroll
             for (int r8 = 0; r8 < 16; r8 += 8) {
                 uint32_t g2[8], q2[8];
@@ -540,8 +535,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 for (int x = 0; x < 8; ++x) {
                     float l0, l1;
                     decay_pair(g2[x], r8 + x, l0, l1);
-                    f0 *= l0;
-                    f1 *= l1;
+                    mul2_pair(f0, f1, l0, l1);
                     if (kFused) {
                         // q = SiLU(q~) = q~ (1 + tanh(q~ / 2)) / 2, scaled in the same step
                         const float x0 = bf16_lo(q2[x]), x1 = bf16_hi(q2[x]);
@@ -568,8 +562,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                         *reinterpret_cast<uint32_t*>(tk + row_off(r8 + x)) = mul_bf16x2(k2[x], pack_bf16(t0, t1));
                         float l0, l1;
                         decay_pair(g2[x], r8 + x, l0, l1);
-                        t0 *= l0;
-                        t1 *= l1;
+                        mul2_pair(t0, t1, l0, l1);
                     }
                 }
             } else {
@@ -590,8 +583,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                                 pack_bf16((one - bf16_lo(g2[x])) * t0, (one - bf16_hi(g2[x])) * t1);
                         float l0, l1;
                         decay_pair(g2[x], r8 + x, l0, l1);
-                        t0 *= l0;
-                        t1 *= l1;
+                        mul2_pair(t0, t1, l0, l1);
                     }
                 }
             }
@@ -601,6 +593,55 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             tc_fence_before();
             mbar_arrive(&bar.x_ready);
 
+            // ---- the carried state: in from the other pipeline's chunk (or from where the unit
+            //      starts), out to the other pipeline's next chunk (or to where the unit ends).  Taking it
+            //      in and writing its bf16 copy needs no MMA result, so the plain form does it while
+            //      the score MMAs run; the fused form, whose sweeps are longer, runs faster with it
+            //      after E1 -------------------------------------------------------------------------
+            bool given_up = false;          // this chain has been given up (here or earlier)
+            auto take_state = [&]() -> bool {
+                if (g > 0) {
+                    // the other pipeline is done with chunk g - 1 (its j index: j for X = 1, j - 1 for X = 0)
+                    if (!mbar_wait(&other.state_ready, (j - 1 + X) & 1, limit, abort_flag, p.status)) return false;
+                }
+                if (g == u.g0) {
+                    if (u.recv < 0) {
+                        // a chain starts: the caller's state or zero
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) st[e] = 0.0f;
+                        if (p.state_in) {
+                            const float* sin = p.state_in + (size_t)u.chain * kD * kD;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const float2 a = *reinterpret_cast<const float2*>(sin + (size_t)r0 * kD + c0 + 8 * k);
+                                const float2 c = *reinterpret_cast<const float2*>(sin + (size_t)(r0 + 8) * kD + c0 + 8 * k);
+                                st[4 * k] = a.x; st[4 * k + 1] = a.y; st[4 * k + 2] = c.x; st[4 * k + 3] = c.y;
+                            }
+                        }
+                    } else {
+                        // the chain was cut here: its state (and whether it has been given up) comes from
+                        // where the part before it was done
+                        if (!slot_receive(p.slots + (size_t)u.recv * kSlotBytes, tid, st, sm.tag, limit, abort_flag, p.status, &given_up))
+                            return false;
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float4 x = sm.sf[k][tid];
+                        st[4 * k] = x.x; st[4 * k + 1] = x.y; st[4 * k + 2] = x.z; st[4 * k + 3] = x.w;
+                    }
+                    given_up = *reinterpret_cast<volatile int*>(&sm.given_up) == u.chain;
+                }
+                if (too_strong && !given_up) {
+                    given_up = true;
+                    if (tid == 0) p.redo[u.chain] = 1;
+                }
+                write_state_bf16(m_a, m_b);
+                fence_proxy_async();
+                mbar_arrive(&bar.sb_ready);
+                return true;
+            };
+            if (!kFused && !(ok = take_state())) break;
             // ---- E1: A = tril(S) -> bf16 over S's own columns (blocks 2 grp, 2 grp + 1 of this
             //      thread's row, kept inside this warp's half of S's columns) -------------------------
             if (!(ok = mbar_wait(&bar.s_done, j & 1, limit, abort_flag, p.status))) break;
@@ -632,50 +673,8 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&bar.p_ready);
+            if (kFused && !(ok = take_state())) break;
 
-            // ---- the carried state: in from the other pipeline's chunk (or from where the unit
-            //      starts), out to the other pipeline's next chunk (or to where the unit ends) -------
-            if (g > 0) {
-                // the other pipeline is done with chunk g - 1 (its j index: j for X = 1, j - 1 for X = 0)
-                if (!(ok = mbar_wait(&other.state_ready, (j - 1 + X) & 1, limit, abort_flag, p.status))) break;
-            }
-            bool given_up = false;          // this chain has been given up (here or earlier)
-            if (g == u.g0) {
-                if (u.recv < 0) {
-                    // a chain starts: the caller's state or zero
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) st[e] = 0.0f;
-                    if (p.state_in) {
-                        const float* sin = p.state_in + (size_t)u.chain * kD * kD;
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const float2 a = *reinterpret_cast<const float2*>(sin + (size_t)r0 * kD + c0 + 8 * k);
-                            const float2 c = *reinterpret_cast<const float2*>(sin + (size_t)(r0 + 8) * kD + c0 + 8 * k);
-                            st[4 * k] = a.x; st[4 * k + 1] = a.y; st[4 * k + 2] = c.x; st[4 * k + 3] = c.y;
-                        }
-                    }
-                } else {
-                    // the chain was cut here: its state (and whether it has been given up) comes from
-                    // where the part before it was done
-                    if (!(ok = slot_receive(p.slots + (size_t)u.recv * kSlotBytes, tid, st, sm.tag, limit, abort_flag, p.status,
-                                            &given_up)))
-                        break;
-                }
-            } else {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float4 x = sm.sf[k][tid];
-                    st[4 * k] = x.x; st[4 * k + 1] = x.y; st[4 * k + 2] = x.z; st[4 * k + 3] = x.w;
-                }
-                given_up = *reinterpret_cast<volatile int*>(&sm.given_up) == u.chain;
-            }
-            if (too_strong && !given_up) {
-                given_up = true;
-                if (tid == 0) p.redo[u.chain] = 1;
-            }
-            write_state_bf16(m_a, m_b);
-            fence_proxy_async();
-            mbar_arrive(&bar.sb_ready);
             // S_new = diag(f) S_prev + diag(m) dS, with f = m * m (rows r0 and r0 + 8)
             if (!(ok = mbar_wait(&bar.ds_done, j & 1, limit, abort_flag, p.status))) break;
             tc_fence_after();

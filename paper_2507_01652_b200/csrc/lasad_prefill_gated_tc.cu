@@ -70,7 +70,8 @@ struct __align__(8) Barriers {
     unsigned long long scan;       // partial sums of the chunk are in shared memory (256 arrivals)
     unsigned long long in_free;    // last read of the gate, query and key tiles of the chunk (256 arrivals)
     unsigned long long stage_free; // the store of the previous output tile has read its staging buffer
-    unsigned long long x_ready;    // Q~, K~ and the state copy are written (256 arrivals)
+    unsigned long long x_ready;    // Q~ and K~ are written (256 arrivals)
+    unsigned long long sb_ready;   // bf16 copy of the scaled state is written (256 arrivals)
     unsigned long long s_done;     // M1 complete
     unsigned long long ds_done;    // dS MMAs complete
     unsigned long long p_ready;    // A in TMEM (256 arrivals)
@@ -167,6 +168,7 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         mbar_init(&sm.bar.in_free, kEThreads);
         mbar_init(&sm.bar.stage_free, 1);
         mbar_init(&sm.bar.x_ready, kEThreads);
+        mbar_init(&sm.bar.sb_ready, kEThreads);
         mbar_init(&sm.bar.s_done, 1);
         mbar_init(&sm.bar.ds_done, 1);
         mbar_init(&sm.bar.p_ready, kEThreads);
@@ -251,10 +253,6 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                 for (int kk = 0; kk < kD / 16; ++kk)  // 32 bytes along K per step
                     mma_ss(tmem + kColS, d_q + 2 * kk, d_k + 2 * kk, idesc_s, kk > 0);
                 mma_commit(&sm.bar.s_done);
-                // the state's contribution opens the O accumulator; A V is added once A is ready
-#pragma unroll
-                for (int kk = 0; kk < kD / 16; ++kk)
-                    mma_ss(tmem + kColO, d_q + 2 * kk, d_sb + 128 * kk, idesc_qs, kk > 0);
             }
             __syncwarp();
             if (!mbar_wait(&sm.bar.full_v, n & 1, limit, abort_flag, p.status)) break;
@@ -264,6 +262,16 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                 for (int kk = 0; kk < kC / 16; ++kk)  // 16 tokens = 2048 B of K~ and of V per step
                     mma_ss(tmem + kColDS, d_k + 128 * kk, d_v + 128 * kk, idesc_kv, kk > 0);
                 mma_commit(&sm.bar.ds_done);
+            }
+            __syncwarp();
+            // the state's contribution opens the O accumulator (its bf16 copy is written while the
+            // score MMAs run); A V is added once A is ready
+            if (!mbar_wait(&sm.bar.sb_ready, n & 1, limit, abort_flag, p.status)) break;
+            tc_fence_after();
+            if (elect_one()) {
+#pragma unroll
+                for (int kk = 0; kk < kD / 16; ++kk)
+                    mma_ss(tmem + kColO, d_q + 2 * kk, d_sb + 128 * kk, idesc_qs, kk > 0);
             }
             __syncwarp();
             if (!mbar_wait(&sm.bar.p_ready, n & 1, limit, abort_flag, p.status)) break;
@@ -423,20 +431,17 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             for (int rr = 0; rr < 16; ++rr) {
                 uint32_t g2 = *reinterpret_cast<const uint32_t*>(sm.g + row_off(rr));
                 if (kFused) {
-                    // u = Sigmoid(-g~) = 1 - lambda, written back in place; lambda = 1 - u
-                    const float e0 = ex2(-1.4426950408889634f * fminf(fmaxf(bf16_lo(g2), -80.0f), 80.0f));
-                    const float e1 = ex2(-1.4426950408889634f * fminf(fmaxf(bf16_hi(g2), -80.0f), 80.0f));
-                    const uint32_t u2 = pack_bf16(e0 * rcp_approx(1.0f + e0), e1 * rcp_approx(1.0f + e1));
+                    // u = Sigmoid(-g~) = 1 / (1 + e^g~) = 1 - lambda, written back in place; lambda = 1 - u
+                    // (e^g~ = inf gives u = 0 and e^g~ = 0 gives u = 1: no clamp is needed)
+                    const uint32_t u2 = pack_bf16(rcp_approx(1.0f + ex2(1.4426950408889634f * bf16_lo(g2))),
+                                                  rcp_approx(1.0f + ex2(1.4426950408889634f * bf16_hi(g2))));
                     *reinterpret_cast<uint32_t*>(sm.g + row_off(rr)) = u2;
-                    if ((dec >> rr) & 1u) {
-                        p0 *= 1.0f - bf16_lo(u2);
-                        p1 *= 1.0f - bf16_hi(u2);
-                    }
+                    const uint32_t us = ((dec >> rr) & 1u) ? u2 : 0u;
+                    mul2_pair(p0, p1, 1.0f - bf16_lo(us), 1.0f - bf16_hi(us));
                     continue;
                 }
                 g2 = ((dec >> rr) & 1u) ? g2 : 0x3f803f80u;
-                p0 *= bf16_lo(g2);
-                p1 *= bf16_hi(g2);
+                mul2_pair(p0, p1, bf16_lo(g2), bf16_hi(g2));
             }
             // a product that has left the fp32 range reads as -inf and fails the range check
             *reinterpret_cast<float2*>(&sm.segsum[warp][2 * lane]) = make_float2(lg2(p0), lg2(p1));
@@ -468,8 +473,9 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             // ---- this warp's place in the chunk, the chunk's total, the range check ----------------
             float f0, f1;       // 2^(b - r) just before this warp's first row
             float t0, t1;       // 2^(r - b) at this warp's last row
+            float tot0 = 0.0f, tot1 = 0.0f;     // log2 of the chunk's total decay, this lane's two channels
             {
-                float base0 = 0.0f, base1 = 0.0f, tot0 = 0.0f, tot1 = 0.0f;
+                float base0 = 0.0f, base1 = 0.0f;
 #pragma unroll
                 for (int x = 0; x < 8; ++x) {
                     const float2 bsx = *reinterpret_cast<const float2*>(&sm.segsum[x][2 * lane]);
@@ -490,13 +496,15 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                 }
             }
             // per-row factors of the state (rows r0 and r0 + 8 are channels): 2^(b_N / 2) = 2^r = 2^(b_N - r)
+            // (channel c's total sits in lane c / 2, component c & 1)
             float m_a, m_b;
             {
-                float ta = 0.0f, tb = 0.0f;
-#pragma unroll
-                for (int x = 0; x < 8; ++x) { ta += sm.segsum[x][r0]; tb += sm.segsum[x][r0 + 8]; }
-                m_a = ex2(0.5f * ta);
-                m_b = ex2(0.5f * tb);
+                const int src = 8 * qd + (lane >> 3);
+                const float a0 = __shfl_sync(0xffffffffu, tot0, src), a1 = __shfl_sync(0xffffffffu, tot1, src);
+                const float b0 = __shfl_sync(0xffffffffu, tot0, src + 4), b1 = __shfl_sync(0xffffffffu, tot1, src + 4);
+                const bool odd = (lane >> 2) & 1;
+                m_a = ex2(0.5f * (odd ? a1 : a0));
+                m_b = ex2(0.5f * (odd ? b1 : b0));
             }
 
             // ---- second sweep: Q~ = Q o 2^(b - r) with the factor carried forward down the rows as a
@@ -518,8 +526,7 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                 for (int x = 0; x < 8; ++x) {
                     float l0, l1;
                     decay_pair(g2[x], r8 + x, l0, l1);
-                    f0 *= l0;
-                    f1 *= l1;
+                    mul2_pair(f0, f1, l0, l1);
                     if (kFused) {
                         // q = SiLU(q~) = q~ (1 + tanh(q~ / 2)) / 2, scaled in the same step
                         const float x0 = bf16_lo(q2[x]), x1 = bf16_hi(q2[x]);
@@ -545,8 +552,7 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                         *reinterpret_cast<uint32_t*>(sm.kt + row_off(r8 + x)) = mul_bf16x2(k2[x], pack_bf16(t0, t1));
                         float l0, l1;
                         decay_pair(g2[x], r8 + x, l0, l1);
-                        t0 *= l0;
-                        t1 *= l1;
+                        mul2_pair(t0, t1, l0, l1);
                     }
                 }
             } else {
@@ -567,17 +573,20 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                                 pack_bf16((one - bf16_lo(g2[x])) * t0, (one - bf16_hi(g2[x])) * t1);
                         float l0, l1;
                         decay_pair(g2[x], r8 + x, l0, l1);
-                        t0 *= l0;
-                        t1 *= l1;
+                        mul2_pair(t0, t1, l0, l1);
                     }
                 }
             }
-            write_state_bf16(m_a, m_b);
             if (kFused) fence_proxy_async();      // the gate tile was rewritten in place: order that before its refill
             mbar_arrive(&sm.bar.in_free);
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(&sm.bar.x_ready);
+            // the state's bf16 copy, while the score MMAs run (the previous chunk's MMAs, the last
+            // readers of the buffer, were waited for at the end of that chunk)
+            write_state_bf16(m_a, m_b);
+            fence_proxy_async();
+            mbar_arrive(&sm.bar.sb_ready);
 
             // ---- E1: A = tril(S) -> bf16 over S's own columns (blocks 2 grp, 2 grp + 1 of this
             //      thread's row, kept inside this warp's half of S's columns) -------------------------

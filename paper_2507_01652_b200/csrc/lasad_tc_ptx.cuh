@@ -183,6 +183,15 @@ __device__ __forceinline__ void mul2(float a0, float a1, float b, float& r0, flo
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(pr) : "l"(pa), "l"(pb));
     asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(pr));
 }
+// {a0 * b0, a1 * b1}, in place
+__device__ __forceinline__ void mul2_pair(float& a0, float& a1, float b0, float b1)
+{
+    unsigned long long pa, pb;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(pa) : "f"(a0), "f"(a1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(pb) : "f"(b0), "f"(b1));
+    asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(pa) : "l"(pb));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(pa));
+}
 // {a0 * b + c0, a1 * b + c1}
 __device__ __forceinline__ void fma2(float a0, float a1, float b, float c0, float c1, float& r0, float& r1)
 {

@@ -352,6 +352,36 @@ def test_balanced_prefill_left_over_chains_cut_into_pieces(ctx, B, H, T):
         assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
 
 
+def test_expired_wait_while_states_cross_ctas_is_reported_and_the_next_call_is_right(ctx):
+    """Implementation 5 on 160 chains of 9 chunks (left-over chains in pieces, their states handed
+    from CTA to CTA) with the poll limit of the device-side waits set to 1: some wait -- on a barrier
+    or on a hand-off packet -- runs out, every CTA must still leave through its normal exit (so the
+    launch counters are put back), the status word must say so, and the next call with the default
+    limit must be correct: the packets the aborted launch left behind carry its tag, not the next one's."""
+    B, H, T, d, w = 1, 160, 1100, 64, 9
+    gen = torch.Generator().manual_seed(81)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+    g = 0.9 + 0.0999 * torch.rand(H, generator=gen)
+    o_ref, s_ref = oracle(q, k, v, g, w)
+    dq, dk, dv, dg = _dev(q, k, v, g)
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 5)
+    try:
+        ctx.set_option(binding.LASAD_OPT_WAIT_LIMIT, 1)
+        ctx.lasad_forward(dq, dk, dv, dg, w)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == binding.LASAD_ERR_TIMEOUT
+        ctx.set_option(binding.LASAD_OPT_WAIT_LIMIT, 0)
+        for rep in range(2):
+            o, s = ctx.lasad_forward(dq, dk, dv, dg, w)
+            torch.cuda.synchronize()
+            assert ctx.device_status() == 0, rep
+            assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+            assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
+    finally:
+        ctx.set_option(binding.LASAD_OPT_WAIT_LIMIT, 0)
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
+
+
 def test_balanced_prefill_recorded_into_a_cuda_graph_and_replayed(ctx):
     """Implementation 5 numbers its launches on the device, so a recorded launch may be replayed: the
     hand-off packets of one replay must not pass for the next one's (160 chains of 9 chunks: the

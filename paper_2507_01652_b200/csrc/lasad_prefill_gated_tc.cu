@@ -510,10 +510,12 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             // ---- second sweep: Q~ = Q o 2^(b - r) with the factor carried forward down the rows as a
             //      running product of the gates, K~ = K o 2^(r - b) with its factor carried backward
             //      from the warp's last row, so that no factor is ever inverted.  The fp32 factors are
-            //      rounded to bf16 and applied with packed bf16 multiplies.  (Rows in groups of eight:
+            //      rounded to bf16 and applied with packed bf16 multiplies; the forward pass keeps the
+            //      16 decay pairs in registers for the backward pass.  (Rows in groups of eight:
             //      a group's loads are issued before its stores, which the compiler must take to
             //      alias later loads.)
             if (n > 0 && !(ok = mbar_wait(&sm.bar.stage_free, (n - 1) & 1, limit, abort_flag, p.status))) break;
+            float ls0[16], ls1[16];     // the 16 decay pairs in fp32, kept for the backward pass
 #pragma unroll
             for (int r8 = 0; r8 < 16; r8 += 8) {
                 uint32_t g2[8], q2[8];
@@ -524,9 +526,8 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                 }
 #pragma unroll
                 for (int x = 0; x < 8; ++x) {
-                    float l0, l1;
-                    decay_pair(g2[x], r8 + x, l0, l1);
-                    mul2_pair(f0, f1, l0, l1);
+                    decay_pair(g2[x], r8 + x, ls0[r8 + x], ls1[r8 + x]);
+                    mul2_pair(f0, f1, ls0[r8 + x], ls1[r8 + x]);
                     if (kFused) {
                         // q = SiLU(q~) = q~ (1 + tanh(q~ / 2)) / 2, scaled in the same step
                         const float x0 = bf16_lo(q2[x]), x1 = bf16_hi(q2[x]);
@@ -541,18 +542,13 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             if (!p.tied) {
 #pragma unroll
                 for (int r8 = 8; r8 >= 0; r8 -= 8) {
-                    uint32_t g2[8], k2[8];
+                    uint32_t k2[8];
 #pragma unroll
-                    for (int x = 0; x < 8; ++x) {
-                        g2[x] = *reinterpret_cast<const uint32_t*>(sm.g + row_off(r8 + x));
-                        k2[x] = *reinterpret_cast<const uint32_t*>(sm.k + row_off(r8 + x));
-                    }
+                    for (int x = 0; x < 8; ++x) k2[x] = *reinterpret_cast<const uint32_t*>(sm.k + row_off(r8 + x));
 #pragma unroll
                     for (int x = 7; x >= 0; --x) {
                         *reinterpret_cast<uint32_t*>(sm.kt + row_off(r8 + x)) = mul_bf16x2(k2[x], pack_bf16(t0, t1));
-                        float l0, l1;
-                        decay_pair(g2[x], r8 + x, l0, l1);
-                        mul2_pair(t0, t1, l0, l1);
+                        mul2_pair(t0, t1, ls0[r8 + x], ls1[r8 + x]);
                     }
                 }
             } else {
@@ -571,9 +567,7 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                         else
                             *reinterpret_cast<uint32_t*>(sm.kt + row_off(r8 + x)) =
                                 pack_bf16((one - bf16_lo(g2[x])) * t0, (one - bf16_hi(g2[x])) * t1);
-                        float l0, l1;
-                        decay_pair(g2[x], r8 + x, l0, l1);
-                        mul2_pair(t0, t1, l0, l1);
+                        mul2_pair(t0, t1, ls0[r8 + x], ls1[r8 + x]);
                     }
                 }
             }

@@ -36,7 +36,7 @@ NCU_TRAFFIC_BYTES = {
     # (config 5a), scaled by tokens to config 5b
     "prefill": 861_900_000,
     # decode_kernel, config 4, inside the kernel (the rest of the written state drains from L2 later)
-    "decode": 112_200_000,
+    "decode": 111_800_000,
 }
 
 

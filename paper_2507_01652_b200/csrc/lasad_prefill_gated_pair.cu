@@ -640,7 +640,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             //      thread's row, kept inside this warp's half of S's columns) -------------------------
             if (!(ok = mbar_wait(&bar.s_done, j & 1, limit, abort_flag, p.status))) break;
             tc_fence_after();
-#pragma unroll
+#pragma unroll 1
             for (int pi = 0; pi < 2; ++pi) {
                 const int pc = 2 * grp + pi;
                 uint32_t pk[16];

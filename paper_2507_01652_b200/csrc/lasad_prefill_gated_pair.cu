@@ -94,7 +94,6 @@ struct GatedPairParams {
     int grid_w, prefix_len;
     long long t0;
     float scale;
-    int tied;                // key tied to the gate: k = 1 - lambda, no key tensor
     const float* state_in;
     float* state_out;
     int* redo;               // [B*H], zero between launches: set to 1 where this kernel gave the chain up
@@ -139,7 +138,8 @@ __device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b)
     return r;
 }
 
-template <bool kFused>
+// kTied: the key is the gate's complement, k = 1 - lambda, and there is no key tensor.
+template <bool kFused, bool kTied>
 __global__ void __launch_bounds__(kPairThreads, 1)
 prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                           const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g,
@@ -244,9 +244,9 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 tma_load_4d(sm.v[X], &tm_v, &bar.full_v, 0, h, tok, b);
             };
             issue_gq(0);
-            if (!p.tied) issue_k();
+            if (!kTied) issue_k();
             issue_v();
-            int gq_issued = 1, k_issued = p.tied ? 0 : 1, v_issued = 1;     // chunks whose loads have been issued
+            int gq_issued = 1, k_issued = kTied ? 0 : 1, v_issued = 1;     // chunks whose loads have been issued
             Unit su;
             su.g0 = 0; su.g1 = -1;
             for (int j = 0; j < J; ++j) {
@@ -255,7 +255,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     if (!mbar_wait(&bar.in_free, j & 1, limit, abort_flag, p.status)) break;
                     issue_gq(j + 1);
                     gq_issued = j + 2;
-                    if (!p.tied) {
+                    if (!kTied) {
                         if (!mbar_wait(&bar.ds_done, j & 1, limit, abort_flag, p.status)) break;
                         issue_k();
                         k_issued = j + 2;
@@ -425,7 +425,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         // moves `nx` to local chunk g and returns which of this warp's 16 rows of it are decaying
         // steps (live and not a row boundary, SAD rule of Section 3.4)
         auto advance = [&](int g) -> unsigned {
-            if (g >= nx.u.g1) {
+            if (__builtin_expect(g >= nx.u.g1, 0)) {
                 nx.u = unit_of(plan, g);
                 nx.n = nx.u.n0 + g - nx.u.g0;
                 if (nx.u.recv >= 0) slot_prefetch(p.slots + (size_t)nx.u.recv * kSlotBytes, tid);
@@ -548,7 +548,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     }
                 }
             }
-            if (!p.tied) {
+            if (!kTied) {
                 if (!(ok = mbar_wait(&bar.full_k, j & 1, limit, abort_flag, p.status))) break;
 #pragma unroll
                 for (int r8 = 8; r8 >= 0; r8 -= 8) {
@@ -598,7 +598,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     // the other pipeline is done with chunk g - 1 (its j index: j for X = 1, j - 1 for X = 0)
                     if (!mbar_wait(&other.state_ready, (j - 1 + X) & 1, limit, abort_flag, p.status)) return false;
                 }
-                if (g == u.g0) {
+                if (__builtin_expect(g == u.g0, 0)) {      // (rare: a unit starts)
                     if (u.recv < 0) {
                         // a chain starts: the caller's state or zero
 #pragma unroll
@@ -626,7 +626,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     }
                     given_up = *reinterpret_cast<volatile int*>(&sm.given_up) == u.chain;
                 }
-                if (too_strong && !given_up) {
+                if (__builtin_expect(too_strong && !given_up, 0)) {
                     given_up = true;
                     if (tid == 0) p.redo[u.chain] = 1;
                 }
@@ -687,7 +687,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                          st[4 * k + 3]);
                 }
             }
-            if (g == u.g1 - 1) {
+            if (__builtin_expect(g == u.g1 - 1, 0)) {      // (rare: a unit ends)
                 if (u.send < 0) {
                     // the chain ends: its final state (a chain that was given up keeps its hands off:
                     // state_out may alias state_in, which the kernel that redoes the chain reads)
@@ -730,7 +730,7 @@ prefill_gated_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(&bar.st_ready);
-            if (more && !swept) {
+            if (__builtin_expect(more && !swept, 0)) {
                 if (!(ok = mbar_wait(&bar.full_gq, (j + 1) & 1, limit, abort_flag, p.status))) break;
                 first_sweep(dec_next);
             }
@@ -776,7 +776,6 @@ cudaError_t launch_prefill_gated_pair(const KernelArgs& a, const void* gate, int
     GatedPairParams p;
     p.B = a.B; p.T = a.T; p.H = a.H;
     p.grid_w = a.grid_w; p.prefix_len = a.prefix_len; p.t0 = a.t0; p.scale = a.scale;
-    p.tied = a.k ? 0 : 1;
     p.state_in = a.state_in; p.state_out = a.state_out;
     p.redo = redo;
     p.work = a.work;
@@ -786,9 +785,11 @@ cudaError_t launch_prefill_gated_pair(const KernelArgs& a, const void* gate, int
     p.status = a.status; p.wait_limit = a.wait_limit;
     p.norm_eps = a.norm_eps;
     const size_t smem = sizeof(Smem) + 1024;
-    auto* kernel = a.fused ? prefill_gated_pair_kernel<true> : prefill_gated_pair_kernel<false>;
-    static bool smem_ok[2][64];      // one set of flags per kernel variant
-    cudaError_t e = allow_dynamic_smem(kernel, smem, smem_ok[a.fused ? 1 : 0]);
+    const bool tied = a.k == nullptr;
+    auto* kernel = a.fused ? (tied ? prefill_gated_pair_kernel<true, true> : prefill_gated_pair_kernel<true, false>)
+                           : (tied ? prefill_gated_pair_kernel<false, true> : prefill_gated_pair_kernel<false, false>);
+    static bool smem_ok[4][64];      // one set of flags per kernel variant
+    cudaError_t e = allow_dynamic_smem(kernel, smem, smem_ok[(a.fused ? 2 : 0) + (tied ? 1 : 0)]);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(chains < sms ? chains : sms);
     // programmatic dependent launch, as in launch_prefill_pair

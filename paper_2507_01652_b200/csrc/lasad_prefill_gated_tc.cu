@@ -586,7 +586,7 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             //      thread's row, kept inside this warp's half of S's columns) -------------------------
             if (!(ok = mbar_wait(&sm.bar.s_done, n & 1, limit, abort_flag, p.status))) break;
             tc_fence_after();
-#pragma unroll 1
+#pragma unroll
             for (int pi = 0; pi < 2; ++pi) {
                 const int pc = 2 * grp + pi;
                 uint32_t pk[16];

@@ -455,7 +455,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     //      32-column blocks 2 grp and 2 grp + 1 of its rows and keeps the result inside
                     //      its own half of S's columns (block pc -> columns 64 grp + 16 (pc & 1), always
                     //      behind this warp's own reads); the A V~ MMAs walk the columns in that order.
-#pragma unroll 1
+#pragma unroll
                     for (int pi = 0; pi < 2; ++pi) {
                         const int pc = 2 * grp + pi;
                         uint32_t pk[16];

@@ -77,6 +77,28 @@ def test_fused_prefill_both_implementations_and_gates_close_to_one(ctx, T, w):
         assert rel_err(s, s_ref) <= TOL[torch.bfloat16], impl
 
 
+@pytest.mark.parametrize("H,T,tied", [(160, 1100, True), (151, 1300, False)])
+def test_fused_balanced_prefill_with_states_crossing_ctas(ctx, H, T, tied):
+    """The fused form on the balanced kernel (option 5) with more chains than SMs: left-over chains
+    are cut into pieces whose state crosses CTAs; an incoming state, a prefix token, a start in
+    mid-row; twice in a row (the hand-off packets of the first call must not pass for the second's)."""
+    B, d, w = 1, 64, 11
+    q, k, v, g = _pre(2300 + H, B, T, H, d, torch.bfloat16)
+    s_in = torch.randn(B, H, d, d, generator=torch.Generator().manual_seed(H)) * 0.2
+    o_ref, s_ref = _oracle(q, None if tied else k, v, g, w, 1, 7, 0.5, s_in, 1e-6)
+    dq, dk, dv, dg, ds = q.cuda(), (None if tied else k.cuda()), v.cuda(), g.cuda(), s_in.cuda()
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 5)
+    try:
+        for rep in range(2):
+            o, s = ctx.lasad_forward_fused(dq, dk, dv, dg, w, prefix_len=1, t0=7, scale=0.5, state_in=ds)
+            torch.cuda.synchronize()
+            assert ctx.device_status() == 0
+            assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+            assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
+    finally:
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
+
+
 def test_fused_prefill_strong_decay_takes_the_exact_path(ctx):
     """Gate pre-activations far below zero (lambda down to e^-20): the tensor-core kernel gives such
     chains up and the CUDA-core kernel behind it computes them; the entry point stays exact."""

@@ -157,6 +157,19 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_v)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_o)) : "memory");
+        // The CTAs' first chains are chains 0 .. gridDim.x - 1 in some order (which CTA takes which
+        // is known only after the ticket): ask for the first chunks of chain blockIdx.x to be brought
+        // into L2 now, while the launch before this one is still finishing.  A prefetch hands no
+        // data to the SM, so it may run ahead of the wait below; whoever takes the chain finds its
+        // first tiles in L2.
+        if (X == 0) {
+            const int pb = (int)blockIdx.x / p.H, ph = (int)blockIdx.x - pb * p.H;
+            for (int n = 0; n < min(2 * kStages, p.nc); ++n) {
+                tma_prefetch_4d(&tm_k, 0, ph, n * kC, pb);
+                tma_prefetch_4d(&tm_v, 0, ph, n * kC, pb);
+                tma_prefetch_4d(&tm_q, 0, ph, n * kC, pb);
+            }
+        }
     }
     if (threadIdx.x >> 5 == 8) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),

@@ -89,8 +89,9 @@ cudaError_t launch_decode(const KernelArgs& a, int dk, int dv, bool bf16, bool d
 cudaError_t launch_decode_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, bool decay_on, int tpu,
                                 cudaStream_t st);
 // `only` (device, [B*H], or null): compute just the chains whose entry is non-zero, and put those
-// entries back to zero.
-cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, int* only,
+// entries back to zero.  `early`: launch as a programmatic dependent of the kernel before it in the
+// stream (the kernel waits for that one's completion before it reads anything).
+cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, int* only, bool early,
                                  cudaStream_t st);
 // Balanced tensor-core form of the gated prefill (one CTA per SM, two chunk pipelines on one chain;
 // bf16, dk = dv = 64).  redo ([B*H], zero on entry): set to 1 for every chain given up; the caller

@@ -24,6 +24,10 @@ constexpr float kMinLog2 = -150.0f;
 template <typename T, int D>
 __global__ void __launch_bounds__(256) prefill_gated_kernel(KernelArgs a, const void* gate_v, int* only)
 {
+    // Launched as a programmatic dependent: the kernel behind this one may take SMs early, and this
+    // one waits here for the kernel before it (whose marks and outputs it reads) to have completed.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // behind the tensor-core kernel: only the chains it gave up are computed here
     if (only && only[blockIdx.x] == 0) return;
     constexpr int LD = D + 1;
@@ -156,21 +160,32 @@ __global__ void __launch_bounds__(256) prefill_gated_kernel(KernelArgs a, const 
 }
 
 template <typename T, int D>
-cudaError_t launch_gated_t(const KernelArgs& a, const void* gate, int* only, cudaStream_t st)
+cudaError_t launch_gated_t(const KernelArgs& a, const void* gate, int* only, bool early, cudaStream_t st)
 {
     const size_t smem = sizeof(float) * D * (D + 1);
-    prefill_gated_kernel<T, D><<<(unsigned)(a.B * a.H), 256, smem, st>>>(a, gate, only);
-    return cudaGetLastError();
+    // (`early`: a programmatic dependent launch; behind the CTA-per-chain tensor-core kernel the
+    // launch latency then overlaps that kernel's tail)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(a.B * a.H));
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = early ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, prefill_gated_kernel<T, D>, a, gate, only);
 }
 
 }  // namespace
 
-cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, int* only,
+cudaError_t launch_prefill_gated(const KernelArgs& a, const void* gate, int dk, bool bf16, int* only, bool early,
                                  cudaStream_t st)
 {
     if (dk == 64)
-        return bf16 ? launch_gated_t<__nv_bfloat16, 64>(a, gate, only, st) : launch_gated_t<float, 64>(a, gate, only, st);
-    return bf16 ? launch_gated_t<__nv_bfloat16, 32>(a, gate, only, st) : launch_gated_t<float, 32>(a, gate, only, st);
+        return bf16 ? launch_gated_t<__nv_bfloat16, 64>(a, gate, only, early, st) : launch_gated_t<float, 64>(a, gate, only, early, st);
+    return bf16 ? launch_gated_t<__nv_bfloat16, 32>(a, gate, only, early, st) : launch_gated_t<float, 32>(a, gate, only, early, st);
 }
 
 }  // namespace lasad

@@ -161,6 +161,9 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     const unsigned limit = p.wait_limit;
 
     // ---- set-up ---------------------------------------------------------------------------
+    // A kernel launched behind this one as a programmatic dependent may start to take SMs as they
+    // become free; it waits for this kernel's completion before it touches device memory.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) {
         mbar_init(&sm.bar.full_in, 1);
         mbar_init(&sm.bar.full_v, 1);
@@ -176,6 +179,9 @@ prefill_gated_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         mbar_init(&sm.bar.st_ready, kEThreads);
         mbar_init(&sm.bar.drain, 1);
         sm.abort_flag = 0;
+        // nothing above reads or writes device memory; everything below may depend on the kernel
+        // before this one in the stream
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 8) {
@@ -689,8 +695,18 @@ cudaError_t launch_prefill_gated_tc(const KernelArgs& a, const void* gate, int* 
     static bool smem_ok[2][64];      // one set of flags per kernel variant
     cudaError_t e = allow_dynamic_smem(kernel, smem, smem_ok[a.fused ? 1 : 0]);
     if (e != cudaSuccess) return e;
-    kernel<<<(unsigned)(a.B * a.H), kThreads, smem, st>>>(mq, mk, mv, mg, mo, p);
-    return cudaGetLastError();
+    // programmatic dependent launch (see the kernel's first lines)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(a.B * a.H));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mg, mo, p);
 }
 
 }  // namespace lasad

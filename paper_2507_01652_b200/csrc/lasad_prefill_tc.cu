@@ -122,6 +122,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const unsigned limit = p.wait_limit;
 
     // ---- set-up ---------------------------------------------------------------------------
+    // A kernel launched behind this one as a programmatic dependent may start to take SMs as they
+    // become free; it waits for this kernel's completion before it touches device memory.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!kSegments && warp == 9 && lane == 0) {
+        // the CTA's first chain is chain blockIdx.x: ask for its first chunks to be brought into L2
+        // now, while the launch before this one may still be finishing (a prefetch hands no data to
+        // the SM, so it may run ahead of the wait below)
+        const int pb = (int)blockIdx.x / p.H, ph = (int)blockIdx.x - pb * p.H;
+        for (int n = 0; n < min(kStages, (p.T + kC - 1) / kC); ++n) {
+            tma_prefetch_4d(&tm_k, 0, ph, n * kC, pb);
+            tma_prefetch_4d(&tm_v, 0, ph, n * kC, pb);
+            tma_prefetch_4d(&tm_q, 0, ph, n * kC, pb);
+        }
+    }
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) mbar_init(&sm.bar.full[s], 1);
         mbar_init(&sm.bar.s_done, 1);
@@ -136,6 +150,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_init(&sm.bar.drain, 1);
         sm.abort_flag = 0;
         sm.ring[0] = (int)blockIdx.x;     // the CTA's first chain; later ones come from the work counter
+        // nothing above reads or writes device memory; everything below may depend on the kernel
+        // before this one in the stream (its outputs, the work counter it puts back to zero)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 8) {
@@ -916,11 +933,25 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, int sms, cudaStream_t st)
     }
     const long long units = chains * p.n_segs;
     const unsigned grid = (unsigned)(units < 2LL * sms ? units : 2LL * sms);
-    if (p.n_segs > 1)
+    if (p.n_segs > 1) {
         prefill_tc_kernel<true><<<grid, kThreads, smem, st>>>(mq, mk, mv, mo, p);
-    else
-        prefill_tc_kernel<false><<<grid, kThreads, smem, st>>>(mq, mk, mv, mo, p);
-    return cudaGetLastError();
+        return cudaGetLastError();
+    }
+    // Whole chains: a programmatic dependent launch, as for the balanced kernel (its CTAs set up, and
+    // ask for their first tiles in L2, on SMs the launch before has left; they read nothing from
+    // device memory before griddepcontrol.wait).  After a kernel that does not let its dependents
+    // go early the launch behaves like an ordinary one.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<false>, mq, mk, mv, mo, p);
 }
 
 }  // namespace lasad

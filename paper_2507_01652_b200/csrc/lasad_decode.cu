@@ -59,6 +59,12 @@ __global__ void __launch_bounds__(256) decode_kernel(KernelArgs a, int decay_on,
 
     __shared__ float red[UPC][WPU > 1 ? WPU : 1][D];
 
+    // Launched as a programmatic dependent: the kernel behind this one (the next step, as a rule)
+    // may bring its CTAs onto the SMs while this one runs, and this one waits here for the kernel
+    // before it (whose state it reads) to have completed.  Nothing above touches device memory.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     const int tid = threadIdx.x;
     const int lt = tid % TPU;
     const int cg = lt % CG;
@@ -180,10 +186,20 @@ cudaError_t launch_decode_t(const KernelArgs& a, bool decay_on, int tpu, const v
 {
     const long long n_units = (long long)a.B * a.H;
     const int on = decay_on ? 1 : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaSuccess;
 #define LASAD_DECODE_CASE(TPU_)                                                               \
     case TPU_: {                                                                              \
         const long long blocks = (n_units + (256 / TPU_) - 1) / (256 / TPU_);                 \
-        decode_kernel<T, D, TPU_, GATED, POS, FUSED><<<(unsigned)blocks, 256, 0, st>>>(a, on, gate); \
+        cfg.gridDim = dim3((unsigned)blocks);                                                 \
+        e = cudaLaunchKernelEx(&cfg, decode_kernel<T, D, TPU_, GATED, POS, FUSED>, a, on, gate); \
         break;                                                                                \
     }
     switch (tpu) {
@@ -194,7 +210,7 @@ cudaError_t launch_decode_t(const KernelArgs& a, bool decay_on, int tpu, const v
         default: return cudaErrorInvalidValue;
     }
 #undef LASAD_DECODE_CASE
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace

@@ -45,6 +45,11 @@ __global__ void __launch_bounds__(256) prefill_simt_kernel(KernelArgs a, SimtSeg
     constexpr int CT = D / 16;           // channel columns per thread (16 column-threads)
     constexpr int JT = C / 16;           // score columns per thread
     constexpr int ST = D / 16;           // state rows per thread
+    // Launched as a programmatic dependent: the kernel behind this one (the main pass behind the
+    // state pass, the next call behind this one) may bring its CTAs onto the SMs early; this one
+    // waits for the kernel before it to have completed before it touches device memory.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     extern __shared__ float smem[];
     float* Qs = smem;                    // [C][LD]
     float* Ks = Qs + C * LD;             // [C][LD]
@@ -239,13 +244,22 @@ cudaError_t launch_simt_t(const KernelArgs& a, float* scratch, size_t scratch_fl
     sg.n_segs = scratch ? simt_segments(n_chunks, chains, sms, scratch_floats, D) : 1;
     sg.seg_chunks = sg.n_segs > 1 ? (n_chunks + sg.n_segs - 1) / sg.n_segs : n_chunks;
     sg.scratch = scratch;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (sg.n_segs > 1) {
-        prefill_simt_kernel<T, D, C, true><<<(unsigned)(chains * (sg.n_segs - 1)), 256, smem, st>>>(a, sg);
-        e = cudaGetLastError();
+        cfg.gridDim = dim3((unsigned)(chains * (sg.n_segs - 1)));
+        e = cudaLaunchKernelEx(&cfg, prefill_simt_kernel<T, D, C, true>, a, sg);
         if (e != cudaSuccess) return e;
     }
-    prefill_simt_kernel<T, D, C, false><<<(unsigned)(chains * sg.n_segs), 256, smem, st>>>(a, sg);
-    return cudaGetLastError();
+    cfg.gridDim = dim3((unsigned)(chains * sg.n_segs));
+    return cudaLaunchKernelEx(&cfg, prefill_simt_kernel<T, D, C, false>, a, sg);
 }
 
 template <typename T, int D>

@@ -664,6 +664,11 @@ __global__ void __launch_bounds__(kThreads, 2)
 prefill_seg_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, TcParams p,
                          SegSteps steps, float* seg_state, int* seg_count)
 {
+    // Launched as a programmatic dependent: the kernel behind this one (the segment pass) may bring
+    // its CTAs onto the SMs early; this one waits for the kernel before it to have completed before
+    // it touches device memory.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     extern __shared__ unsigned char smem_raw[];
     StateSmem& sm = *reinterpret_cast<StateSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x;
@@ -925,22 +930,26 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, int sms, cudaStream_t st)
             }
             // the per-chain counters sit behind the 2 x SMs state slots
             int* seg_count = reinterpret_cast<int*>(a.seg_state + (size_t)2 * sms * kD * kD);
-            prefill_seg_state_kernel<<<(unsigned)(chains * (segs - 1)), kThreads, ssmem, st>>>(mk, mv, p, steps, a.seg_state,
-                                                                                              seg_count);
-            e = cudaGetLastError();
+            cudaLaunchConfig_t scfg = {};
+            scfg.gridDim = dim3((unsigned)(chains * (segs - 1)));
+            scfg.blockDim = dim3(kThreads);
+            scfg.dynamicSmemBytes = ssmem;
+            scfg.stream = st;
+            cudaLaunchAttribute sattr[1];
+            sattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            sattr[0].val.programmaticStreamSerializationAllowed = 1;
+            scfg.attrs = sattr;
+            scfg.numAttrs = 1;
+            e = cudaLaunchKernelEx(&scfg, prefill_seg_state_kernel, mk, mv, p, steps, a.seg_state, seg_count);
             if (e != cudaSuccess) return e;
         }
     }
     const long long units = chains * p.n_segs;
     const unsigned grid = (unsigned)(units < 2LL * sms ? units : 2LL * sms);
-    if (p.n_segs > 1) {
-        prefill_tc_kernel<true><<<grid, kThreads, smem, st>>>(mq, mk, mv, mo, p);
-        return cudaGetLastError();
-    }
-    // Whole chains: a programmatic dependent launch, as for the balanced kernel (its CTAs set up, and
-    // ask for their first tiles in L2, on SMs the launch before has left; they read nothing from
-    // device memory before griddepcontrol.wait).  After a kernel that does not let its dependents
-    // go early the launch behaves like an ordinary one.
+    // A programmatic dependent launch, as for the balanced kernel (its CTAs set up -- and, with whole
+    // chains, ask for their first tiles in L2 -- on SMs the launch before has left; they read
+    // nothing from device memory before griddepcontrol.wait).  After a kernel that does not let its
+    // dependents go early the launch behaves like an ordinary one.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kThreads);
@@ -951,7 +960,8 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, int sms, cudaStream_t st)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<false>, mq, mk, mv, mo, p);
+    return p.n_segs > 1 ? cudaLaunchKernelEx(&cfg, prefill_tc_kernel<true>, mq, mk, mv, mo, p)
+                        : cudaLaunchKernelEx(&cfg, prefill_tc_kernel<false>, mq, mk, mv, mo, p);
 }
 
 }  // namespace lasad

@@ -32,11 +32,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) from the ncu captures
 # summarised under profiles/; None until a capture of that kernel exists.
 NCU_TRAFFIC_BYTES = {
-    # prefill_pair_kernel (the default on config 5b): 384.9 MB measured on the 405.8 MB capture case
+    # prefill_pair_kernel (the default on config 5b): 385.4 MB measured on the 405.8 MB capture case
     # (config 5a), scaled by tokens to config 5b
-    "prefill": 861_900_000,
+    "prefill": 863_400_000,
     # decode_kernel, config 4, inside the kernel (the rest of the written state drains from L2 later)
-    "decode": 111_800_000,
+    "decode": 112_500_000,
 }
 
 

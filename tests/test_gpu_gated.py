@@ -172,6 +172,38 @@ def test_gated_state_handoff(ctx):
         assert rel_err(s2, s_ref) <= TOL[torch.bfloat16]
 
 
+@pytest.mark.parametrize("impl", [2, 5])
+def test_gated_dependent_calls_enqueued_without_a_synchronise_in_between(ctx, impl):
+    """As the test of the same name for the scalar decay: the gated kernels (and the CUDA-core kernel
+    launched behind them) are programmatic dependents of whatever precedes them; three calls on 160
+    sequences, each from the state the call before leaves, with a gated decode step in between and
+    nothing else on the stream."""
+    B, H, T, d, w = 1, 160, 1501, 64, 11
+    gen = torch.Generator().manual_seed(94)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+    lam = torch.sigmoid(2.0 + torch.randn(B, T, H, d, generator=gen)).to(torch.bfloat16)
+    o_ref, s_ref = oracle(q, k, v, lam, w)
+    dq, dk_, dv_, dl = _dev(q, k, v, lam)
+    a, b = 500, 1000
+    o = torch.empty_like(dv_)
+    s = torch.empty(B, H, d, d, device="cuda")
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, impl)
+    try:
+        for rep in range(2):
+            ctx.lasad_forward_gated(dq[:, :a], dk_[:, :a], dv_[:, :a], dl[:, :a], w, o=o[:, :a], state_out=s)
+            ctx.lasad_forward_gated(dq[:, a:b], dk_[:, a:b], dv_[:, a:b], dl[:, a:b], w, t0=a, o=o[:, a:b], state_in=s,
+                                    state_out=s)
+            ctx.lasad_decode_step_gated(dq[:, b], dk_[:, b], dv_[:, b], dl[:, b], s, w, 0, b, o=o[:, b])
+            ctx.lasad_forward_gated(dq[:, b + 1:], dk_[:, b + 1:], dv_[:, b + 1:], dl[:, b + 1:], w, t0=b + 1,
+                                    o=o[:, b + 1:], state_in=s, state_out=s)
+            torch.cuda.synchronize()
+            assert ctx.device_status() == 0
+            assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+            assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
+    finally:
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
+
+
 @pytest.mark.parametrize("impl,H", [(2, 3), (5, 3), (5, 80)])
 def test_gated_prefill_recorded_into_a_cuda_graph_and_replayed(ctx, impl, H):
     """Both launches of the gated prefill (tensor-core kernel, CUDA-core kernel for flagged chains)

@@ -175,6 +175,39 @@ def test_state_handoff_mid_row(ctx, impl):
         assert rel_err(s2, s_ref) <= TOL[torch.bfloat16]
 
 
+@pytest.mark.parametrize("impl", [1, 2, 5])
+def test_dependent_calls_enqueued_without_a_synchronise_in_between(ctx, impl):
+    """The kernels are launched as programmatic dependents: a call's CTAs may come onto the SMs while
+    the call before it is still running, and must wait for it before they read what it wrote.  Three
+    calls are enqueued back to back on one stream with nothing in between -- the first third of 160
+    sequences, the second third from the state the first call leaves (in place), then one decode
+    step per sequence on that state, and the last third -- large enough for each call to find its
+    predecessor still at work; outputs and final state against the oracle on the whole sequence."""
+    B, H, T, d, w = 1, 160, 2101, 64, 11
+    gen = torch.Generator().manual_seed(93)
+    q, k, v = [(torch.randn(B, T, H, d, generator=gen) / 8).to(torch.bfloat16) for _ in range(3)]
+    g = 0.9 + 0.0999 * torch.rand(H, generator=gen)
+    o_ref, s_ref = oracle(q, k, v, g, w)
+    dq, dk, dv, dg = _dev(q, k, v, g)
+    a, b = 700, 1400
+    o = torch.empty_like(dv)
+    s = torch.empty(B, H, d, d, device="cuda")
+    ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, impl)
+    try:
+        for rep in range(2):
+            ctx.lasad_forward(dq[:, :a], dk[:, :a], dv[:, :a], dg, w, o=o[:, :a], state_out=s)
+            ctx.lasad_forward(dq[:, a:b], dk[:, a:b], dv[:, a:b], dg, w, t0=a, o=o[:, a:b], state_in=s, state_out=s)
+            ctx.lasad_decode_step(dq[:, b], dk[:, b], dv[:, b], dg, s, w, 0, b, o=o[:, b])
+            ctx.lasad_forward(dq[:, b + 1:], dk[:, b + 1:], dv[:, b + 1:], dg, w, t0=b + 1, o=o[:, b + 1:], state_in=s,
+                              state_out=s)
+            torch.cuda.synchronize()
+            assert ctx.device_status() == 0
+            assert rel_err(o, o_ref) <= TOL[torch.bfloat16], rep
+            assert rel_err(s, s_ref) <= TOL[torch.bfloat16], rep
+    finally:
+        ctx.set_option(binding.LASAD_OPT_PREFILL_IMPL, 0)
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 def test_head_major_layout_through_strides(ctx, impl):
     """[B,H,T,d] storage viewed as [B,T,H,d]: only the strides change."""

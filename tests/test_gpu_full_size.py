@@ -61,6 +61,30 @@ def test_gated_prefill_full_size_sampled_chains(ctx, name):
         assert rel_err(s[b:b + 1, h:h + 1], s_ref) <= TOL[torch.bfloat16], (b, h)
 
 
+@pytest.mark.parametrize("name", ["config3", "config5b"])
+def test_fused_prefill_full_size_sampled_chains(ctx, name):
+    """The fused call (Algorithm 1's loop body: SiLU, Sigmoid, key tied to the gate, operator, RMS
+    norm) as bench.py times it -- pre-activations q~ ~ N(0,1), gate~ ~ N(2,1), the workload's v --
+    on sampled chains against the oracle's layer_core."""
+    from oracle import lasad_oracle as orc
+    from tests._util import to64
+    wl = workloads.WORKLOADS[name]
+    gen = torch.Generator().manual_seed(wl.seed + 11)
+    qp = torch.randn(wl.B, wl.T, wl.H, wl.d, generator=gen).to(torch.bfloat16)
+    gp = (torch.randn(wl.B, wl.T, wl.H, wl.d, generator=gen) + 2.0).to(torch.bfloat16)
+    v = workloads.make_qkv(wl)[2]
+    o, s = ctx.lasad_forward_fused(qp.cuda(), None, v.cuda(), gp.cuda(), wl.grid_w, prefix_len=wl.prefix_len)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    o, s = o.cpu(), s.cpu()
+    for b, h in _sampled_chains(wl, 4):
+        sl = (slice(b, b + 1), slice(None), slice(h, h + 1))
+        o_ref, s_ref = orc.layer_core(to64(qp[sl]), None, to64(v[sl]), to64(gp[sl]), wl.grid_w, wl.prefix_len, 0, 1.0, None,
+                                      1e-6)
+        assert rel_err(o[sl], o_ref) <= TOL[torch.bfloat16], (b, h)
+        assert rel_err(s[b:b + 1, h:h + 1], s_ref) <= TOL[torch.bfloat16], (b, h)
+
+
 def test_decode_full_size_config4_sampled_chains(ctx):
     """Config 4 as the bench runs it: one prefill call for the class token, then one decode step per
     grid token (all 256 of them) on all 256 x 20 states; sampled chains against the oracle over the

@@ -160,6 +160,9 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     const unsigned limit = p.wait_limit;
 
     // ---- set-up ---------------------------------------------------------------------------
+    // A kernel launched behind this one as a programmatic dependent may start to take SMs as they
+    // become free; it waits for this kernel's completion before it touches device memory.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) mbar_init(&sm.bar.full[s], 1);
         mbar_init(&sm.bar.s_done, 1);
@@ -181,6 +184,9 @@ prefill_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    // nothing above reads or writes device memory; everything below may depend on the kernel before
+    // this one in the stream
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (p.H <= kHeadCache) {
         for (int hh = tid; hh < p.H; hh += kThreads) {
             const float gm = p.decay[hh];
@@ -708,8 +714,18 @@ cudaError_t launch_prefill_stream(const KernelArgs& a, const TcRelay& r, cudaStr
     cudaError_t e = allow_dynamic_smem(prefill_stream_kernel, smem, smem_ok_1);
     if (e != cudaSuccess) return e;
     const int grid = p.n_tasks < r.max_ctas ? p.n_tasks : r.max_ctas;
-    prefill_stream_kernel<<<(unsigned)grid, kThreads, smem, st>>>(mq, mk, mv, mo, p);
-    return cudaGetLastError();
+    // programmatic dependent launch (see the kernel's first lines)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prefill_stream_kernel, mq, mk, mv, mo, p);
 }
 
 }  // namespace lasad

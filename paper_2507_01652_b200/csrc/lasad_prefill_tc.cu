@@ -129,8 +129,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // the CTA's first chain is chain blockIdx.x: ask for its first chunks to be brought into L2
         // now, while the launch before this one may still be finishing (a prefetch hands no data to
         // the SM, so it may run ahead of the wait below)
+        // (a short chain whole, of a longer one what the stages hold: asking for more than that of
+        // long chains measured slower)
         const int pb = (int)blockIdx.x / p.H, ph = (int)blockIdx.x - pb * p.H;
-        for (int n = 0; n < min(kStages, (p.T + kC - 1) / kC); ++n) {
+        const int nc = (p.T + kC - 1) / kC;
+        for (int n = 0; n < (nc <= 5 ? nc : kStages); ++n) {
             tma_prefetch_4d(&tm_k, 0, ph, n * kC, pb);
             tma_prefetch_4d(&tm_v, 0, ph, n * kC, pb);
             tma_prefetch_4d(&tm_q, 0, ph, n * kC, pb);

